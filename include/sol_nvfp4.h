@@ -1,0 +1,158 @@
+/*
+ * sol_nvfp4.h -- C ABI of the B200 (sm_100a) NVFP4 linear-layer library.
+ *
+ * The library computes the W4A4 linear layers of a diffusion-transformer rollout:
+ *     Y = Q(X) . Q(W)^T + bias
+ * where Q is the NVFP4 quantizer of the paper's Section 2 ("FP4 Quantization and
+ * Hardware Acceleration"):  x~ = S * Pi_FP4(x / S), FP4 = E2M1 (1 sign, 2 exponent,
+ * 1 mantissa bit), one E4M3 scale per 16 contiguous elements along K.  S is split in two
+ * levels: the E4M3 block scale and one FP32 scale T per tensor.  A BF16 linear of the
+ * same shape is the full-precision reference the paper's second stage runs in.
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless its comment says host.  The caller owns
+ *     every buffer; the library allocates no device memory (it keeps a small host-side
+ *     cache of TMA descriptors and reads device properties once).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     All work is asynchronous on it; no call synchronises or reads device scalars on the
+ *     host.  T flows from kernel to kernel through device memory.
+ *   - Every function returns a sol_status_t; nothing throws.  Arguments are validated on
+ *     the host before anything is launched: on an error status no kernel was launched.
+ *   - Matrices are row-major with the K dimension contiguous: X is [M, K], W is [N, K]
+ *     (the nn.Linear convention), Y is [M, N].  ld* are row pitches in ELEMENTS.
+ *   - Requirements: M, N, K > 0; K % 32 == 0; N % 8 == 0; pointers 16-byte aligned; BF16
+ *     row pitches multiples of 8 elements.  Inputs must be finite.
+ *   - Only sm_100 devices are supported (SOL_ERR_UNSUPPORTED_ARCH otherwise); there is
+ *     no CPU path.
+ *
+ * NVFP4 storage
+ *   data   : uint8 [rows, K/2]; byte j of a row holds element 2j in its low nibble and
+ *            element 2j+1 in its high nibble; nibble = s e e m.
+ *   scales : uint8 E4M3 (unsigned use).  SOL_SF_ROW_MAJOR: [rows, K/16].
+ *            SOL_SF_SWIZZLED_128x4: 512-byte chunks of 128 rows x 4 blocks, chunk order
+ *            [ceil(rows/128)][ceil(K/64)]; inside a chunk the scale of (row r, block b) is at
+ *            (r%32)*16 + ((r%128)/32)*4 + b%4.  Padding bytes are written as 0.  This is
+ *            the layout the tensor core's scale-factor copy consumes; the GEMM entries
+ *            require it.
+ *   T      : one float; dequantized value = E2M1(nibble) * E4M3(scale) * T.
+ */
+#ifndef SOL_NVFP4_H_
+#define SOL_NVFP4_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SOL_OK = 0,
+    SOL_ERR_NULL_POINTER = 1,
+    SOL_ERR_BAD_SHAPE = 2,
+    SOL_ERR_ALIGNMENT = 3,
+    SOL_ERR_WORKSPACE_TOO_SMALL = 4,
+    SOL_ERR_UNSUPPORTED_ARCH = 5,
+    SOL_ERR_CUDA = 6,
+    SOL_ERR_TIMEOUT = 7,
+    SOL_ERR_BAD_LAYOUT = 8
+} sol_status_t;
+
+typedef enum { SOL_SF_ROW_MAJOR = 0, SOL_SF_SWIZZLED_128x4 = 1 } sol_sf_layout_t;
+
+/* Static, human-readable name of a status (host pointer, never NULL). */
+const char *sol_status_string(sol_status_t status);
+
+/* Bytes of packed FP4 data for a [rows, K] tensor: rows * K / 2.  0 on bad arguments. */
+size_t sol_nvfp4_data_bytes(int64_t rows, int64_t K);
+
+/* Bytes of the scale buffer in the given layout (swizzled: ceil(rows/128) * ceil(K/64) * 512).
+ * 0 on bad arguments. */
+size_t sol_nvfp4_scale_bytes(int64_t rows, int64_t K, sol_sf_layout_t layout);
+
+/* Bytes of workspace nvfp4_quantize_linear needs for an [M, K] activation: packed data,
+ * swizzled scales and one float, each region 256-byte aligned.  0 on bad arguments. */
+size_t sol_nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
+/*
+ * Per-tensor scale (second scaling level; the paper's single S is split so that block
+ * scales span E4M3's range):  T = max|x| / (6 * 448), or 1 for an all-zero tensor.
+ *   x                [rows, K] BF16, pitch ld
+ *   tensor_scale_out one float (device), overwritten
+ * The max is exact (order-independent), so the result is deterministic.
+ */
+sol_status_t sol_amax_bf16(const void *x, int64_t rows, int64_t K, int64_t ld,
+                           float *tensor_scale_out, void *stream);
+
+/*
+ * Activation quantizer, Section 2's Q(x) with S = block scale * T.  Per row and per block
+ * of 16 elements along K, in IEEE binary32 (round-to-nearest-even, no contraction):
+ *     a = max|x|;  sb = E4M3_rne_sat(a / (6*T));  rcp = 1 / (float(sb) * T)  (0 if sb == 0)
+ *     nibble_k = E2M1_rne_sat(x_k * rcp)   (ties to the even code, sign bit of x kept)
+ *   x_bf16       [M, K] BF16, pitch ldx
+ *   tensor_scale one float (device), read by the kernel; > 0
+ *   q_out        sol_nvfp4_data_bytes(M, K) bytes
+ *   sf_out       sol_nvfp4_scale_bytes(M, K, layout) bytes; every byte is written
+ */
+sol_status_t nvfp4_quantize(const void *x_bf16, int64_t M, int64_t K, int64_t ldx,
+                            const float *tensor_scale, void *q_out, void *sf_out,
+                            sol_sf_layout_t layout, void *stream);
+
+/*
+ * Weight quantizer: the same mapping applied to W [N, K] along K, preceded by the
+ * per-tensor scale of W (the paper re-quantizes the policy weights after each update,
+ * Section 3.4 / Appendix B.2).
+ *   tensor_scale_out one float (device), written by the first kernel, read by the second
+ */
+sol_status_t nvfp4_quantize_weight(const void *w_bf16, int64_t N, int64_t K, int64_t ldw,
+                                   void *q_out, void *sf_out, float *tensor_scale_out,
+                                   sol_sf_layout_t layout, void *stream);
+
+/*
+ * Block-scaled FP4 GEMM with BF16 output (the NVFP4 linear the rollout runs, Section 3.4):
+ *     acc[m,n] = sum_b sx[m,b] * sw[n,b] * sum_{k in b} qx[m,k] * qw[n,k]      (FP32 accumulate)
+ *     Y[m,n]   = bf16_rne( fma(acc, Tx*Tw, bias[n]) )
+ *   xq, wq     packed data [M, K/2], [N, K/2] (dense pitch K/2 bytes)
+ *   xsf, wsf   scales in SOL_SF_SWIZZLED_128x4 layout
+ *   x_tscale, w_tscale   one float each (device)
+ *   bias_bf16  [N] BF16 or NULL
+ *   y_bf16     [M, N] BF16, pitch ldy
+ */
+sol_status_t nvfp4_linear(const void *xq, const void *xsf, const float *x_tscale,
+                          const void *wq, const void *wsf, const float *w_tscale,
+                          const void *bias_bf16, void *y_bf16, int64_t M, int64_t N, int64_t K,
+                          int64_t ldy, void *stream);
+
+/*
+ * BF16 linear, the full-precision stage-2 reference (Section 3.4):
+ *     Y[m,n] = bf16_rne( sum_k x[m,k] * w[n,k] + bias[n] ),  FP32 accumulate.
+ */
+sol_status_t bf16_linear(const void *x_bf16, const void *w_bf16, const void *bias_bf16,
+                         void *y_bf16, int64_t M, int64_t N, int64_t K, int64_t ldx,
+                         int64_t ldw, int64_t ldy, void *stream);
+
+/*
+ * Fused entry: dynamic per-tensor scale of X, quantize X, NVFP4 GEMM against
+ * pre-quantized weights, in one call on one stream.
+ *   workspace  device scratch of at least sol_nvfp4_linear_workspace_bytes(M, N, K) bytes,
+ *              256-byte aligned; holds Q(X) between the kernels; contents undefined after.
+ */
+sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *wq,
+                                   const void *wsf, const float *w_tscale,
+                                   const void *bias_bf16, void *y_bf16, int64_t M, int64_t N,
+                                   int64_t K, int64_t ldy, void *workspace,
+                                   size_t workspace_bytes, void *stream);
+
+/*
+ * Device-side waits in the GEMM kernels are bounded; a wait that runs out records a code
+ * in a device status word and the kernel returns.  This call synchronises `stream`, reads
+ * that word, clears it, and returns SOL_ERR_TIMEOUT if it was set, SOL_ERR_CUDA if the
+ * stream reported an error, SOL_OK otherwise.  `detail_out` (host, nullable) receives the
+ * raw word.
+ */
+sol_status_t sol_last_device_status(void *stream, uint32_t *detail_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SOL_NVFP4_H_ */

@@ -1,0 +1,187 @@
+"""ctypes binding of the C-ABI CUDA library (``include/sol_nvfp4.h``).
+
+Argument marshalling only: torch supplies device memory and the current stream, every
+compute step runs in the library's kernels.  There is no fallback: if the library is
+missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsol_nvfp4.so")
+
+SF_ROW_MAJOR = 0
+SF_SWIZZLED_128x4 = 1
+
+EXPORTS = [
+    "sol_status_string", "sol_nvfp4_data_bytes", "sol_nvfp4_scale_bytes",
+    "sol_nvfp4_linear_workspace_bytes", "sol_amax_bf16", "nvfp4_quantize", "nvfp4_quantize_weight",
+    "nvfp4_linear", "bf16_linear", "nvfp4_quantize_linear", "sol_last_device_status",
+]
+
+_lib = None
+
+
+class SolError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2604_06916_b200.build` "
+            "(there is no CPU or PyTorch fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i64, sz, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_int
+    L.sol_status_string.restype, L.sol_status_string.argtypes = ctypes.c_char_p, [i32]
+    L.sol_nvfp4_data_bytes.restype, L.sol_nvfp4_data_bytes.argtypes = sz, [i64, i64]
+    L.sol_nvfp4_scale_bytes.restype, L.sol_nvfp4_scale_bytes.argtypes = sz, [i64, i64, i32]
+    L.sol_nvfp4_linear_workspace_bytes.restype = sz
+    L.sol_nvfp4_linear_workspace_bytes.argtypes = [i64, i64, i64]
+    L.sol_amax_bf16.restype, L.sol_amax_bf16.argtypes = i32, [vp, i64, i64, i64, vp, vp]
+    L.nvfp4_quantize.restype, L.nvfp4_quantize.argtypes = i32, [vp, i64, i64, i64, vp, vp, vp, i32, vp]
+    L.nvfp4_quantize_weight.restype = i32
+    L.nvfp4_quantize_weight.argtypes = [vp, i64, i64, i64, vp, vp, vp, i32, vp]
+    L.nvfp4_linear.restype = i32
+    L.nvfp4_linear.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp]
+    L.bf16_linear.restype = i32
+    L.bf16_linear.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, vp]
+    L.nvfp4_quantize_linear.restype = i32
+    L.nvfp4_quantize_linear.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, sz, vp]
+    L.sol_last_device_status.restype = i32
+    L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return lib().sol_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise SolError(code, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def data_bytes(rows: int, K: int) -> int:
+    return lib().sol_nvfp4_data_bytes(rows, K)
+
+
+def scale_bytes(rows: int, K: int, layout: int = SF_SWIZZLED_128x4) -> int:
+    return lib().sol_nvfp4_scale_bytes(rows, K, layout)
+
+
+def linear_workspace_bytes(M: int, N: int, K: int) -> int:
+    return lib().sol_nvfp4_linear_workspace_bytes(M, N, K)
+
+
+def _need_2d_bf16(x: torch.Tensor, name: str):
+    if x.dtype != torch.bfloat16 or x.dim() != 2 or x.stride(1) != 1 or not x.is_cuda:
+        raise TypeError(f"{name}: expected a 2-D CUDA bf16 tensor with contiguous rows")
+
+
+def sol_amax_bf16(x: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Per-tensor scale T = max|x| / 2688 (1 for zeros) as a 1-element float32 device tensor."""
+    _need_2d_bf16(x, "x")
+    if out is None:
+        out = torch.empty(1, dtype=torch.float32, device=x.device)
+    _check(lib().sol_amax_bf16(_ptr(x), x.shape[0], x.shape[1], x.stride(0), _ptr(out), _stream()), "sol_amax_bf16")
+    return out
+
+
+def _alloc_q(rows: int, K: int, layout: int, device):
+    nq, ns = data_bytes(rows, K), scale_bytes(rows, K, layout)
+    if nq == 0 or ns == 0:
+        raise SolError(2, "shape check")
+    q = torch.empty((rows, K // 2), dtype=torch.uint8, device=device)
+    sf = torch.empty(ns, dtype=torch.uint8, device=device)
+    return q, sf
+
+
+def nvfp4_quantize(x: torch.Tensor, tensor_scale: torch.Tensor, layout: int = SF_SWIZZLED_128x4,
+                   out: tuple[torch.Tensor, torch.Tensor] | None = None):
+    """BF16 [M, K] -> (packed nibbles uint8 [M, K/2], E4M3 scales uint8 flat buffer)."""
+    _need_2d_bf16(x, "x")
+    M, K = x.shape
+    q, sf = out if out is not None else _alloc_q(M, K, layout, x.device)
+    _check(lib().nvfp4_quantize(_ptr(x), M, K, x.stride(0), _ptr(tensor_scale), _ptr(q), _ptr(sf), layout,
+                                _stream()), "nvfp4_quantize")
+    return q, sf
+
+
+def nvfp4_quantize_weight(w: torch.Tensor, layout: int = SF_SWIZZLED_128x4):
+    """BF16 [N, K] -> (packed nibbles, scales, per-tensor scale T_w)."""
+    _need_2d_bf16(w, "w")
+    N, K = w.shape
+    q, sf = _alloc_q(N, K, layout, w.device)
+    ts = torch.empty(1, dtype=torch.float32, device=w.device)
+    _check(lib().nvfp4_quantize_weight(_ptr(w), N, K, w.stride(0), _ptr(q), _ptr(sf), _ptr(ts), layout, _stream()),
+           "nvfp4_quantize_weight")
+    return q, sf, ts
+
+
+def nvfp4_linear(xq, xsf, x_tscale, wq, wsf, w_tscale, bias=None, out: torch.Tensor | None = None):
+    """Y = dequant(X) . dequant(W)^T + bias in BF16 from quantized operands (swizzled scales)."""
+    M, K = xq.shape[0], xq.shape[1] * 2
+    N = wq.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=xq.device)
+    _check(lib().nvfp4_linear(_ptr(xq), _ptr(xsf), _ptr(x_tscale), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
+                              _ptr(out), M, N, K, out.stride(0), _stream()), "nvfp4_linear")
+    return out
+
+
+def bf16_linear(x, w, bias=None, out: torch.Tensor | None = None):
+    """Y = X . W^T + bias, BF16 in / BF16 out, FP32 accumulation."""
+    _need_2d_bf16(x, "x")
+    _need_2d_bf16(w, "w")
+    M, K = x.shape
+    N = w.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    _check(lib().bf16_linear(_ptr(x), _ptr(w), _ptr(bias), _ptr(out), M, N, K, x.stride(0), w.stride(0),
+                             out.stride(0), _stream()), "bf16_linear")
+    return out
+
+
+def nvfp4_quantize_linear(x, wq, wsf, w_tscale, bias=None, workspace: torch.Tensor | None = None,
+                          out: torch.Tensor | None = None):
+    """Dynamic per-tensor scale + quantize X + NVFP4 GEMM against pre-quantized W, one call."""
+    _need_2d_bf16(x, "x")
+    M, K = x.shape
+    N = wq.shape[0]
+    if workspace is None:
+        workspace = torch.empty(linear_workspace_bytes(M, N, K), dtype=torch.uint8, device=x.device)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    _check(lib().nvfp4_quantize_linear(_ptr(x), x.stride(0), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
+                                       _ptr(out), M, N, K, out.stride(0), _ptr(workspace), workspace.numel(),
+                                       _stream()), "nvfp4_quantize_linear")
+    return out
+
+
+def sol_last_device_status() -> int:
+    """Synchronises the current stream; raises SolError if a bounded device wait ran out."""
+    detail = ctypes.c_uint32(0)
+    code = lib().sol_last_device_status(_stream(), ctypes.byref(detail))
+    if code != 0:
+        raise SolError(code, f"device status word 0x{detail.value:x}")
+    return 0

@@ -1,0 +1,265 @@
+// C-ABI entry points: argument validation, size queries, device checks, TMA descriptor
+// encoding.  Every compute step runs in the kernels of quantize.cu and gemm.cu.
+#include "sol_internal.h"
+
+#include <mutex>
+
+namespace sol {
+
+__device__ uint32_t g_status_word = 0;
+
+namespace {
+
+std::mutex g_mutex;
+DeviceInfo g_devices[64];
+uint32_t *g_status_ptr[64] = {};
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+EncodeTiledFn encode_fn() {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_encode == nullptr) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    return g_encode;
+}
+
+}  // namespace
+
+const DeviceInfo *current_device_info() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceInfo &d = g_devices[dev];
+    if (!d.ok) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return nullptr;
+        d.device = dev;
+        d.sm_count = prop.multiProcessorCount;
+        d.cc_major = prop.major;
+        d.cc_minor = prop.minor;
+        void *sym = nullptr;
+        if (cudaGetSymbolAddress(&sym, g_status_word) != cudaSuccess) return nullptr;
+        g_status_ptr[dev] = static_cast<uint32_t *>(sym);
+        d.ok = true;
+    }
+    return &d;
+}
+
+sol_status_t check_arch(const DeviceInfo **info_out) {
+    const DeviceInfo *d = current_device_info();
+    if (d == nullptr) {
+        cudaGetLastError();
+        return SOL_ERR_CUDA;
+    }
+    if (d->cc_major != 10) return SOL_ERR_UNSUPPORTED_ARCH;
+    *info_out = d;
+    return SOL_OK;
+}
+
+uint32_t *device_status_word() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    return g_status_ptr[dev];
+}
+
+bool make_tmap_2d(CUtensorMap *out, CUtensorMapDataType dtype, uint32_t elem_bytes, const void *base,
+                  uint64_t inner, uint64_t outer, uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer,
+                  CUtensorMapSwizzle swizzle) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    (void)elem_bytes;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {pitch_bytes};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(out, dtype, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+namespace {
+
+bool shape_ok(int64_t rows, int64_t K) {
+    return rows > 0 && K > 0 && K % 32 == 0 && rows <= (1LL << 30) && K <= (1LL << 24);
+}
+
+size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+
+}  // namespace
+}  // namespace sol
+
+using namespace sol;
+
+extern "C" {
+
+const char *sol_status_string(sol_status_t status) {
+    switch (status) {
+        case SOL_OK: return "SOL_OK";
+        case SOL_ERR_NULL_POINTER: return "SOL_ERR_NULL_POINTER";
+        case SOL_ERR_BAD_SHAPE: return "SOL_ERR_BAD_SHAPE";
+        case SOL_ERR_ALIGNMENT: return "SOL_ERR_ALIGNMENT";
+        case SOL_ERR_WORKSPACE_TOO_SMALL: return "SOL_ERR_WORKSPACE_TOO_SMALL";
+        case SOL_ERR_UNSUPPORTED_ARCH: return "SOL_ERR_UNSUPPORTED_ARCH";
+        case SOL_ERR_CUDA: return "SOL_ERR_CUDA";
+        case SOL_ERR_TIMEOUT: return "SOL_ERR_TIMEOUT";
+        case SOL_ERR_BAD_LAYOUT: return "SOL_ERR_BAD_LAYOUT";
+    }
+    return "SOL_ERR_UNKNOWN";
+}
+
+size_t sol_nvfp4_data_bytes(int64_t rows, int64_t K) {
+    if (!shape_ok(rows, K)) return 0;
+    return static_cast<size_t>(rows) * static_cast<size_t>(K / 2);
+}
+
+size_t sol_nvfp4_scale_bytes(int64_t rows, int64_t K, sol_sf_layout_t layout) {
+    if (!shape_ok(rows, K)) return 0;
+    if (layout == SOL_SF_ROW_MAJOR) return static_cast<size_t>(rows) * static_cast<size_t>(K / 16);
+    if (layout == SOL_SF_SWIZZLED_128x4)
+        return static_cast<size_t>(ceil_div(rows, 128)) * static_cast<size_t>(ceil_div(K, 64)) * 512;
+    return 0;
+}
+
+size_t sol_nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (!shape_ok(M, K) || N <= 0) return 0;
+    return align256(sol_nvfp4_data_bytes(M, K)) + align256(sol_nvfp4_scale_bytes(M, K, SOL_SF_SWIZZLED_128x4)) + 256;
+}
+
+sol_status_t sol_amax_bf16(const void *x, int64_t rows, int64_t K, int64_t ld, float *tensor_scale_out,
+                           void *stream) {
+    if (x == nullptr || tensor_scale_out == nullptr) return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(rows, K) || ld < K) return SOL_ERR_BAD_SHAPE;
+    if (!aligned16(x) || ld % 8 != 0 || (reinterpret_cast<uintptr_t>(tensor_scale_out) & 3u)) return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_amax(x, rows, K, ld, tensor_scale_out, static_cast<cudaStream_t>(stream), dev);
+}
+
+sol_status_t nvfp4_quantize(const void *x_bf16, int64_t M, int64_t K, int64_t ldx, const float *tensor_scale,
+                            void *q_out, void *sf_out, sol_sf_layout_t layout, void *stream) {
+    if (x_bf16 == nullptr || tensor_scale == nullptr || q_out == nullptr || sf_out == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(M, K) || ldx < K) return SOL_ERR_BAD_SHAPE;
+    if (layout != SOL_SF_ROW_MAJOR && layout != SOL_SF_SWIZZLED_128x4) return SOL_ERR_BAD_LAYOUT;
+    if (!aligned16(x_bf16) || !aligned16(q_out) || !aligned16(sf_out) || ldx % 8 != 0 ||
+        (reinterpret_cast<uintptr_t>(tensor_scale) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_quantize(x_bf16, M, K, ldx, tensor_scale, q_out, sf_out, layout, static_cast<cudaStream_t>(stream));
+}
+
+sol_status_t nvfp4_quantize_weight(const void *w_bf16, int64_t N, int64_t K, int64_t ldw, void *q_out,
+                                   void *sf_out, float *tensor_scale_out, sol_sf_layout_t layout, void *stream) {
+    if (w_bf16 == nullptr || tensor_scale_out == nullptr || q_out == nullptr || sf_out == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(N, K) || ldw < K) return SOL_ERR_BAD_SHAPE;
+    if (layout != SOL_SF_ROW_MAJOR && layout != SOL_SF_SWIZZLED_128x4) return SOL_ERR_BAD_LAYOUT;
+    if (!aligned16(w_bf16) || !aligned16(q_out) || !aligned16(sf_out) || ldw % 8 != 0 ||
+        (reinterpret_cast<uintptr_t>(tensor_scale_out) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = launch_amax(w_bf16, N, K, ldw, tensor_scale_out, s, dev);
+    if (st != SOL_OK) return st;
+    return launch_quantize(w_bf16, N, K, ldw, tensor_scale_out, q_out, sf_out, layout, s);
+}
+
+static sol_status_t check_linear_common(const void *bias, const void *y, int64_t M, int64_t N, int64_t K,
+                                        int64_t ldy) {
+    if (!shape_ok(M, K) || N <= 0 || N % 8 != 0 || N > (1LL << 24) || ldy < N) return SOL_ERR_BAD_SHAPE;
+    if (!aligned16(y) || ldy % 8 != 0 || (bias != nullptr && !aligned16(bias))) return SOL_ERR_ALIGNMENT;
+    return SOL_OK;
+}
+
+sol_status_t nvfp4_linear(const void *xq, const void *xsf, const float *x_tscale, const void *wq, const void *wsf,
+                          const float *w_tscale, const void *bias_bf16, void *y_bf16, int64_t M, int64_t N,
+                          int64_t K, int64_t ldy, void *stream) {
+    if (xq == nullptr || xsf == nullptr || x_tscale == nullptr || wq == nullptr || wsf == nullptr ||
+        w_tscale == nullptr || y_bf16 == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    sol_status_t st = check_linear_common(bias_bf16, y_bf16, M, N, K, ldy);
+    if (st != SOL_OK) return st;
+    if (!aligned16(xq) || !aligned16(xsf) || !aligned16(wq) || !aligned16(wsf) ||
+        (reinterpret_cast<uintptr_t>(x_tscale) & 3u) || (reinterpret_cast<uintptr_t>(w_tscale) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_gemm_nvfp4(xq, xsf, x_tscale, wq, wsf, w_tscale, bias_bf16, y_bf16, M, N, K, ldy,
+                             static_cast<cudaStream_t>(stream), dev);
+}
+
+sol_status_t bf16_linear(const void *x_bf16, const void *w_bf16, const void *bias_bf16, void *y_bf16, int64_t M,
+                         int64_t N, int64_t K, int64_t ldx, int64_t ldw, int64_t ldy, void *stream) {
+    if (x_bf16 == nullptr || w_bf16 == nullptr || y_bf16 == nullptr) return SOL_ERR_NULL_POINTER;
+    sol_status_t st = check_linear_common(bias_bf16, y_bf16, M, N, K, ldy);
+    if (st != SOL_OK) return st;
+    if (ldx < K || ldw < K) return SOL_ERR_BAD_SHAPE;
+    if (!aligned16(x_bf16) || !aligned16(w_bf16) || ldx % 8 != 0 || ldw % 8 != 0) return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_gemm_bf16(x_bf16, w_bf16, bias_bf16, y_bf16, M, N, K, ldx, ldw, ldy,
+                            static_cast<cudaStream_t>(stream), dev);
+}
+
+sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,
+                                   const float *w_tscale, const void *bias_bf16, void *y_bf16, int64_t M,
+                                   int64_t N, int64_t K, int64_t ldy, void *workspace, size_t workspace_bytes,
+                                   void *stream) {
+    if (x_bf16 == nullptr || wq == nullptr || wsf == nullptr || w_tscale == nullptr || y_bf16 == nullptr ||
+        workspace == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    sol_status_t st = check_linear_common(bias_bf16, y_bf16, M, N, K, ldy);
+    if (st != SOL_OK) return st;
+    if (ldx < K) return SOL_ERR_BAD_SHAPE;
+    if (!aligned16(x_bf16) || !aligned16(wq) || !aligned16(wsf) || ldx % 8 != 0 ||
+        (reinterpret_cast<uintptr_t>(w_tscale) & 3u) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return SOL_ERR_ALIGNMENT;
+    if (workspace_bytes < sol_nvfp4_linear_workspace_bytes(M, N, K)) return SOL_ERR_WORKSPACE_TOO_SMALL;
+    const DeviceInfo *dev = nullptr;
+    st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    uint8_t *xq = ws;
+    uint8_t *xsf = xq + align256(sol_nvfp4_data_bytes(M, K));
+    float *xts = reinterpret_cast<float *>(xsf + align256(sol_nvfp4_scale_bytes(M, K, SOL_SF_SWIZZLED_128x4)));
+    st = launch_amax(x_bf16, M, K, ldx, xts, s, dev);
+    if (st != SOL_OK) return st;
+    st = launch_quantize(x_bf16, M, K, ldx, xts, xq, xsf, SOL_SF_SWIZZLED_128x4, s);
+    if (st != SOL_OK) return st;
+    return launch_gemm_nvfp4(xq, xsf, xts, wq, wsf, w_tscale, bias_bf16, y_bf16, M, N, K, ldy, s, dev);
+}
+
+sol_status_t sol_last_device_status(void *stream, uint32_t *detail_out) {
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint32_t word = 0;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return SOL_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&word, g_status_word, sizeof(word)) != cudaSuccess) return SOL_ERR_CUDA;
+    if (detail_out != nullptr) *detail_out = word;
+    if (word != 0) {
+        const uint32_t zero = 0;
+        if (cudaMemcpyToSymbol(g_status_word, &zero, sizeof(zero)) != cudaSuccess) return SOL_ERR_CUDA;
+        return SOL_ERR_TIMEOUT;
+    }
+    return SOL_OK;
+}
+
+}  // extern "C"

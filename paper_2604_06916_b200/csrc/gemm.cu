@@ -1,0 +1,404 @@
+// Persistent, warp-specialised tcgen05 GEMM for sm_100a: Y[M,N] = A[M,K] . B[N,K]^T (+ bias),
+// BF16 output, FP32 accumulation in TMEM.  Two instantiations share the skeleton:
+//   - BF16 inputs            (tcgen05.mma kind::f16), the stage-2 reference linear;
+//   - NVFP4 inputs           (tcgen05.mma kind::mxf4nvf4.block_scale.scale_vec::4X), packed E2M1
+//     data with one E4M3 scale per 16 elements along K held in TMEM, the stage-1 rollout linear.
+//
+// CTA = 6 warps.  Warp 0: TMA producer (one lane).  Warp 1: TMEM owner and MMA issuer (one
+// lane).  Warps 2..5: epilogue, one TMEM lane quadrant each: tcgen05.ld -> alpha*acc + bias ->
+// BF16 -> swizzled shared memory -> TMA store.  A ring of kStages shared-memory stages feeds
+// the tensor core; two accumulator stages in TMEM let the epilogue of tile i overlap the
+// main loop of tile i+1.  Each stage holds 128 bytes of K per row (64 BF16 or 256 FP4), i.e.
+// four MMA instructions.  Every mbarrier wait is bounded: on expiry the CTA records a code in
+// the device status word and leaves through the normal teardown.
+#include "ptx.cuh"
+#include "sol_internal.h"
+
+#include <cuda_bf16.h>
+
+namespace sol {
+namespace {
+
+enum class Kind { kBf16, kNvfp4 };
+
+constexpr int kBM = 128;
+constexpr int kRowBytes = 128;        // bytes of K per row per stage (one swizzle atom wide)
+constexpr int kMmasPerStage = 4;      // 32 bytes of K per MMA
+constexpr int kThreads = 192;
+constexpr int kEpiWarps = 4;
+constexpr int kEpiBufBytes = 32 * 128;  // 32 rows x 64 BF16
+constexpr int kTmemCols = 512;
+constexpr int kGroupM = 8;            // tile raster: groups of 8 row tiles sweep all column tiles
+constexpr long long kWaitLimitCycles = 4000000000LL;
+
+template <Kind kKind, int kBN, int kStages>
+struct Cfg {
+    static constexpr bool kFp4 = kKind == Kind::kNvfp4;
+    static constexpr int kBK = kFp4 ? 256 : 64;                 // elements of K per stage
+    static constexpr int kMmaK = kBK / kMmasPerStage;
+    static constexpr int kABytes = kBM * kRowBytes;
+    static constexpr int kBBytes = kBN * kRowBytes;
+    static constexpr int kSfRowChunksB = kFp4 ? (kBN > 128 ? 2 : 1) : 0;  // 128-row scale chunks of B
+    static constexpr int kSfaBytes = kFp4 ? 2048 : 0;           // 4 chunks of 512 bytes
+    static constexpr int kSfbBytes = kSfRowChunksB * 2048;
+    static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
+    static constexpr int kAccStages = (2 * kBN + (kFp4 ? 16 + 16 * kSfRowChunksB : 0) <= kTmemCols) ? 2 : 1;
+    static constexpr int kSfaCol = kAccStages * kBN;            // TMEM columns of the scale factors
+    static constexpr int kSfbCol = kSfaCol + 16;
+    static constexpr int kEpiBytes = kEpiWarps * 2 * kEpiBufBytes;
+    static constexpr int kBarBytes = 256;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kBarBytes + 1024;
+    static_assert(kStageBytes % 1024 == 0, "stage tiles must stay 1024-byte aligned");
+    static_assert(kBN % 64 == 0 && kBN >= 64 && kBN <= 256, "tile N");
+    static_assert(!kFp4 || kSfbCol + 16 * kSfRowChunksB <= kTmemCols, "TMEM budget");
+    static_assert(kAccStages * kBN <= kTmemCols, "TMEM budget");
+    static_assert(kSmemBytes <= 232448, "shared memory budget");
+};
+
+struct Params {
+    const uint8_t *sfa;    // scales of A, chunked layout (NVFP4 only)
+    const uint8_t *sfb;
+    const float *ts_a;     // per-tensor scales (NVFP4 only)
+    const float *ts_b;
+    const uint16_t *bias;  // BF16 [N] or null
+    uint32_t *status;
+    int M, N, K;
+    int m_tiles, n_tiles;
+};
+
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                             uint32_t *status, uint32_t code) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!ptx::mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            *abort_flag = 1;
+            atomicExch(status, code);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int &mt, int &nt) {
+    const int per_group = kGroupM * n_tiles;
+    const int g = t / per_group;
+    const int first = g * kGroupM;
+    const int gsize = min(kGroupM, m_tiles - first);
+    const int r = t - g * per_group;
+    mt = first + r % gsize;
+    nt = r / gsize;
+}
+
+template <Kind kKind, int kBN, int kStages>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+            const __grid_constant__ CUtensorMap tm_y, const Params p) {
+    using C = Cfg<kKind, kBN, kStages>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+
+    const uint32_t epi_base = smem_base + kStages * C::kStageBytes;
+    const uint32_t bar_base = epi_base + C::kEpiBytes;
+    uint8_t *bar_gen = smem_gen + kStages * C::kStageBytes + C::kEpiBytes;
+    // barrier block: full[kStages], empty[kStages], acc_full[2], acc_empty[2], tmem ptr, abort flag
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+    auto acc_full_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+    auto acc_empty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 2 + s); };
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * (2 * kStages + 4));
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * (2 * kStages + 4) + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int k_tiles = (p.K + C::kBK - 1) / C::kBK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(acc_full_bar(s), 1);
+            ptx::mbar_init(acc_empty_bar(s), kEpiWarps);
+        }
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tm_a);
+        ptx::prefetch_tmap(&tm_b);
+        ptx::prefetch_tmap(&tm_y);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(tmem_ptr_smem), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_ptr_smem;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+                int mt, nt;
+                tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
+                const int m0 = mt * kBM, n0 = nt * kBN;
+                for (int kt = 0; kt < k_tiles; ++kt) {
+                    if (!wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x100u | stage)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t sa = smem_base + stage * C::kStageBytes;
+                    const uint32_t sb = sa + C::kABytes;
+                    uint32_t tx = C::kABytes + C::kBBytes;
+                    if (C::kFp4) {
+                        const int chunks_k = (p.K + 63) >> 6;
+                        const int nchunk = min(4, chunks_k - kt * 4);
+                        const int row_chunks_n = (p.N + 127) >> 7;
+                        const int rc0 = n0 >> 7;
+                        int n_rc = 0;
+                        for (int rc = 0; rc < C::kSfRowChunksB; ++rc) n_rc += (rc0 + rc < row_chunks_n);
+                        tx += static_cast<uint32_t>(nchunk * 512 * (1 + n_rc));
+                        ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+                        const uint32_t ssfa = sb + C::kBBytes;
+                        const uint32_t ssfb = ssfa + C::kSfaBytes;
+                        ptx::bulk_load_1d(ssfa, p.sfa + (static_cast<int64_t>(mt) * chunks_k + kt * 4) * 512,
+                                          nchunk * 512, full_bar(stage));
+                        for (int rc = 0; rc < C::kSfRowChunksB; ++rc) {
+                            if (rc0 + rc < row_chunks_n)
+                                ptx::bulk_load_1d(ssfb + rc * 2048,
+                                                  p.sfb + (static_cast<int64_t>(rc0 + rc) * chunks_k + kt * 4) * 512,
+                                                  nchunk * 512, full_bar(stage));
+                        }
+                    } else {
+                        ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+                    }
+                    // inner coordinate in elements of the tensor map (BF16 elements, or bytes of packed FP4)
+                    const int kx = C::kFp4 ? kt * kRowBytes : kt * C::kBK;
+                    ptx::tma_load_2d(sa, &tm_a, kx, m0, full_bar(stage));
+                    ptx::tma_load_2d(sb, &tm_b, kx, n0, full_bar(stage));
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t idesc;
+            if (C::kFp4) {
+                idesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kBN >> 3) << 17) |
+                        (static_cast<uint32_t>(kBM >> 4) << 24);  // E2M1 x E2M1, UE4M3 scales
+            } else {
+                idesc = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kBN >> 3) << 17) |
+                        (static_cast<uint32_t>(kBM >> 4) << 24);  // FP32 accum, BF16 x BF16, K-major
+            }
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int it = 0;
+            for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x, ++it) {
+                int mt, nt;
+                tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
+                const int as = it % C::kAccStages;
+                const uint32_t acc_parity = static_cast<uint32_t>(it / C::kAccStages) & 1u;
+                if (!wait_bounded(acc_empty_bar(as), acc_parity ^ 1u, abort_flag, p.status, 0x200u | as)) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + as * kBN;
+                const uint32_t sfb_shift = C::kFp4 ? static_cast<uint32_t>(((nt * kBN) & 127) >> 5) : 0u;
+                for (int kt = 0; kt < k_tiles; ++kt) {
+                    if (!wait_bounded(full_bar(stage), phase, abort_flag, p.status, 0x300u | stage)) {
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t sa = smem_base + stage * C::kStageBytes;
+                    const uint32_t sb = sa + C::kABytes;
+                    const uint64_t a_desc = ptx::smem_desc_sw128(sa);
+                    const uint64_t b_desc = ptx::smem_desc_sw128(sb);
+                    const int k_left = p.K - kt * C::kBK;
+                    const int nmma = min(kMmasPerStage, (k_left + C::kMmaK - 1) / C::kMmaK);
+                    if (C::kFp4) {
+                        const uint32_t ssfa = sb + C::kBBytes;
+                        const uint32_t ssfb = ssfa + C::kSfaBytes;
+                        for (int j = 0; j < nmma; ++j) {
+                            ptx::tc_copy_sf(tmem_base + C::kSfaCol + 4 * j, ptx::smem_desc_sf(ssfa + j * 512));
+                            for (int rc = 0; rc < C::kSfRowChunksB; ++rc)
+                                ptx::tc_copy_sf(tmem_base + C::kSfbCol + 4 * C::kSfRowChunksB * j + 4 * rc,
+                                                ptx::smem_desc_sf(ssfb + rc * 2048 + j * 512));
+                        }
+                        for (int j = 0; j < nmma; ++j)
+                            ptx::mma_nvfp4(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc,
+                                           tmem_base + C::kSfaCol + 4 * j,
+                                           tmem_base + C::kSfbCol + 4 * C::kSfRowChunksB * j + sfb_shift,
+                                           (kt | j) != 0);
+                    } else {
+                        for (int j = 0; j < nmma; ++j)
+                            ptx::mma_bf16(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kt | j) != 0);
+                    }
+                    ptx::tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (ok) ptx::tc_commit(acc_full_bar(as));
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32) are this warp's
+        const uint32_t epi_warp = epi_base + (warp - 2) * 2 * kEpiBufBytes;
+        const float alpha = C::kFp4 ? __fmul_rn(__ldg(p.ts_a), __ldg(p.ts_b)) : 1.0f;
+        int it = 0;
+        uint32_t buf = 0;
+        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++it) {
+            int mt, nt;
+            tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
+            const int m0 = mt * kBM + quad * 32, n0 = nt * kBN;
+            const int as = it % C::kAccStages;
+            const uint32_t acc_parity = static_cast<uint32_t>(it / C::kAccStages) & 1u;
+            if (!wait_bounded(acc_full_bar(as), acc_parity, abort_flag, p.status, 0x400u | as)) break;
+            ptx::tc_fence_after_sync();
+            const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + as * kBN;
+#pragma unroll 1
+            for (int c = 0; c < kBN / 64; ++c) {
+                const uint32_t sbuf = epi_warp + buf * kEpiBufBytes;
+                if (lane == 0) ptx::tma_store_wait_read<1>();  // the store issued two chunks ago has left sbuf
+                __syncwarp();
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t acc[32];
+                    ptx::tmem_ld_32x32(t_acc + c * 64 + h * 32, acc);
+                    ptx::tmem_ld_wait();
+                    if (c == kBN / 64 - 1 && h == 1) {
+                        // accumulator fully read: hand the TMEM stage back to the MMA warp
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(acc_empty_bar(as));
+                    }
+                    const int nb = n0 + c * 64 + h * 32;
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {  // 8 columns -> one 16-byte shared store
+                        uint4 bb = make_uint4(0, 0, 0, 0);
+                        if (p.bias != nullptr && nb + g * 8 < p.N)
+                            bb = __ldg(reinterpret_cast<const uint4 *>(p.bias + nb + g * 8));
+                        const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float b0 = __uint_as_float(bw[e] << 16);
+                            const float b1 = __uint_as_float(bw[e] & 0xFFFF0000u);
+                            const float y0 = fmaf(__uint_as_float(acc[g * 8 + 2 * e]), alpha, b0);
+                            const float y1 = fmaf(__uint_as_float(acc[g * 8 + 2 * e + 1]), alpha, b1);
+                            __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
+                            o[e] = *reinterpret_cast<uint32_t *>(&pk);
+                        }
+                        const uint32_t chunk16 = static_cast<uint32_t>(h * 4 + g) ^ (lane & 7u);  // 128-byte swizzle
+                        const uint32_t dst = sbuf + lane * 128 + chunk16 * 16;
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]),
+                                     "r"(o[2]), "r"(o[3])
+                                     : "memory");
+                    }
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (n0 + c * 64 < p.N && m0 < p.M) ptx::tma_store_2d(&tm_y, n0 + c * 64, m0, sbuf);
+                    ptx::tma_store_commit();
+                }
+                buf ^= 1u;
+            }
+        }
+        if (lane == 0) ptx::tma_store_wait_all<0>();
+    }
+
+    // ---------------------------------------------------------------- teardown
+    if (*abort_flag) __nanosleep(2000000);  // let copies already in flight land before the CTA exits
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+template <Kind kKind, int kBN, int kStages>
+sol_status_t launch(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUtensorMap &tm_y, Params p,
+                    cudaStream_t stream, const DeviceInfo *dev) {
+    using C = Cfg<kKind, kBN, kStages>;
+    static bool configured[64] = {};
+    auto kern = gemm_kernel<kKind, kBN, kStages>;
+    if (dev->device < 64 && !configured[dev->device]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
+            return SOL_ERR_CUDA;
+        configured[dev->device] = true;
+    }
+    p.m_tiles = static_cast<int>(ceil_div(p.M, kBM));
+    p.n_tiles = static_cast<int>(ceil_div(p.N, kBN));
+    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
+    const int grid = static_cast<int>(tiles < dev->sm_count ? tiles : dev->sm_count);
+    kern<<<grid, kThreads, C::kSmemBytes, stream>>>(tm_a, tm_b, tm_y, p);
+    return launch_status();
+}
+
+}  // namespace
+
+sol_status_t launch_gemm_bf16(const void *x, const void *w, const void *bias, void *y, int64_t M, int64_t N,
+                              int64_t K, int64_t ldx, int64_t ldw, int64_t ldy, cudaStream_t stream,
+                              const DeviceInfo *dev) {
+    constexpr int kBN = 256;
+    CUtensorMap tm_a, tm_b, tm_y;
+    if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, K, M, ldx * 2, 64, kBM,
+                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w, K, N, ldw * 2, 64, kBN,
+                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, N, M, ldy * 2, 64, 32,
+                      CU_TENSOR_MAP_SWIZZLE_128B))
+        return SOL_ERR_CUDA;
+    Params p{};
+    p.bias = static_cast<const uint16_t *>(bias);
+    p.status = device_status_word();
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    return launch<Kind::kBf16, kBN, 4>(tm_a, tm_b, tm_y, p, stream, dev);
+}
+
+sol_status_t launch_gemm_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
+                               const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
+                               int64_t N, int64_t K, int64_t ldy, cudaStream_t stream,
+                               const DeviceInfo *dev) {
+    constexpr int kBN = 192;
+    CUtensorMap tm_a, tm_b, tm_y;
+    if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, xq, K / 2, M, K / 2, 128, kBM,
+                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, wq, K / 2, N, K / 2, 128, kBN,
+                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, N, M, ldy * 2, 64, 32,
+                      CU_TENSOR_MAP_SWIZZLE_128B))
+        return SOL_ERR_CUDA;
+    Params p{};
+    p.sfa = static_cast<const uint8_t *>(xsf);
+    p.sfb = static_cast<const uint8_t *>(wsf);
+    p.ts_a = xts;
+    p.ts_b = wts;
+    p.bias = static_cast<const uint16_t *>(bias);
+    p.status = device_status_word();
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    return launch<Kind::kNvfp4, kBN, 4>(tm_a, tm_b, tm_y, p, stream, dev);
+}
+
+}  // namespace sol

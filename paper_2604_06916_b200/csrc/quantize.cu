@@ -1,0 +1,205 @@
+// NVFP4 quantizer kernels (per-tensor amax, activation / weight quantizer) for sm_100a.
+//
+// Q(x) = S * Pi_FP4(x / S) with S = E4M3 block scale * FP32 tensor scale T (paper Section 2).
+// Both kernels are streaming codecs bound by HBM bandwidth: 16-byte loads, many loads in
+// flight per thread, packed 4-byte nibble stores, scale bytes staged in shared memory and
+// written as whole 512-byte chunks of the layout the tensor core consumes.
+#include "sol_internal.h"
+
+namespace sol {
+namespace {
+
+constexpr int kQuantThreads = 256;
+constexpr int kTileRows = 128;     // rows per block = one row tile of the chunked scale layout
+constexpr int kTileK = 256;        // elements along K per block = 4 scale chunks = 32 vectors of 8
+constexpr int kRowsPerWarp = kTileRows / (kQuantThreads / 32);  // 16
+constexpr int kBatch = 8;          // independent 16-byte loads in flight per thread
+
+__device__ __forceinline__ uint32_t abs_max_bits(const uint4 &v) {
+    // packed per-halfword max of |bf16| bit patterns (magnitudes order like unsigned integers)
+    uint32_t a = __vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu);
+    uint32_t b = __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu);
+    a = __vmaxu2(a, b);
+    return max(a & 0xFFFFu, a >> 16);
+}
+
+__device__ __forceinline__ uint32_t f32_to_e4m3_sat(float v) {
+    uint16_t packed;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(packed) : "f"(0.0f), "f"(v));
+    return packed & 0xFFu;
+}
+
+__device__ __forceinline__ float e4m3_to_f32(uint32_t code) {
+    uint32_t e = (code >> 3) & 15u, m = code & 7u;
+    if (e == 0) return __uint2float_rn(m) * 0x1p-9f;
+    return __uint_as_float(((e + 120u) << 23) | (m << 20));
+}
+
+// Eight FP32 values -> eight E2M1 nibbles (element 0 in the lowest nibble).
+__device__ __forceinline__ uint32_t pack_e2m1x8(float y0, float y1, float y2, float y3, float y4,
+                                                float y5, float y6, float y7) {
+    uint32_t out;
+    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+        "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
+        : "=r"(out)
+        : "f"(y0), "f"(y1), "f"(y2), "f"(y3), "f"(y4), "f"(y5), "f"(y6), "f"(y7));
+    return out;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// One block quantizes a 128-row x 256-element tile.  Lane l of a warp owns the 8 elements
+// [8l, 8l+8) of the tile's K range; lanes 2b and 2b+1 share scale block b.
+template <bool kSwizzled>
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
+                const float *__restrict__ tscale, uint8_t *__restrict__ q, uint8_t *__restrict__ sf) {
+    __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kTileK / 16)];  // 2 KB = 4 chunks
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row0 = static_cast<int64_t>(blockIdx.y) * kTileRows;
+    const int64_t k0 = static_cast<int64_t>(blockIdx.x) * kTileK;
+    const int64_t k = k0 + lane * 8;
+    const bool k_ok = k < K;
+
+    if (kSwizzled) {
+        reinterpret_cast<uint64_t *>(sf_tile)[threadIdx.x] = 0;  // padding bytes must read as 0
+        __syncthreads();
+    }
+
+    const float T = __ldg(tscale);
+    const float c = __fmul_rn(6.0f, T);
+    const int64_t nb = K >> 4;
+
+#pragma unroll 1
+    for (int batch = 0; batch < kRowsPerWarp / kBatch; ++batch) {
+        uint4 v[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            const int64_t r = row0 + warp * kRowsPerWarp + batch * kBatch + i;
+            v[i] = make_uint4(0, 0, 0, 0);
+            if (k_ok && r < rows) v[i] = __ldcs(reinterpret_cast<const uint4 *>(x + r * ld + k));
+        }
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            const int rl = warp * kRowsPerWarp + batch * kBatch + i;  // row inside the tile
+            const int64_t r = row0 + rl;
+            uint32_t mb = abs_max_bits(v[i]);
+            mb = max(mb, __shfl_xor_sync(0xFFFFFFFFu, mb, 1));
+            const float a = __uint_as_float(mb << 16);
+            const float sv = __fdiv_rn(a, c);
+            const uint32_t sb = f32_to_e4m3_sat(sv);
+            const float d = __fmul_rn(e4m3_to_f32(sb), T);
+            const float rcp = sb ? __frcp_rn(d) : 0.0f;
+            const uint32_t packed = pack_e2m1x8(
+                __fmul_rn(bf16_lo(v[i].x), rcp), __fmul_rn(bf16_hi(v[i].x), rcp),
+                __fmul_rn(bf16_lo(v[i].y), rcp), __fmul_rn(bf16_hi(v[i].y), rcp),
+                __fmul_rn(bf16_lo(v[i].z), rcp), __fmul_rn(bf16_hi(v[i].z), rcp),
+                __fmul_rn(bf16_lo(v[i].w), rcp), __fmul_rn(bf16_hi(v[i].w), rcp));
+            if (k_ok && r < rows) {
+                __stcs(reinterpret_cast<uint32_t *>(q + r * (K >> 1) + (k >> 1)), packed);
+                if ((lane & 1) == 0) {
+                    const int b = lane >> 1;  // scale block inside the tile, 0..15
+                    if (kSwizzled) {
+                        sf_tile[(b >> 2) * 512 + (rl & 31) * 16 + (rl >> 5) * 4 + (b & 3)] =
+                            static_cast<uint8_t>(sb);
+                    } else {
+                        sf[r * nb + (k >> 4)] = static_cast<uint8_t>(sb);
+                    }
+                }
+            }
+        }
+    }
+
+    if (kSwizzled) {
+        __syncthreads();
+        // 4 chunks x 32 lines of 16 bytes; chunk c of this tile is k chunk blockIdx.x*4 + c
+        const int64_t chunks_k = (nb + 3) >> 2;
+        if (threadIdx.x < 128) {
+            const int cidx = threadIdx.x >> 5;
+            const int64_t kc = static_cast<int64_t>(blockIdx.x) * 4 + cidx;
+            if (kc < chunks_k) {
+                uint8_t *dst = sf + (static_cast<int64_t>(blockIdx.y) * chunks_k + kc) * 512 +
+                               (threadIdx.x & 31) * 16;
+                *reinterpret_cast<uint4 *>(dst) = reinterpret_cast<const uint4 *>(sf_tile)[threadIdx.x];
+            }
+        }
+    }
+}
+
+// max |x| over the tensor as the bit pattern of the FP32 value (BF16 magnitude << 16).
+__global__ void __launch_bounds__(256)
+amax_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t vecs_per_row, int64_t ld,
+            uint32_t *__restrict__ out_bits) {
+    uint32_t m = 0;
+    const int64_t total = rows * vecs_per_row;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+    int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (ld == vecs_per_row * 8) {
+        const uint4 *p = reinterpret_cast<const uint4 *>(x);
+        for (; i + 3 * stride < total; i += 4 * stride) {
+            uint4 a = __ldcs(p + i), b = __ldcs(p + i + stride), c = __ldcs(p + i + 2 * stride),
+                  d = __ldcs(p + i + 3 * stride);
+            m = max(m, max(max(abs_max_bits(a), abs_max_bits(b)), max(abs_max_bits(c), abs_max_bits(d))));
+        }
+        for (; i < total; i += stride) m = max(m, abs_max_bits(__ldcs(p + i)));
+    } else {
+        for (; i < total; i += stride) {
+            const int64_t r = i / vecs_per_row, vcol = i - r * vecs_per_row;
+            m = max(m, abs_max_bits(__ldcs(reinterpret_cast<const uint4 *>(x + r * ld + vcol * 8))));
+        }
+    }
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    __shared__ uint32_t warp_max[8];
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        m = threadIdx.x < 8 ? warp_max[threadIdx.x] : 0;
+        m = __reduce_max_sync(0xFFFFFFFFu, m);
+        if (threadIdx.x == 0 && m) atomicMax(out_bits, m << 16);
+    }
+}
+
+// In place: amax bits -> T = amax / (6 * 448), or 1 for an all-zero tensor.
+__global__ void tensor_scale_kernel(float *t) {
+    const float a = *t;
+    *t = (a == 0.0f) ? 1.0f : __fdiv_rn(a, 2688.0f);
+}
+
+}  // namespace
+
+sol_status_t launch_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *tscale_out,
+                         cudaStream_t stream, const DeviceInfo *dev) {
+    if (cudaMemsetAsync(tscale_out, 0, sizeof(float), stream) != cudaSuccess) return SOL_ERR_CUDA;
+    const int64_t vecs = rows * (K / 8);
+    int64_t blocks = ceil_div(vecs, 256 * 4);
+    const int64_t cap = static_cast<int64_t>(dev->sm_count) * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    amax_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
+        static_cast<const uint16_t *>(x), rows, K / 8, ld, reinterpret_cast<uint32_t *>(tscale_out));
+    tensor_scale_kernel<<<1, 1, 0, stream>>>(tscale_out);
+    return launch_status();
+}
+
+sol_status_t launch_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale,
+                             void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream) {
+    dim3 grid(static_cast<unsigned>(ceil_div(K, kTileK)), static_cast<unsigned>(ceil_div(rows, kTileRows)));
+    if (layout == SOL_SF_SWIZZLED_128x4) {
+        quantize_kernel<true><<<grid, kQuantThreads, 0, stream>>>(
+            static_cast<const uint16_t *>(x), rows, K, ld, tscale, static_cast<uint8_t *>(q),
+            static_cast<uint8_t *>(sf));
+    } else {
+        quantize_kernel<false><<<grid, kQuantThreads, 0, stream>>>(
+            static_cast<const uint16_t *>(x), rows, K, ld, tscale, static_cast<uint8_t *>(q),
+            static_cast<uint8_t *>(sf));
+    }
+    return launch_status();
+}
+
+}  // namespace sol

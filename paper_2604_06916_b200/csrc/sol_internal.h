@@ -1,0 +1,54 @@
+// Host-side helpers shared by the entry points: argument checks, device query, launch checks.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/sol_nvfp4.h"
+
+namespace sol {
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+struct DeviceInfo {
+    int device = -1;
+    int sm_count = 0;
+    int cc_major = 0;
+    int cc_minor = 0;
+    bool ok = false;
+};
+
+// Properties of the current device (queried once per device, cached on the host).
+const DeviceInfo *current_device_info();
+
+// SOL_OK when the current device is an sm_100 part, SOL_ERR_UNSUPPORTED_ARCH / SOL_ERR_CUDA otherwise.
+sol_status_t check_arch(const DeviceInfo **info_out);
+
+inline sol_status_t launch_status() {
+    return cudaGetLastError() == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
+}
+
+// Device status word written by bounded waits (0 = fine).
+uint32_t *device_status_word();
+
+// Internal launchers (arguments already validated).
+sol_status_t launch_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *tscale_out,
+                         cudaStream_t stream, const DeviceInfo *dev);
+sol_status_t launch_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale,
+                             void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream);
+sol_status_t launch_gemm_bf16(const void *x, const void *w, const void *bias, void *y, int64_t M,
+                              int64_t N, int64_t K, int64_t ldx, int64_t ldw, int64_t ldy,
+                              cudaStream_t stream, const DeviceInfo *dev);
+sol_status_t launch_gemm_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
+                               const void *wsf, const float *wts, const void *bias, void *y,
+                               int64_t M, int64_t N, int64_t K, int64_t ldy, cudaStream_t stream,
+                               const DeviceInfo *dev);
+
+// 2-D row-major tensor map: `inner` contiguous elements per row, `outer` rows, row pitch in bytes.
+// Returns false if the driver rejects it.
+bool make_tmap_2d(CUtensorMap *out, CUtensorMapDataType dtype, uint32_t elem_bytes, const void *base,
+                  uint64_t inner, uint64_t outer, uint64_t pitch_bytes, uint32_t box_inner,
+                  uint32_t box_outer, CUtensorMapSwizzle swizzle);
+
+}  // namespace sol

@@ -1,0 +1,53 @@
+"""Shared helpers for the GPU parity tests (host-side glue only)."""
+import numpy as np
+import torch
+
+import oracle
+
+
+def bits_of(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def from_bits(bits: np.ndarray, device) -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).to(device)
+
+
+def swizzled_offsets(rows: np.ndarray, K: int) -> np.ndarray:
+    """[len(rows), K/16] byte offsets into the 128x4-chunked scale buffer (vectorised copy of the
+    index rule; checked against the oracle's scalar function in the tests)."""
+    nb = K // 16
+    chunks_k = (nb + 3) // 4
+    r = np.asarray(rows, dtype=np.int64)[:, None]
+    b = np.arange(nb, dtype=np.int64)[None, :]
+    rr = r % 128
+    return ((r // 128) * chunks_k + b // 4) * 512 + (rr % 32) * 16 + (rr // 32) * 4 + b % 4
+
+
+def unswizzle_rows(sf_swizzled: np.ndarray, rows, K: int) -> np.ndarray:
+    return sf_swizzled[swizzled_offsets(rows, K)]
+
+
+def sample_rows(M: int, seed: int = 0) -> np.ndarray:
+    """First and last 128-row tile in full plus one pseudo-random row of every other tile."""
+    rng = np.random.default_rng(seed)
+    tiles = (M + 127) // 128
+    rows = set(range(min(128, M))) | set(range((tiles - 1) * 128, M))
+    for t in range(1, tiles - 1):
+        rows.add(t * 128 + int(rng.integers(0, 128)))
+    return np.array(sorted(rows), dtype=np.int64)
+
+
+def check_linear(y_gpu_bits: np.ndarray, Y: np.ndarray, what: str = ""):
+    """|gpu - oracle| <= 2^-7 |oracle| + 1e-4 rms(oracle row) for every output."""
+    g = oracle.bits_to_f64(y_gpu_bits)
+    tol = oracle.linear_tolerance(Y)
+    err = np.abs(g - Y)
+    bad = err > tol
+    if bad.any():
+        i, j = np.argwhere(bad)[0]
+        raise AssertionError(
+            f"{what}: {int(bad.sum())} of {bad.size} outputs out of tolerance; first at ({i},{j}): "
+            f"gpu={g[i, j]!r} oracle={Y[i, j]!r} err={err[i, j]:.3e} tol={tol[i, j]:.3e}; "
+            f"bad rows={np.unique(np.argwhere(bad)[:, 0])[:8]} bad cols={np.unique(np.argwhere(bad)[:, 1])[:8]}")
+    return float(np.max(err / np.maximum(tol, 1e-300)))
