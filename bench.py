@@ -1,0 +1,400 @@
+#!/usr/bin/env python
+"""Benchmark of the NVFP4 linear path on FLUX.1-shaped layers (one B200 per rank).
+
+One "step" = the whole hot path over one batch: for each of the six FLUX.1 linears
+(M = 8 samples x 4608 tokens) the dynamic per-tensor scale, the activation quantizer and the
+block-scaled FP4 GEMM with BF16 output (weights are quantized once, outside the timed region,
+as they change once per policy update).  The same layers then run through the BF16 tcgen05
+GEMM to give the FP4-over-BF16 speedup on our own kernels.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "nvfp4_linear_tflops_flux_shapes"
+UNIT = "TFLOP/s"
+NOMINAL_FP4_TFLOPS = 9000.0     # vendor dense NVFP4 peak
+NOMINAL_BF16_TFLOPS = 2250.0    # vendor dense BF16 peak
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [s.strip() for s in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def flops_of(layers) -> float:
+    return float(sum(2.0 * l.M * l.N * l.K for l in layers))
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample_tflops(cfg, layer_index: int, rows: int):
+    """Times the oracle (quantize + FP64 dequantized matmul) on `rows` rows of one layer."""
+    import numpy as np
+    import oracle
+    from paper_2604_06916_b200 import workloads
+
+    layer = cfg.layers[layer_index]
+    X, W, bias = workloads.make_layer(cfg, layer_index, "cpu", M=rows)
+    xb, wb, bb = workloads.to_bits(X), workloads.to_bits(W), workloads.to_bits(bias)
+    Tw = oracle.tensor_scale(wb)
+    qw, sfw = oracle.quantize(wb, Tw)         # weights: outside the timed region, like the GPU arm
+    t0 = time.perf_counter()
+    Tx = oracle.tensor_scale(xb)
+    qx, sfx = oracle.quantize(xb, Tx)
+    Y = oracle.nvfp4_linear(qx, sfx, Tx, qw, sfw, Tw, bb)
+    dt = time.perf_counter() - t0
+    assert np.isfinite(Y).all()
+    flops = 2.0 * rows * layer.N * layer.K
+    return flops / dt / 1e12, dt, oracle.num_threads(), f"{rows} rows of {cfg.name}/{layer.name} (N={layer.N}, K={layer.K})"
+
+
+def calibrated_rows(cfg, layer_index: int, target_s: float, fixed: int) -> int:
+    """Rows of the sample so that one oracle pass takes about target_s on this host."""
+    if fixed > 0:
+        return fixed
+    _, dt, _, _ = oracle_sample_tflops(cfg, layer_index, 256)
+    rows = int(256 * target_s / max(dt, 1e-3))
+    return max(256, min(cfg.layers[layer_index].M, (rows // 128) * 128))
+
+
+def run_reference(args):
+    from paper_2604_06916_b200 import workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = workloads.CONFIG_FLUX
+    vals, secs = [], []
+    sample = ""
+    cores = 1
+    rows = calibrated_rows(cfg, 1, 3.0, args.ref_rows)
+    for i in range(args.warmup + args.steps):
+        v, dt, cores, sample = oracle_sample_tflops(cfg, 1, rows)
+        if i >= args.warmup:
+            vals.append(v)
+            secs.append(dt)
+    value = sum(vals) / len(vals) if vals else 0.0
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / max(1, len(secs)), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "note": "CPU oracle on a bounded row sample of one layer per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import torch
+    from paper_2604_06916_b200 import binding as B
+    from paper_2604_06916_b200 import workloads
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    B.lib()
+    peaks, peak_src = load_peaks()
+    cfg = workloads.CONFIGS[args.workload] if args.workload in workloads.CONFIGS else workloads.config_sweep(
+        int(args.workload.split("_g")[-1]))
+    layers = cfg.layers
+    dev = torch.device("cuda", local_rank)
+
+    # ---- inputs (resident in HBM), weights quantized once
+    acts = {}
+    data = []
+    for i, l in enumerate(layers):
+        X, W, bias = workloads.make_layer(cfg, i, dev)
+        if l.K in acts:
+            X = acts[l.K]          # one activation tensor per distinct K (all larger than L2)
+        else:
+            acts[l.K] = X
+        wq, wsf, wts = B.nvfp4_quantize_weight(W)
+        Y = torch.empty((l.M, l.N), dtype=torch.bfloat16, device=dev)
+        ws = torch.empty(B.linear_workspace_bytes(l.M, l.N, l.K), dtype=torch.uint8, device=dev)
+        data.append(dict(l=l, X=X, W=W, bias=bias, wq=wq, wsf=wsf, wts=wts, Y=Y, ws=ws))
+    torch.cuda.synchronize()
+
+    def fp4_step():
+        for d in data:
+            B.nvfp4_quantize_linear(d["X"], d["wq"], d["wsf"], d["wts"], d["bias"], workspace=d["ws"], out=d["Y"])
+
+    def bf16_step():
+        for d in data:
+            B.bf16_linear(d["X"], d["W"], d["bias"], out=d["Y"])
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(max(3, args.warmup)):
+        fp4_step()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_fp4 = timed(fp4_step, args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+    B.sol_last_device_status()
+
+    for _ in range(max(3, args.warmup)):
+        bf16_step()
+    ms_bf16 = timed(bf16_step, args.steps)
+    B.sol_last_device_status()
+
+    # ---- per-kernel timing with events on the launching stream (same kernels, unfused calls)
+    per_layer = []
+    n_detail = max(3, min(args.steps, 10))
+    tot = {"amax": 0.0, "quant": 0.0, "gemm": 0.0}
+    for d in data:
+        l = d["l"]
+        xts = torch.empty(1, dtype=torch.float32, device=dev)
+        xq = torch.empty((l.M, l.K // 2), dtype=torch.uint8, device=dev)
+        xsf = torch.empty(B.scale_bytes(l.M, l.K), dtype=torch.uint8, device=dev)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_detail + 2)]
+        for it in range(n_detail + 2):
+            ev[it][0].record()
+            B.sol_amax_bf16(d["X"], out=xts)
+            ev[it][1].record()
+            B.nvfp4_quantize(d["X"], xts, out=(xq, xsf))
+            ev[it][2].record()
+            B.nvfp4_linear(xq, xsf, xts, d["wq"], d["wsf"], d["wts"], d["bias"], out=d["Y"])
+            ev[it][3].record()
+        torch.cuda.synchronize()
+        t = [sum(ev[it][j].elapsed_time(ev[it][j + 1]) for it in range(2, n_detail + 2)) / n_detail for j in range(3)]
+        eb = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        B.bf16_linear(d["X"], d["W"], d["bias"], out=d["Y"])
+        eb[0].record()
+        for _ in range(n_detail):
+            B.bf16_linear(d["X"], d["W"], d["bias"], out=d["Y"])
+        eb[1].record()
+        torch.cuda.synchronize()
+        t_bf16 = eb[0].elapsed_time(eb[1]) / n_detail
+        fl = 2.0 * l.M * l.N * l.K
+        qbytes = l.M * l.K * 2 + l.M * l.K // 2 + B.scale_bytes(l.M, l.K)
+        per_layer.append({
+            "layer": l.name, "M": l.M, "K": l.K, "N": l.N,
+            "amax_ms": round(t[0], 4), "quant_ms": round(t[1], 4), "gemm_ms": round(t[2], 4), "bf16_ms": round(t_bf16, 4),
+            "gemm_tflops": round(fl / t[2] / 1e9, 1), "bf16_tflops": round(fl / t_bf16 / 1e9, 1),
+            "quant_gbs": round(qbytes / t[1] / 1e6, 1), "amax_gbs": round(l.M * l.K * 2 / t[0] / 1e6, 1),
+            "stack_speedup": round(t_bf16 / (t[0] + t[1] + t[2]), 3),
+        })
+        tot["amax"] += t[0]
+        tot["quant"] += t[1]
+        tot["gemm"] += t[2]
+        del xq, xsf
+    B.sol_last_device_status()
+
+    flops = flops_of(layers)
+    ms_step = ms_fp4 / args.steps
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    bf16_value = world * flops / (ms_bf16 / args.steps * 1e-3) / 1e12
+    gemm_tflops = flops / (tot["gemm"] * 1e-3) / 1e12
+    fp4_peak = peaks["bf16_tflops_sustained"] * (NOMINAL_FP4_TFLOPS / NOMINAL_BF16_TFLOPS)
+    quant_bytes = sum(l.M * l.K * 2 + l.M * l.K // 2 + B.scale_bytes(l.M, l.K) for l in layers)
+
+    # ---- end to end: host buffers, copies inside the timed region, through the same entry point
+    e2e = None
+    if rank == 0 or world > 1:
+        d = data[1]  # d_proj layer: 226 MB in, 226 MB out per call
+        l = d["l"]
+        xh = torch.empty((l.M, l.K), dtype=torch.bfloat16).pin_memory()
+        xh.copy_(d["X"])
+        yh = torch.empty((l.M, l.N), dtype=torch.bfloat16).pin_memory()
+        xd = torch.empty_like(d["X"])
+
+        def e2e_step():
+            xd.copy_(xh, non_blocking=True)
+            B.nvfp4_quantize_linear(xd, d["wq"], d["wsf"], d["wts"], d["bias"], workspace=d["ws"], out=d["Y"])
+            yh.copy_(d["Y"], non_blocking=True)
+
+        for _ in range(2):
+            e2e_step()
+        n_e2e = max(3, min(args.steps, 5))
+        ms_e2e = timed(e2e_step, n_e2e) / n_e2e
+        e2e = {"value": world * 2.0 * l.M * l.N * l.K / (ms_e2e * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": xh.numel() * 2, "d2h_bytes_per_step": yh.numel() * 2,
+               "workload": f"{cfg.name}/{l.name} through nvfp4_quantize_linear with pinned host X and Y",
+               "ms_per_step": ms_e2e}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 or rank == 0:
+        rows = calibrated_rows(workloads.CONFIG_FLUX, 1, 12.0, args.ref_rows)
+        v, dt, cores, sample = oracle_sample_tflops(workloads.CONFIG_FLUX, 1, rows)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "seconds": round(dt, 2)}
+
+    kernels_per_layer = 4  # amax, tensor-scale finalize, quantize, GEMM (+1 memset, not a kernel)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "nvfp4 (e2m1 x e4m3 block scales, fp32 accumulate, bf16 out)", "data": "synthetic",
+        "config": {"workload": cfg.name, "layers": [f"{l.name}:{l.M}x{l.K}->{l.N}" for l in layers],
+                   "l2": "every activation tensor is larger than L2 (>= 226 MB)",
+                   "multi_gpu": "independent replicas, no collective"},
+        "pct_of_nominal_fp4_peak": 100.0 * value / world / NOMINAL_FP4_TFLOPS,
+        "bf16_stack_tflops": bf16_value, "fp4_over_bf16_speedup": ms_bf16 / ms_fp4,
+        "gemm_only_tflops": gemm_tflops, "gemm_pct_of_nominal_fp4_peak": 100.0 * gemm_tflops / NOMINAL_FP4_TFLOPS,
+        "quantizer_gbs": quant_bytes / (tot["quant"] * 1e-3) / 1e9,
+        "quantizer_pct_of_8tbs": 100.0 * quant_bytes / (tot["quant"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "roofline": {"bound": "tensor", "kernel": "gemm_kernel<nvfp4>", "achieved": gemm_tflops, "peak": fp4_peak,
+                     "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak, "traffic": None,
+                     "peak_source": f"{peak_src} sustained bf16 {peaks['bf16_tflops_sustained']} TF x 4 (nominal fp4:bf16)"},
+        "roofline_quantizer": {"bound": "hbm", "kernel": "quantize_kernel", "achieved": quant_bytes / (tot["quant"] * 1e-3) / 1e9,
+                               "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": quant_bytes / (tot["quant"] * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                               "peak_source": peak_src},
+        "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+        "gpu_launches": kernels_per_layer * len(layers) * args.steps,
+        "per_layer": per_layer,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def run_only(args):
+    """Small fixed case for profilers: one layer, `steps` passes of the FP4 stack then the BF16 GEMM."""
+    import torch
+    from paper_2604_06916_b200 import binding as B
+    from paper_2604_06916_b200 import workloads
+
+    cfg = workloads.CONFIGS[args.workload]
+    index = [l.name for l in cfg.layers].index(args.only)
+    l = cfg.layers[index]
+    M = args.rows if args.rows > 0 else l.M
+    X, W, bias = workloads.make_layer(cfg, index, "cuda", M=M)
+    wq, wsf, wts = B.nvfp4_quantize_weight(W)
+    Y = torch.empty((M, l.N), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(B.linear_workspace_bytes(M, l.N, l.K), dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    times = []
+    for it in range(args.warmup + args.steps):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        B.nvfp4_quantize_linear(X, wq, wsf, wts, bias, workspace=ws, out=Y)
+        e[1].record()
+        B.bf16_linear(X, W, bias, out=Y)
+        e[2].record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            times.append((e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])))
+    B.sol_last_device_status()
+    fl = 2.0 * M * l.N * l.K
+    t4 = sum(t[0] for t in times) / len(times)
+    t16 = sum(t[1] for t in times) / len(times)
+    print(json.dumps({"only": l.name, "M": M, "K": l.K, "N": l.N, "fp4_stack_ms": t4, "bf16_ms": t16,
+                      "fp4_stack_tflops": fl / t4 / 1e9, "bf16_tflops": fl / t16 / 1e9}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload")
+    ap.add_argument("--rows", type=int, default=0, help="profile mode: override M")
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="flux1_12b_g8")
+    ap.add_argument("--ref-rows", type=int, default=0, help="rows of the oracle sample (0 = calibrate)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    elif args.only:
+        run_only(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -12,7 +12,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsol_nvfp4.so")
+LIB_PATH = os.environ.get("SOL_NVFP4_LIB", os.path.join(_HERE, "libsol_nvfp4.so"))
 
 SF_ROW_MAJOR = 0
 SF_SWIZZLED_128x4 = 1

@@ -15,6 +15,7 @@
 #include "sol_internal.h"
 
 #include <cuda_bf16.h>
+#include <cstdlib>
 
 namespace sol {
 namespace {
@@ -24,7 +25,6 @@ enum class Kind { kBf16, kNvfp4 };
 constexpr int kBM = 128;
 constexpr int kRowBytes = 128;        // bytes of K per row per stage (one swizzle atom wide)
 constexpr int kMmasPerStage = 4;      // 32 bytes of K per MMA
-constexpr int kThreads = 192;
 constexpr int kEpiWarps = 4;
 constexpr int kEpiBufBytes = 32 * 128;  // 32 rows x 64 BF16
 constexpr int kTmemCols = 512;
@@ -42,18 +42,31 @@ struct Cfg {
     static constexpr int kSfaBytes = kFp4 ? 2048 : 0;           // 4 chunks of 512 bytes
     static constexpr int kSfbBytes = kSfRowChunksB * 2048;
     static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
-    static constexpr int kAccStages = (2 * kBN + (kFp4 ? 16 + 16 * kSfRowChunksB : 0) <= kTmemCols) ? 2 : 1;
-    static constexpr int kSfaCol = kAccStages * kBN;            // TMEM columns of the scale factors
-    static constexpr int kSfbCol = kSfaCol + 16;
+    // TMEM columns of one scale-factor buffer: 4 MMAs x (4 columns of A + 4 per 128-row chunk of B).
+    // Two buffers, so the copies for k-tile i+1 run while the MMAs of k-tile i read the other one.
+    static constexpr int kSfBufCols = kFp4 ? 16 + 16 * kSfRowChunksB : 0;
+    static constexpr int kSfBufs = 2;
+    static constexpr int kAccStages = (2 * kBN + kSfBufs * kSfBufCols <= kTmemCols) ? 2 : 1;
+    static constexpr int kSfCol = kAccStages * kBN;             // first scale-factor column
+    static constexpr int kSfWarps = kFp4 ? kMmasPerStage : 0;   // one copy warp per MMA of a stage
+    static constexpr int kThreads = 192 + 32 * kSfWarps;
     static constexpr int kEpiBytes = kEpiWarps * 2 * kEpiBufBytes;
     static constexpr int kBarBytes = 256;
     static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kBarBytes + 1024;
     static_assert(kStageBytes % 1024 == 0, "stage tiles must stay 1024-byte aligned");
     static_assert(kBN % 64 == 0 && kBN >= 64 && kBN <= 256, "tile N");
-    static_assert(!kFp4 || kSfbCol + 16 * kSfRowChunksB <= kTmemCols, "TMEM budget");
-    static_assert(kAccStages * kBN <= kTmemCols, "TMEM budget");
+    static_assert(kSfCol + kSfBufs * kSfBufCols <= kTmemCols, "TMEM budget");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
 };
+
+// Diagnostic switches, compiled in only with -DSOL_TUNING (never in the product build): they
+// drop one part of the pipeline so its share of the time can be read off a timing run.
+#ifdef SOL_TUNING
+constexpr bool kTuning = true;
+#else
+constexpr bool kTuning = false;
+#endif
+enum : uint32_t { kDbgNoSfCopy = 1, kDbgNoMma = 2, kDbgNoEpilogue = 4, kDbgNoSfLoad = 8, kDbgNoStore = 16 };
 
 struct Params {
     const uint8_t *sfa;    // scales of A, chunked layout (NVFP4 only)
@@ -62,6 +75,7 @@ struct Params {
     const float *ts_b;
     const uint16_t *bias;  // BF16 [N] or null
     uint32_t *status;
+    uint32_t dbg;
     int M, N, K;
     int m_tiles, n_tiles;
 };
@@ -92,7 +106,7 @@ __device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int
 }
 
 template <Kind kKind, int kBN, int kStages>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__((Cfg<kKind, kBN, kStages>::kThreads), 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
             const __grid_constant__ CUtensorMap tm_y, const Params p) {
     using C = Cfg<kKind, kBN, kStages>;
@@ -103,13 +117,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
     const uint32_t epi_base = smem_base + kStages * C::kStageBytes;
     const uint32_t bar_base = epi_base + C::kEpiBytes;
     uint8_t *bar_gen = smem_gen + kStages * C::kStageBytes + C::kEpiBytes;
-    // barrier block: full[kStages], empty[kStages], acc_full[2], acc_empty[2], tmem ptr, abort flag
+    // barrier block: full[kStages], empty[kStages], acc_full[2], acc_empty[2], sf_ready[2], tmem ptr, abort flag
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
     auto acc_full_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
     auto acc_empty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 2 + s); };
-    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * (2 * kStages + 4));
-    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * (2 * kStages + 4) + 4);
+    auto sf_ready_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 4 + s); };
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * (2 * kStages + 6));
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * (2 * kStages + 6) + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int total_tiles = p.m_tiles * p.n_tiles;
@@ -123,6 +138,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(acc_full_bar(s), 1);
             ptx::mbar_init(acc_empty_bar(s), kEpiWarps);
+            ptx::mbar_init(sf_ready_bar(s), C::kSfWarps > 0 ? C::kSfWarps : 1);
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -164,14 +180,16 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                         const int rc0 = n0 >> 7;
                         int n_rc = 0;
                         for (int rc = 0; rc < C::kSfRowChunksB; ++rc) n_rc += (rc0 + rc < row_chunks_n);
-                        tx += static_cast<uint32_t>(nchunk * 512 * (1 + n_rc));
+                        const bool sf_load = !(kTuning && (p.dbg & kDbgNoSfLoad));
+                        if (sf_load) tx += static_cast<uint32_t>(nchunk * 512 * (1 + n_rc));
                         ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
                         const uint32_t ssfa = sb + C::kBBytes;
                         const uint32_t ssfb = ssfa + C::kSfaBytes;
-                        ptx::bulk_load_1d(ssfa, p.sfa + (static_cast<int64_t>(mt) * chunks_k + kt * 4) * 512,
-                                          nchunk * 512, full_bar(stage));
+                        if (sf_load)
+                            ptx::bulk_load_1d(ssfa, p.sfa + (static_cast<int64_t>(mt) * chunks_k + kt * 4) * 512,
+                                              nchunk * 512, full_bar(stage));
                         for (int rc = 0; rc < C::kSfRowChunksB; ++rc) {
-                            if (rc0 + rc < row_chunks_n)
+                            if (sf_load && rc0 + rc < row_chunks_n)
                                 ptx::bulk_load_1d(ssfb + rc * 2048,
                                                   p.sfb + (static_cast<int64_t>(rc0 + rc) * chunks_k + kt * 4) * 512,
                                                   nchunk * 512, full_bar(stage));
@@ -204,6 +222,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             }
             int stage = 0;
             uint32_t phase = 0;
+            uint32_t gi = 0;  // k-tiles issued so far by this CTA
             bool ok = true;
             int it = 0;
             for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x, ++it) {
@@ -228,30 +247,80 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                     const int k_left = p.K - kt * C::kBK;
                     const int nmma = min(kMmasPerStage, (k_left + C::kMmaK - 1) / C::kMmaK);
                     if (C::kFp4) {
-                        const uint32_t ssfa = sb + C::kBBytes;
-                        const uint32_t ssfb = ssfa + C::kSfaBytes;
-                        for (int j = 0; j < nmma; ++j) {
-                            ptx::tc_copy_sf(tmem_base + C::kSfaCol + 4 * j, ptx::smem_desc_sf(ssfa + j * 512));
-                            for (int rc = 0; rc < C::kSfRowChunksB; ++rc)
-                                ptx::tc_copy_sf(tmem_base + C::kSfbCol + 4 * C::kSfRowChunksB * j + 4 * rc,
-                                                ptx::smem_desc_sf(ssfb + rc * 2048 + j * 512));
+                        // scale factors of this k-tile were copied into TMEM buffer gi&1 by the copy warps
+                        const uint32_t sf_buf = gi & 1u;
+                        if (!(kTuning && (p.dbg & kDbgNoSfCopy)) &&
+                            !wait_bounded(sf_ready_bar(sf_buf), (gi >> 1) & 1u, abort_flag, p.status, 0x500u | sf_buf)) {
+                            ok = false;
+                            break;
                         }
-                        for (int j = 0; j < nmma; ++j)
-                            ptx::mma_nvfp4(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc,
-                                           tmem_base + C::kSfaCol + 4 * j,
-                                           tmem_base + C::kSfbCol + 4 * C::kSfRowChunksB * j + sfb_shift,
-                                           (kt | j) != 0);
+                        ptx::tc_fence_after_sync();
+                        const uint32_t sfa_t = tmem_base + C::kSfCol + sf_buf * C::kSfBufCols;
+                        const uint32_t sfb_t = sfa_t + 16 + sfb_shift;
+                        for (int j = 0; j < nmma && !(kTuning && (p.dbg & kDbgNoMma)); ++j)
+                            ptx::mma_nvfp4(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, sfa_t + 4 * j,
+                                           sfb_t + 4 * C::kSfRowChunksB * j, (kt | j) != 0);
                     } else {
-                        for (int j = 0; j < nmma; ++j)
+                        for (int j = 0; j < nmma && !(kTuning && (p.dbg & kDbgNoMma)); ++j)
                             ptx::mma_bf16(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, (kt | j) != 0);
                     }
                     ptx::tc_commit(empty_bar(stage));  // frees the stage once these MMAs have read it
+                    ++gi;
                     if (++stage == kStages) {
                         stage = 0;
                         phase ^= 1u;
                     }
                 }
                 if (ok) ptx::tc_commit(acc_full_bar(as));
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------ scale-factor copy warps (NVFP4)
+        // tcgen05.cp holds its issuing warp for ~100 cycles, so the copies are spread over four
+        // warps (one per MMA of a stage) and kept off the MMA-issuing thread.  Warp j copies the
+        // scales of k-block j: one 512-byte chunk of A and one per 128-row chunk of B.
+        if (lane == 0 && !(kTuning && (p.dbg & kDbgNoSfCopy))) {
+            const int j = warp - 6;
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t gi = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+                for (int kt = 0; kt < k_tiles; ++kt) {
+                    if (!wait_bounded(full_bar(stage), phase, abort_flag, p.status, 0x600u | stage)) {
+                        ok = false;
+                        break;
+                    }
+                    if (gi >= 2) {
+                        // buffer gi&1 was last read by the MMAs of k-tile gi-2; their commit frees its stage
+                        const uint32_t g2 = gi - 2;
+                        if (!wait_bounded(empty_bar(g2 % kStages), (g2 / kStages) & 1u, abort_flag, p.status,
+                                          0x700u | (g2 % kStages))) {
+                            ok = false;
+                            break;
+                        }
+                    }
+                    ptx::tc_fence_after_sync();
+                    const int k_left = p.K - kt * C::kBK;
+                    const int nmma = min(kMmasPerStage, (k_left + C::kMmaK - 1) / C::kMmaK);
+                    const uint32_t sf_buf = gi & 1u;
+                    if (j < nmma) {
+                        const uint32_t ssfa = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
+                        const uint32_t ssfb = ssfa + C::kSfaBytes;
+                        const uint32_t sfa_t = tmem_base + C::kSfCol + sf_buf * C::kSfBufCols;
+                        ptx::tc_copy_sf(sfa_t + 4 * j, ptx::smem_desc_sf(ssfa + j * 512));
+                        for (int rc = 0; rc < C::kSfRowChunksB; ++rc)
+                            ptx::tc_copy_sf(sfa_t + 16 + 4 * C::kSfRowChunksB * j + 4 * rc,
+                                            ptx::smem_desc_sf(ssfb + rc * 2048 + j * 512));
+                    }
+                    ptx::tc_commit(sf_ready_bar(sf_buf));
+                    ++gi;
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
             }
         }
         __syncwarp();
@@ -271,6 +340,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
             if (!wait_bounded(acc_full_bar(as), acc_parity, abort_flag, p.status, 0x400u | as)) break;
             ptx::tc_fence_after_sync();
             const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + as * kBN;
+            if (kTuning && (p.dbg & kDbgNoEpilogue)) {
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(acc_empty_bar(as));
+                continue;
+            }
 #pragma unroll 1
             for (int c = 0; c < kBN / 64; ++c) {
                 const uint32_t sbuf = epi_warp + buf * kEpiBufBytes;
@@ -314,7 +389,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    if (n0 + c * 64 < p.N && m0 < p.M) ptx::tma_store_2d(&tm_y, n0 + c * 64, m0, sbuf);
+                    if (n0 + c * 64 < p.N && m0 < p.M && !(kTuning && (p.dbg & kDbgNoStore)))
+                        ptx::tma_store_2d(&tm_y, n0 + c * 64, m0, sbuf);
                     ptx::tma_store_commit();
                 }
                 buf ^= 1u;
@@ -344,11 +420,14 @@ sol_status_t launch(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUte
             return SOL_ERR_CUDA;
         configured[dev->device] = true;
     }
+#ifdef SOL_TUNING
+    if (const char *e = getenv("SOL_DBG")) p.dbg = static_cast<uint32_t>(atoi(e));
+#endif
     p.m_tiles = static_cast<int>(ceil_div(p.M, kBM));
     p.n_tiles = static_cast<int>(ceil_div(p.N, kBN));
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
     const int grid = static_cast<int>(tiles < dev->sm_count ? tiles : dev->sm_count);
-    kern<<<grid, kThreads, C::kSmemBytes, stream>>>(tm_a, tm_b, tm_y, p);
+    kern<<<grid, C::kThreads, C::kSmemBytes, stream>>>(tm_a, tm_b, tm_y, p);
     return launch_status();
 }
 
