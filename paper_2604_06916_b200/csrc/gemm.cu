@@ -11,25 +11,11 @@
 // main loop of tile i+1.  Each stage holds 128 bytes of K per row (64 BF16 or 256 FP4), i.e.
 // four MMA instructions.  Every mbarrier wait is bounded: on expiry the CTA records a code in
 // the device status word and leaves through the normal teardown.
-#include "ptx.cuh"
-#include "sol_internal.h"
-
-#include <cuda_bf16.h>
-#include <cstdlib>
+#include "gemm_common.cuh"
 
 namespace sol {
+namespace gemm {
 namespace {
-
-enum class Kind { kBf16, kNvfp4 };
-
-constexpr int kBM = 128;
-constexpr int kRowBytes = 128;        // bytes of K per row per stage (one swizzle atom wide)
-constexpr int kMmasPerStage = 4;      // 32 bytes of K per MMA
-constexpr int kEpiWarps = 4;
-constexpr int kEpiBufBytes = 32 * 128;  // 32 rows x 64 BF16
-constexpr int kTmemCols = 512;
-constexpr int kGroupM = 8;            // tile raster: groups of 8 row tiles sweep all column tiles
-constexpr long long kWaitLimitCycles = 4000000000LL;
 
 template <Kind kKind, int kBN, int kStages>
 struct Cfg {
@@ -58,52 +44,6 @@ struct Cfg {
     static_assert(kSfCol + kSfBufs * kSfBufCols <= kTmemCols, "TMEM budget");
     static_assert(kSmemBytes <= 232448, "shared memory budget");
 };
-
-// Diagnostic switches, compiled in only with -DSOL_TUNING (never in the product build): they
-// drop one part of the pipeline so its share of the time can be read off a timing run.
-#ifdef SOL_TUNING
-constexpr bool kTuning = true;
-#else
-constexpr bool kTuning = false;
-#endif
-enum : uint32_t { kDbgNoSfCopy = 1, kDbgNoMma = 2, kDbgNoEpilogue = 4, kDbgNoSfLoad = 8, kDbgNoStore = 16 };
-
-struct Params {
-    const uint8_t *sfa;    // scales of A, chunked layout (NVFP4 only)
-    const uint8_t *sfb;
-    const float *ts_a;     // per-tensor scales (NVFP4 only)
-    const float *ts_b;
-    const uint16_t *bias;  // BF16 [N] or null
-    uint32_t *status;
-    uint32_t dbg;
-    int M, N, K;
-    int m_tiles, n_tiles;
-};
-
-__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                             uint32_t *status, uint32_t code) {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!ptx::mbar_try_wait(bar, parity)) {
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
-            *abort_flag = 1;
-            atomicExch(status, code);
-            return false;
-        }
-    }
-    return true;
-}
-
-__device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int &mt, int &nt) {
-    const int per_group = kGroupM * n_tiles;
-    const int g = t / per_group;
-    const int first = g * kGroupM;
-    const int gsize = min(kGroupM, m_tiles - first);
-    const int r = t - g * per_group;
-    mt = first + r % gsize;
-    nt = r / gsize;
-}
 
 template <Kind kKind, int kBN, int kStages>
 __global__ void __launch_bounds__((Cfg<kKind, kBN, kStages>::kThreads), 1)
@@ -346,55 +286,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
                 if (lane == 0) ptx::mbar_arrive(acc_empty_bar(as));
                 continue;
             }
-#pragma unroll 1
-            for (int c = 0; c < kBN / 64; ++c) {
-                const uint32_t sbuf = epi_warp + buf * kEpiBufBytes;
-                if (lane == 0) ptx::tma_store_wait_read<1>();  // the store issued two chunks ago has left sbuf
-                __syncwarp();
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t acc[32];
-                    ptx::tmem_ld_32x32(t_acc + c * 64 + h * 32, acc);
-                    ptx::tmem_ld_wait();
-                    if (c == kBN / 64 - 1 && h == 1) {
-                        // accumulator fully read: hand the TMEM stage back to the MMA warp
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(acc_empty_bar(as));
-                    }
-                    const int nb = n0 + c * 64 + h * 32;
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {  // 8 columns -> one 16-byte shared store
-                        uint4 bb = make_uint4(0, 0, 0, 0);
-                        if (p.bias != nullptr && nb + g * 8 < p.N)
-                            bb = __ldg(reinterpret_cast<const uint4 *>(p.bias + nb + g * 8));
-                        const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
-                        uint32_t o[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float b0 = __uint_as_float(bw[e] << 16);
-                            const float b1 = __uint_as_float(bw[e] & 0xFFFF0000u);
-                            const float y0 = fmaf(__uint_as_float(acc[g * 8 + 2 * e]), alpha, b0);
-                            const float y1 = fmaf(__uint_as_float(acc[g * 8 + 2 * e + 1]), alpha, b1);
-                            __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
-                            o[e] = *reinterpret_cast<uint32_t *>(&pk);
-                        }
-                        const uint32_t chunk16 = static_cast<uint32_t>(h * 4 + g) ^ (lane & 7u);  // 128-byte swizzle
-                        const uint32_t dst = sbuf + lane * 128 + chunk16 * 16;
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]),
-                                     "r"(o[2]), "r"(o[3])
-                                     : "memory");
-                    }
-                }
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    if (n0 + c * 64 < p.N && m0 < p.M && !(kTuning && (p.dbg & kDbgNoStore)))
-                        ptx::tma_store_2d(&tm_y, n0 + c * 64, m0, sbuf);
-                    ptx::tma_store_commit();
-                }
-                buf ^= 1u;
-            }
+            epilogue_tile<kBN>(&tm_y, p, t_acc, m0, n0, alpha, epi_warp, buf, lane,
+                               [&] { ptx::mbar_arrive(acc_empty_bar(as)); });
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();
     }
@@ -433,7 +326,7 @@ sol_status_t launch(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const CUte
 
 }  // namespace
 
-sol_status_t launch_gemm_bf16(const void *x, const void *w, const void *bias, void *y, int64_t M, int64_t N,
+sol_status_t launch_single_bf16(const void *x, const void *w, const void *bias, void *y, int64_t M, int64_t N,
                               int64_t K, int64_t ldx, int64_t ldw, int64_t ldy, cudaStream_t stream,
                               const DeviceInfo *dev) {
     constexpr int kBN = 256;
@@ -454,7 +347,7 @@ sol_status_t launch_gemm_bf16(const void *x, const void *w, const void *bias, vo
     return launch<Kind::kBf16, kBN, 4>(tm_a, tm_b, tm_y, p, stream, dev);
 }
 
-sol_status_t launch_gemm_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
+sol_status_t launch_single_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
                                const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
                                int64_t N, int64_t K, int64_t ldy, cudaStream_t stream,
                                const DeviceInfo *dev) {
@@ -478,6 +371,32 @@ sol_status_t launch_gemm_nvfp4(const void *xq, const void *xsf, const float *xts
     p.N = static_cast<int>(N);
     p.K = static_cast<int>(K);
     return launch<Kind::kNvfp4, kBN, 4>(tm_a, tm_b, tm_y, p, stream, dev);
+}
+
+}  // namespace gemm
+
+// Pair tiles (two CTAs per MMA) halve the weight-tile traffic per SM; a single 128-row tile is
+// enough when the whole problem has at most 128 rows.
+sol_status_t launch_gemm_bf16(const void *x, const void *w, const void *bias, void *y, int64_t M, int64_t N,
+                              int64_t K, int64_t ldx, int64_t ldw, int64_t ldy, cudaStream_t stream,
+                              const DeviceInfo *dev) {
+#ifdef SOL_TUNING
+    if (getenv("SOL_FORCE_SINGLE")) return gemm::launch_single_bf16(x, w, bias, y, M, N, K, ldx, ldw, ldy, stream, dev);
+#endif
+    if (M <= 128) return gemm::launch_single_bf16(x, w, bias, y, M, N, K, ldx, ldw, ldy, stream, dev);
+    return gemm::launch_pair_bf16(x, w, bias, y, M, N, K, ldx, ldw, ldy, stream, dev);
+}
+
+sol_status_t launch_gemm_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
+                               const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
+                               int64_t N, int64_t K, int64_t ldy, cudaStream_t stream,
+                               const DeviceInfo *dev) {
+#ifdef SOL_TUNING
+    if (getenv("SOL_FORCE_SINGLE"))
+        return gemm::launch_single_nvfp4(xq, xsf, xts, wq, wsf, wts, bias, y, M, N, K, ldy, stream, dev);
+#endif
+    if (M <= 128) return gemm::launch_single_nvfp4(xq, xsf, xts, wq, wsf, wts, bias, y, M, N, K, ldy, stream, dev);
+    return gemm::launch_pair_nvfp4(xq, xsf, xts, wq, wsf, wts, bias, y, M, N, K, ldy, stream, dev);
 }
 
 }  // namespace sol

@@ -51,4 +51,9 @@ bool make_tmap_2d(CUtensorMap *out, CUtensorMapDataType dtype, uint32_t elem_byt
                   uint64_t inner, uint64_t outer, uint64_t pitch_bytes, uint32_t box_inner,
                   uint32_t box_outer, CUtensorMapSwizzle swizzle);
 
+// Scale-factor buffer in the chunked layout as a 3-D tensor [row chunk][k chunk][128 x u32]; the box
+// covers 4 k-chunks of `box_row_chunks` row chunks (out-of-range chunks read as zero).
+bool make_tmap_sf(CUtensorMap *out, const void *base, uint64_t chunks_k, uint64_t row_chunks,
+                  uint32_t box_row_chunks);
+
 }  // namespace sol
