@@ -144,6 +144,29 @@ sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *
                                    size_t workspace_bytes, void *stream);
 
 /*
+ * (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
+ *
+ * Same computation and result as nvfp4_quantize_linear, but without a workspace argument: the
+ * scratch for the quantized activations lives in a fixed 64 MiB device array that is part of the
+ * library image, so the call performs no device allocation of any kind.  It is meant for callers
+ * that are handed input and output buffers only, or that run after their memory pool has been
+ * frozen (serving loops, plugins, frameworks that forbid allocation once set up).
+ *   - Problems whose scratch (sol_nvfp4_linear_workspace_bytes(M, N, K)) exceeds
+ *     sol_nvfp4_static_scratch_bytes() are rejected with SOL_ERR_WORKSPACE_TOO_SMALL; nothing is launched.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents.  Calls
+ *     that may overlap on the GPU (different streams, or several host threads) race on it and give
+ *     undefined results; serialise them.  Every GPU that loads the library holds the array until
+ *     the process exits.
+ */
+size_t sol_nvfp4_static_scratch_bytes(void);
+sol_status_t nvfp4_quantize_linear_static(const void *x_bf16, int64_t ldx, const void *wq,
+                                          const void *wsf, const float *w_tscale,
+                                          const void *bias_bf16, void *y_bf16, int64_t M, int64_t N,
+                                          int64_t K, int64_t ldy, void *stream);
+
+/*
  * Device-side waits in the GEMM kernels are bounded; a wait that runs out records a code
  * in a device status word and the kernel returns.  This call synchronises `stream`, reads
  * that word, clears it, and returns SOL_ERR_TIMEOUT if it was set, SOL_ERR_CUDA if the

@@ -21,6 +21,7 @@ EXPORTS = [
     "sol_status_string", "sol_nvfp4_data_bytes", "sol_nvfp4_scale_bytes",
     "sol_nvfp4_linear_workspace_bytes", "sol_amax_bf16", "nvfp4_quantize", "nvfp4_quantize_weight",
     "nvfp4_linear", "bf16_linear", "nvfp4_quantize_linear", "sol_last_device_status",
+    "sol_nvfp4_static_scratch_bytes", "nvfp4_quantize_linear_static",
 ]
 
 _lib = None
@@ -58,6 +59,9 @@ def lib() -> ctypes.CDLL:
     L.bf16_linear.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, vp]
     L.nvfp4_quantize_linear.restype = i32
     L.nvfp4_quantize_linear.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, sz, vp]
+    L.sol_nvfp4_static_scratch_bytes.restype, L.sol_nvfp4_static_scratch_bytes.argtypes = sz, []
+    L.nvfp4_quantize_linear_static.restype = i32
+    L.nvfp4_quantize_linear_static.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -175,6 +179,25 @@ def nvfp4_quantize_linear(x, wq, wsf, w_tscale, bias=None, workspace: torch.Tens
     _check(lib().nvfp4_quantize_linear(_ptr(x), x.stride(0), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
                                        _ptr(out), M, N, K, out.stride(0), _ptr(workspace), workspace.numel(),
                                        _stream()), "nvfp4_quantize_linear")
+    return out
+
+
+def static_scratch_bytes() -> int:
+    return lib().sol_nvfp4_static_scratch_bytes()
+
+
+def nvfp4_quantize_linear_static(x, wq, wsf, w_tscale, bias=None, out: torch.Tensor | None = None):
+    """nvfp4_quantize_linear for callers that may not allocate: the scratch is a fixed array inside
+    the library (64 MiB, shared by every call on the device; overlapping calls race).  Only the output
+    tensor is created here when `out` is not given -- pass `out` to allocate nothing at all."""
+    _need_2d_bf16(x, "x")
+    M, K = x.shape
+    N = wq.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    _check(lib().nvfp4_quantize_linear_static(_ptr(x), x.stride(0), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
+                                              _ptr(out), M, N, K, out.stride(0), _stream()),
+           "nvfp4_quantize_linear_static")
     return out
 
 
