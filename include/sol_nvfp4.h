@@ -144,6 +144,20 @@ sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *
                                    size_t workspace_bytes, void *stream);
 
 /*
+ * The fused entry for HOST activations and outputs (the end-to-end path a caller with data in host
+ * memory takes): copies X host -> x_dev, runs nvfp4_quantize_linear, copies y_dev -> Y host, all
+ * queued on `stream` (truly asynchronous only if the host buffers are pinned).
+ *   x_host, y_host  HOST pointers, BF16 [M, K] / [M, N], pitches ldx / ldy in elements
+ *   x_dev, y_dev    device staging buffers, dense [M, K] / [M, N] BF16, 16-byte aligned
+ *   weights, bias, workspace: device, as for nvfp4_quantize_linear
+ */
+sol_status_t nvfp4_quantize_linear_host(const void *x_host, int64_t ldx, const void *wq,
+                                        const void *wsf, const float *w_tscale,
+                                        const void *bias_bf16, void *y_host, int64_t M, int64_t N,
+                                        int64_t K, int64_t ldy, void *x_dev, void *y_dev,
+                                        void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
  *
  * Same computation and result as nvfp4_quantize_linear, but without a workspace argument: the

@@ -21,7 +21,7 @@ EXPORTS = [
     "sol_status_string", "sol_nvfp4_data_bytes", "sol_nvfp4_scale_bytes",
     "sol_nvfp4_linear_workspace_bytes", "sol_amax_bf16", "nvfp4_quantize", "nvfp4_quantize_weight",
     "nvfp4_linear", "bf16_linear", "nvfp4_quantize_linear", "sol_last_device_status",
-    "sol_nvfp4_static_scratch_bytes", "nvfp4_quantize_linear_static",
+    "sol_nvfp4_static_scratch_bytes", "nvfp4_quantize_linear_static", "nvfp4_quantize_linear_host",
 ]
 
 _lib = None
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
     L.sol_nvfp4_static_scratch_bytes.restype, L.sol_nvfp4_static_scratch_bytes.argtypes = sz, []
     L.nvfp4_quantize_linear_static.restype = i32
     L.nvfp4_quantize_linear_static.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp]
+    L.nvfp4_quantize_linear_host.restype = i32
+    L.nvfp4_quantize_linear_host.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, vp, sz, vp]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -180,6 +182,17 @@ def nvfp4_quantize_linear(x, wq, wsf, w_tscale, bias=None, workspace: torch.Tens
                                        _ptr(out), M, N, K, out.stride(0), _ptr(workspace), workspace.numel(),
                                        _stream()), "nvfp4_quantize_linear")
     return out
+
+
+def nvfp4_quantize_linear_host(x_host, wq, wsf, w_tscale, bias, y_host, x_dev, y_dev, workspace):
+    """End-to-end form: host X (ideally pinned) -> device, fused quantize + NVFP4 linear, Y -> host."""
+    M, K = x_host.shape
+    N = wq.shape[0]
+    _check(lib().nvfp4_quantize_linear_host(_ptr(x_host), x_host.stride(0), _ptr(wq), _ptr(wsf), _ptr(w_tscale),
+                                            _ptr(bias), _ptr(y_host), M, N, K, y_host.stride(0), _ptr(x_dev),
+                                            _ptr(y_dev), _ptr(workspace), workspace.numel(), _stream()),
+           "nvfp4_quantize_linear_host")
+    return y_host
 
 
 def static_scratch_bytes() -> int:

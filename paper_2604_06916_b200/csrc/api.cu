@@ -258,6 +258,36 @@ sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *
     return launch_gemm_nvfp4(xq, xsf, xts, wq, wsf, w_tscale, bias_bf16, y_bf16, M, N, K, ldy, s, dev);
 }
 
+sol_status_t nvfp4_quantize_linear_host(const void *x_host, int64_t ldx, const void *wq, const void *wsf,
+                                        const float *w_tscale, const void *bias_bf16, void *y_host, int64_t M,
+                                        int64_t N, int64_t K, int64_t ldy, void *x_dev, void *y_dev,
+                                        void *workspace, size_t workspace_bytes, void *stream) {
+    if (x_host == nullptr || y_host == nullptr || x_dev == nullptr || y_dev == nullptr) return SOL_ERR_NULL_POINTER;
+    if (M <= 0 || N <= 0 || K <= 0 || ldx < K || ldy < N) return SOL_ERR_BAD_SHAPE;
+    // validate everything else (and the device) before the first copy is queued
+    if (wq == nullptr || wsf == nullptr || w_tscale == nullptr || workspace == nullptr) return SOL_ERR_NULL_POINTER;
+    sol_status_t st = check_linear_common(bias_bf16, y_dev, M, N, K, N);
+    if (st != SOL_OK) return st;
+    if (!aligned16(x_dev) || !aligned16(wq) || !aligned16(wsf) || (reinterpret_cast<uintptr_t>(w_tscale) & 3u) ||
+        (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return SOL_ERR_ALIGNMENT;
+    if (workspace_bytes < sol_nvfp4_linear_workspace_bytes(M, N, K)) return SOL_ERR_WORKSPACE_TOO_SMALL;
+    const DeviceInfo *dev = nullptr;
+    st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpy2DAsync(x_dev, static_cast<size_t>(K) * 2, x_host, static_cast<size_t>(ldx) * 2,
+                          static_cast<size_t>(K) * 2, static_cast<size_t>(M), cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return SOL_ERR_CUDA;
+    st = nvfp4_quantize_linear(x_dev, K, wq, wsf, w_tscale, bias_bf16, y_dev, M, N, K, N, workspace, workspace_bytes,
+                               stream);
+    if (st != SOL_OK) return st;
+    if (cudaMemcpy2DAsync(y_host, static_cast<size_t>(ldy) * 2, y_dev, static_cast<size_t>(N) * 2,
+                          static_cast<size_t>(N) * 2, static_cast<size_t>(M), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return SOL_ERR_CUDA;
+    return SOL_OK;
+}
+
 sol_status_t sol_last_device_status(void *stream, uint32_t *detail_out) {
     const DeviceInfo *dev = nullptr;
     sol_status_t st = check_arch(&dev);

@@ -1,0 +1,140 @@
+"""CPU-only checks of the boundary: the shared library loads and exports every symbol the header
+declares, size queries, argument validation (no kernel is launched on an error), and the
+multi-rank timing aggregation on a world-size-2 gloo group."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "sol_nvfp4.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2604_06916_b200 import build
+
+    path = build.build()
+    from paper_2604_06916_b200 import binding
+
+    return binding.lib()
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b([a-z_0-9]+)\s*\(", text)) - {"defined"})
+
+
+def test_library_exports_every_declared_symbol(lib):
+    from paper_2604_06916_b200 import binding
+
+    names = declared_functions()
+    assert set(binding.EXPORTS) == set(names)
+    raw = ctypes.CDLL(binding.LIB_PATH)
+    for n in names:
+        assert hasattr(raw, n), n
+
+
+def test_status_strings(lib):
+    from paper_2604_06916_b200 import binding as B
+
+    assert B.status_string(0) == "SOL_OK"
+    assert B.status_string(4) == "SOL_ERR_WORKSPACE_TOO_SMALL"
+    assert B.status_string(7) == "SOL_ERR_TIMEOUT"
+    assert B.status_string(99) == "SOL_ERR_UNKNOWN"
+
+
+def test_size_queries(lib):
+    from paper_2604_06916_b200 import binding as B
+
+    assert B.data_bytes(256, 512) == 256 * 256
+    assert B.scale_bytes(256, 512, B.SF_ROW_MAJOR) == 256 * 32
+    assert B.scale_bytes(256, 512, B.SF_SWIZZLED_128x4) == 2 * 8 * 512
+    assert B.scale_bytes(130, 160, B.SF_SWIZZLED_128x4) == 2 * 3 * 512       # padded rows and k chunks
+    assert B.scale_bytes(40, 5600, B.SF_SWIZZLED_128x4) == 1 * 88 * 512
+    assert B.data_bytes(16, 24) == 0 and B.scale_bytes(0, 64) == 0            # K % 32, rows > 0
+    ws = B.linear_workspace_bytes(36864, 3072, 3072)
+    assert ws >= B.data_bytes(36864, 3072) + B.scale_bytes(36864, 3072) + 4 and ws % 256 == 0
+    assert B.static_scratch_bytes() == 64 << 20
+
+
+def test_argument_validation_happens_before_any_cuda_call(lib):
+    """Bad arguments are refused on the host; this box has no GPU, so reaching CUDA would fail differently."""
+    L = lib
+    buf = ctypes.create_string_buffer(4096)
+    p = (ctypes.addressof(buf) + 255) & ~255   # aligned fake pointer, never dereferenced
+    NULLP, SHAPE, ALIGN, WS, LAYOUT = 1, 2, 3, 4, 8
+    assert L.sol_amax_bf16(None, 4, 64, 64, p, None) == NULLP
+    assert L.sol_amax_bf16(p, 4, 48, 48, p, None) == SHAPE                     # K % 32
+    assert L.sol_amax_bf16(p, 4, 64, 32, p, None) == SHAPE                     # ld < K
+    assert L.sol_amax_bf16(p + 2, 4, 64, 64, p, None) == ALIGN
+    assert L.nvfp4_quantize(p, 4, 64, 64, None, p, p, 1, None) == NULLP
+    assert L.nvfp4_quantize(p, 4, 64, 64, p, p, p, 5, None) == LAYOUT
+    assert L.nvfp4_quantize(p, 0, 64, 64, p, p, p, 1, None) == SHAPE
+    assert L.nvfp4_quantize(p, 4, 64, 68, p, p, p, 1, None) == ALIGN           # pitch not a multiple of 8
+    assert L.nvfp4_quantize_weight(p, 4, 64, 64, p, p, None, 1, None) == NULLP
+    assert L.nvfp4_linear(p, p, p, p, p, p, None, None, 4, 8, 64, 8, None) == NULLP
+    assert L.nvfp4_linear(p, p, p, p, p, p, None, p, 4, 12, 64, 16, None) == SHAPE   # N % 8
+    assert L.nvfp4_linear(p, p, p, p, p, p, None, p, 4, 8, 64, 4, None) == SHAPE     # ldy < N
+    assert L.nvfp4_linear(p, p, p, p, p, p, p + 8, p, 4, 8, 64, 8, None) == ALIGN    # bias alignment
+    assert L.bf16_linear(p, p, None, p, 4, 8, 64, 32, 64, 8, None) == SHAPE          # ldx < K
+    assert L.bf16_linear(None, p, None, p, 4, 8, 64, 64, 64, 8, None) == NULLP
+    assert L.nvfp4_quantize_linear(p, 64, p, p, p, None, p, 4, 8, 64, 8, None, 0, None) == NULLP
+    assert L.nvfp4_quantize_linear(p, 64, p, p, p, None, p, 4, 8, 64, 8, p, 16, None) == WS
+    assert L.nvfp4_quantize_linear(p, 64, p, p, p, None, p, 4, 8, 64, 8, p + 16, 1 << 20, None) == ALIGN
+    assert L.nvfp4_quantize_linear_static(p, 4096, p, p, p, None, p, 1 << 20, 8, 4096, 8, None) == WS
+    assert L.nvfp4_quantize_linear_static(None, 64, p, p, p, None, p, 4, 8, 64, 8, None) == NULLP
+
+
+def test_binding_refuses_to_run_without_the_library(tmp_path):
+    code = ("import os, sys; sys.path.insert(0, %r); os.environ['SOL_NVFP4_LIB'] = %r\n"
+            "from paper_2604_06916_b200 import binding\n"
+            "try:\n    binding.lib()\nexcept FileNotFoundError as e:\n    print('refused'); sys.exit(0)\n"
+            "sys.exit(1)\n") % (ROOT, str(tmp_path / "missing.so"))
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0 and "refused" in out.stdout, out.stderr
+
+
+WORKER = r"""
+import os, sys
+sys.path.insert(0, %r)
+import torch.distributed as dist
+from paper_2604_06916_b200 import replicas
+rank = int(os.environ["RANK"])
+dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d", rank=rank, world_size=2)
+dist.barrier()
+ms, units, world = replicas.aggregate(10.0 + 5.0 * rank, 100.0)
+assert (ms, units, world) == (15.0, 200.0, 2), (ms, units, world)
+assert abs(replicas.throughput(10.0 + 5.0 * rank, 100.0) - 200.0 / 15e-3) < 1e-6
+dist.barrier()
+dist.destroy_process_group()
+print("rank", rank, "ok")
+"""
+
+
+def test_replica_aggregation_world_size_2_gloo():
+    import socket
+
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    procs = []
+    for rank in range(2):
+        env = dict(os.environ, RANK=str(rank), WORLD_SIZE="2", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, "-c", WORKER % (ROOT, port)], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True))
+    for rank, pr in enumerate(procs):
+        out, err = pr.communicate(timeout=300)
+        assert pr.returncode == 0, err
+        assert f"rank {rank} ok" in out
+
+
+def test_replica_aggregation_without_a_process_group():
+    from paper_2604_06916_b200 import replicas
+
+    assert replicas.aggregate(3.0, 7.0) == (3.0, 7.0, 1)

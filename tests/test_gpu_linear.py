@@ -164,6 +164,20 @@ def test_flux_shaped_layers_sampled_rows(B, index):
     run_layer_sampled(B, workloads.CONFIG_FLUX, index)
 
 
+def test_host_buffer_entry_matches_device_entry(B):
+    cfg = workloads.CONFIG_SANA
+    X, W, bias = workloads.make_layer(cfg, 1, "cuda", M=2500)
+    wq, wsf, wts = B.nvfp4_quantize_weight(W)
+    want = B.nvfp4_quantize_linear(X, wq, wsf, wts, bias)
+    xh = torch.empty(X.shape[0], X.shape[1] + 8, dtype=torch.bfloat16).pin_memory()[:, :X.shape[1]]
+    xh.copy_(X)
+    yh = torch.zeros(want.shape[0], want.shape[1] + 16, dtype=torch.bfloat16).pin_memory()[:, :want.shape[1]]
+    ws = torch.empty(B.linear_workspace_bytes(*want.shape, X.shape[1]), dtype=torch.uint8, device="cuda")
+    B.nvfp4_quantize_linear_host(xh, wq, wsf, wts, bias, yh, torch.empty_like(X), torch.empty_like(want), ws)
+    B.sol_last_device_status()
+    assert torch.equal(yh, want.cpu())
+
+
 def test_deterministic_run_to_run(B):
     cfg = workloads.CONFIG_SANA
     X, W, bias = workloads.make_layer(cfg, 1, "cuda", M=4096)
