@@ -396,7 +396,10 @@ sol_status_t launch_gemm_nvfp4(const void *xq, const void *xsf, const float *xts
         return gemm::launch_single_nvfp4(xq, xsf, xts, wq, wsf, wts, bias, y, M, N, K, ldy, stream, dev);
 #endif
     if (M <= 128) return gemm::launch_single_nvfp4(xq, xsf, xts, wq, wsf, wts, bias, y, M, N, K, ldy, stream, dev);
-    return gemm::launch_pair_nvfp4(xq, xsf, xts, wq, wsf, wts, bias, y, M, N, K, ldy, stream, dev);
+#ifdef SOL_TUNING
+    if (getenv("SOL_PAIR192")) return gemm::launch_pair_nvfp4(xq, xsf, xts, wq, wsf, wts, bias, y, M, N, K, ldy, stream, dev);
+#endif
+    return gemm::launch_pair256_nvfp4(xq, xsf, xts, wq, wsf, wts, bias, y, M, N, K, ldy, stream, dev);
 }
 
 }  // namespace sol

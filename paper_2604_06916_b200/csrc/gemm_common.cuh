@@ -146,6 +146,9 @@ sol_status_t launch_pair_bf16(const void *x, const void *w, const void *bias, vo
 sol_status_t launch_pair_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
                                const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
                                int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev);
+sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
+                                  const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
+                                  int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev);
 
 }  // namespace gemm
 }  // namespace sol

@@ -6,9 +6,9 @@
 // reported to the even CTA's barrier.
 //
 // Warps per CTA: 0 = TMA producer, 1 = TMEM owner (+ MMA issuer in the even CTA), 2..5 = epilogue,
-// 6..9 = scale-factor copy warps (NVFP4, even CTA only; tcgen05.cp holds its issuing warp for
-// ~100 cycles, so the copies are spread over four warps and kept off the MMA thread), 10 = TMA
-// producer of the scale-factor tiles (NVFP4).
+// 6..17 = scale-factor copy warps (NVFP4, even CTA only; tcgen05.cp holds its issuing warp for
+// ~100 cycles, so each of the twelve copies of a k-tile has its own warp, off the MMA thread),
+// 18 = TMA producer of the scale-factor tiles (NVFP4).
 // Barriers: full[s] (even CTA; bytes of both CTAs' loads), empty[s] and acc_full[a] (both CTAs,
 // signalled by multicast tcgen05.commit), acc_empty[a] (even CTA, 8 epilogue warps arrive),
 // sf_ready[b] (even CTA).  All waits are bounded.
@@ -33,8 +33,9 @@ struct PairCfg {
     static constexpr int kSfBufs = 2;
     static constexpr int kAccStages = (2 * kBN + kSfBufs * kSfBufCols <= kTmemCols) ? 2 : 1;
     static constexpr int kSfCol = kAccStages * kBN;
-    static constexpr int kSfWarps = kFp4 ? kMmasPerStage : 0;
-    static constexpr int kThreads = 192 + (kFp4 ? 32 * (kSfWarps + 1) : 0);  // + one scale-factor load warp
+    static constexpr int kSfCopiesPerMma = 1 + kSfRowChunksB;          // one 512-byte chunk of A, one per row chunk of B
+    static constexpr int kSfWarps = kFp4 ? kMmasPerStage * kSfCopiesPerMma : 0;  // one tcgen05.cp per warp per k-tile
+    static constexpr int kThreads = 192 + (kFp4 ? 32 * (kSfWarps + 1) : 0);  // + one scale-factor TMA warp
     static constexpr int kEpiBytes = kEpiWarps * 2 * kEpiBufBytes;
     static constexpr int kBarBytes = 256;
     static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kBarBytes + 1024;
@@ -145,7 +146,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             }
         }
         __syncwarp();
-    } else if (warp == 10) {
+    } else if (warp == 6 + C::kSfWarps) {
         // ------------------------------------------------------------ TMA producer: scale factors (NVFP4, both CTAs)
         // Each tensor-copy instruction costs its issuing thread tens of cycles, so the scale tiles get
         // their own thread.  The byte count was announced by the A/B producer of the even CTA.
@@ -280,7 +281,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         // ------------------------------------------------------------ scale-factor copy warps 6..9 (even CTA)
         if (leader && !(kTuning && (p.dbg & kDbgNoSfCopy))) {
             const bool elected = ptx::elect_one();
-            const int j = warp - 6;
+            // warp w copies part (w % copies-per-MMA) of MMA j = w / copies-per-MMA: part 0 = scales of A,
+            // part 1.. = scales of the B tile's 128-row chunks
+            const int j = (warp - 6) / C::kSfCopiesPerMma, part = (warp - 6) % C::kSfCopiesPerMma;
             int stage = 0;
             uint32_t phase = 0;
             uint32_t gi = 0;
@@ -305,14 +308,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                     const uint32_t sf_buf = gi & 1u;
                     if (elected) {
                         if (j < nmma) {
-                            const uint32_t ssfa = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
-                            const uint32_t ssfb = ssfa + C::kSfaBytes;
-                            const uint32_t sfa_t = tmem_base + C::kSfCol + sf_buf * C::kSfBufCols;
-                            ptx::tc_copy_sf_pair(sfa_t + 4 * j, ptx::smem_desc_sf(ssfa + j * 512));
-#pragma unroll
-                            for (int rc = 0; rc < C::kSfRowChunksB; ++rc)
-                                ptx::tc_copy_sf_pair(sfa_t + 16 + 4 * C::kSfRowChunksB * j + 4 * rc,
-                                                     ptx::smem_desc_sf(ssfb + rc * 2048 + j * 512));
+                            const uint32_t ssf = smem_base + stage * C::kStageBytes + C::kABytes + C::kBBytes;
+                            const uint32_t sf_t = tmem_base + C::kSfCol + sf_buf * C::kSfBufCols;
+                            const uint32_t src = part == 0 ? ssf + j * 512 : ssf + C::kSfaBytes + (part - 1) * 2048 + j * 512;
+                            const uint32_t dst = part == 0 ? sf_t + 4 * j
+                                                           : sf_t + 16 + 4 * C::kSfRowChunksB * j + 4 * (part - 1);
+                            ptx::tc_copy_sf_pair(dst, ptx::smem_desc_sf(src));
                         }
                         ptx::tc_commit_pair(sf_ready_bar(sf_buf));
                     }

@@ -1,0 +1,451 @@
+// NVFP4 CTA-pair GEMM with 256 x 256 pair tiles (tcgen05.mma.cta_group::2, kind::mxf4nvf4).
+//
+// Why this shape: one MMA instruction costs its issuing thread 60-70 cycles and a k-tile needs
+// about 250 more for barrier polling and the commit, so the single MMA-issuing thread spends
+// ~500 cycles per k-tile of four MMAs.  Only at N = 256 does the tensor core need that long
+// (4 x 128 cycles); narrower tiles leave it idle.  N = 256 also has the lowest L2 -> SM traffic
+// per flop (38 KB per CTA per k-tile = 74 B/clk, against the SM's 128 B/clk ingest port).
+//
+// TMEM does not hold two 256-column accumulators plus the scale factors, so the two accumulators
+// overlap: A = columns [0,256), B = [160,416), scale-factor buffers 2 x 48 columns at [416,512).
+// Tiles alternate between A and B.  The epilogue drains the shared columns [160,256) first and
+// signals `ovl_free`; the MMAs of the next tile start then, while the rest of the tile is still
+// being converted and stored.  Eight epilogue warps (two per TMEM lane quadrant) halve that wait.
+//
+// Warps per CTA: 0 = TMA producer (A, B); 1 = TMEM owner, MMA issuer in the even CTA;
+// 2..9 = epilogue; 10..21 = scale-factor copy warps (even CTA; tcgen05.cp blocks its warp for
+// ~100 cycles, so each of the twelve copies of a k-tile has its own warp); 22 = TMA producer (scales).
+// No multicast loads; every mbarrier wait is bounded.
+#include "gemm_common.cuh"
+
+namespace sol {
+namespace gemm {
+namespace {
+
+constexpr int kBN = 256;
+constexpr int kStages = 5;
+constexpr int kBK = 256;                       // FP4 elements of K per stage = 128 bytes per row
+constexpr int kMmaK = 64;
+constexpr int kABytes = kBM * kRowBytes;       // 16 KB: this CTA's 128 rows of A
+constexpr int kBBytes = (kBN / 2) * kRowBytes; // 16 KB: this CTA's half of the B tile
+constexpr int kSfaBytes = 2048;                // 4 k-chunks x 512 bytes
+constexpr int kSfbBytes = 4096;                // 2 row chunks x 4 k-chunks x 512 bytes
+constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 38 912
+constexpr int kSfBufCols = 48;                 // per k-tile: 4 MMAs x (4 columns of A + 8 of B)
+constexpr int kAccStride = 160;                // accumulator B starts here; [160,256) is shared
+constexpr int kSfCol = 416;
+constexpr int kEpiWarpsFp4 = 8;
+constexpr int kSfCopyWarps = 12;
+constexpr int kWarps = 2 + kEpiWarpsFp4 + kSfCopyWarps + 1;
+constexpr int kThreadsFp4 = 32 * kWarps;       // 544
+constexpr int kEpiBytes = kEpiWarpsFp4 * kEpiBufBytes;
+constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 256 + 1024;
+static_assert(kSfCol + 2 * kSfBufCols <= kTmemCols && kAccStride + kBN <= kSfCol, "TMEM budget");
+static_assert(kSmemBytes <= 232448, "shared memory budget");
+
+// One 64-column chunk of this warp's 32 accumulator rows: TMEM -> fma(acc, alpha, bias) -> BF16 ->
+// swizzled staging buffer -> TMA store.  `release()` runs as soon as the TMEM loads have completed.
+template <class Release>
+__device__ __forceinline__ void epilogue_chunk(const CUtensorMap *tm_y, const Params &p, uint32_t t_chunk, int m0,
+                                               int nc, float alpha, uint32_t sbuf, int lane, Release release) {
+    if (lane == 0) ptx::tma_store_wait_read<0>();  // the previous store of this warp has left the staging buffer
+    __syncwarp();
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        uint32_t acc[32];
+        ptx::tmem_ld_32x32(t_chunk + h * 32, acc);
+        ptx::tmem_ld_wait();
+        if (h == 1) {  // both halves of the chunk have left TMEM
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) release();
+        }
+        const int nb = nc + h * 32;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            uint4 bb = make_uint4(0, 0, 0, 0);
+            if (p.bias != nullptr && nb + g * 8 < p.N) bb = __ldg(reinterpret_cast<const uint4 *>(p.bias + nb + g * 8));
+            const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float y0 = fmaf(__uint_as_float(acc[g * 8 + 2 * e]), alpha, __uint_as_float(bw[e] << 16));
+                const float y1 =
+                    fmaf(__uint_as_float(acc[g * 8 + 2 * e + 1]), alpha, __uint_as_float(bw[e] & 0xFFFF0000u));
+                __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
+                o[e] = *reinterpret_cast<uint32_t *>(&pk);
+            }
+            const uint32_t chunk16 = static_cast<uint32_t>(h * 4 + g) ^ (lane & 7u);  // 128-byte swizzle
+            const uint32_t dst = sbuf + lane * 128 + chunk16 * 16;
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]),
+                         "r"(o[3])
+                         : "memory");
+        }
+    }
+    ptx::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        if (nc < p.N && m0 < p.M && !(kTuning && (p.dbg & kDbgNoStore))) ptx::tma_store_2d(tm_y, nc, m0, sbuf);
+        ptx::tma_store_commit();
+    }
+}
+
+__global__ void __launch_bounds__(kThreadsFp4, 1)
+gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
+                     const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_sfa,
+                     const __grid_constant__ CUtensorMap tm_sfb, const Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+
+    const uint32_t epi_base = smem_base + kStages * kStageBytes;
+    const uint32_t bar_base = epi_base + kEpiBytes;
+    uint8_t *bar_gen = smem_gen + kStages * kStageBytes + kEpiBytes;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+    auto acc_full_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
+    auto acc_empty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 2 + s); };
+    auto ovl_free_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 4 + s); };
+    auto sf_ready_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 6 + s); };
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * (2 * kStages + 8));
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * (2 * kStages + 8) + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();
+    const bool leader = rank == 0;
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int k_tiles = (p.K + kBK - 1) / kBK;
+    const int tail_mmas = (p.K - (k_tiles - 1) * kBK + kMmaK - 1) / kMmaK;  // MMAs of the last k-tile (1..4)
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            ptx::mbar_init(acc_full_bar(s), 1);
+            ptx::mbar_init(acc_empty_bar(s), 2 * kEpiWarpsFp4);
+            ptx::mbar_init(ovl_free_bar(s), 2 * kEpiWarpsFp4);
+            ptx::mbar_init(sf_ready_bar(s), kSfCopyWarps);
+        }
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tm_a);
+        ptx::prefetch_tmap(&tm_b);
+        ptx::prefetch_tmap(&tm_y);
+        ptx::prefetch_tmap(&tm_sfa);
+        ptx::prefetch_tmap(&tm_sfb);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(ptx::smem_u32(tmem_ptr_smem), kTmemCols);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_ptr_smem;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer: A and B tiles (both CTAs)
+        const bool elected = ptx::elect_one();
+        const uint32_t full0 = ptx::map_to_cta(full_bar(0), 0);  // the even CTA's barriers
+        const bool sf_load = !(kTuning && (p.dbg & kDbgNoSfLoad));
+        const uint32_t tx = 2u * (kStageBytes - (sf_load ? 0 : kSfaBytes + kSfbBytes));
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int t = pair; ok && t < total_tiles; t += num_pairs) {
+            int mt, nt;
+            tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
+            const int m0 = mt * 2 * kBM + static_cast<int>(rank) * kBM;
+            const int nb0 = nt * kBN + static_cast<int>(rank) * (kBN / 2);
+            int kx = 0;
+            for (int kt = 0; kt < k_tiles; ++kt, kx += kRowBytes) {
+                if (!wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x100u | stage)) {
+                    ok = false;
+                    break;
+                }
+                const uint32_t sa = smem_base + stage * kStageBytes;
+                if (elected) {
+                    if (leader) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+                    ptx::tma_load_2d_pair(sa, &tm_a, kx, m0, full0 + 8u * stage);
+                    ptx::tma_load_2d_pair(sa + kABytes, &tm_b, kx, nb0, full0 + 8u * stage);
+                }
+                if (++stage == kStages) {
+                    stage = 0;
+                    phase ^= 1u;
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == kWarps - 1) {
+        // ------------------------------------------------------------ TMA producer: scale-factor tiles (both CTAs)
+        if (!(kTuning && (p.dbg & kDbgNoSfLoad))) {
+            const bool elected = ptx::elect_one();
+            const uint32_t full0 = ptx::map_to_cta(full_bar(0), 0);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int t = pair; ok && t < total_tiles; t += num_pairs) {
+                int mt, nt;
+                tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
+                const int rca = mt * 2 + static_cast<int>(rank);  // 128-row chunk of A owned by this CTA
+                const int rcb = nt * 2;                            // first of the tile's two 128-row chunks of B
+                for (int kt = 0; kt < k_tiles; ++kt) {
+                    if (!wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x800u | stage)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t ssfa = smem_base + stage * kStageBytes + kABytes + kBBytes;
+                    if (elected) {
+                        ptx::tma_load_3d_pair(ssfa, &tm_sfa, 0, kt * 4, rca, full0 + 8u * stage);
+                        ptx::tma_load_3d_pair(ssfa + kSfaBytes, &tm_sfb, 0, kt * 4, rcb, full0 + 8u * stage);
+                    }
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (even CTA)
+        // The loop is warp-uniform so every operand lives in uniform registers; one elected lane issues.
+        if (leader) {
+            const bool elected = ptx::elect_one();
+            const uint32_t idesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kBN >> 3) << 17) |
+                                   (static_cast<uint32_t>((2 * kBM) >> 4) << 24);  // E2M1 x E2M1, UE4M3, M=256
+            const uint64_t desc_hi = ptx::smem_desc_sw128(0);
+            const uint32_t a_lo0 = (smem_base & 0x3FFFFu) >> 4;
+            const uint32_t b_lo0 = ((smem_base + kABytes) & 0x3FFFFu) >> 4;
+            constexpr uint32_t kStageLo = kStageBytes >> 4;
+            const bool no_sf_wait = kTuning && (p.dbg & kDbgNoSfCopy);
+            const bool no_mma = kTuning && (p.dbg & kDbgNoMma);
+            const bool trace = kTuning && (p.dbg & kDbgTrace);
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t gi = 0;
+            bool ok = true;
+            for (int t = pair, it = 0; ok && t < total_tiles; t += num_pairs, ++it) {
+                const int x = it & 1;
+                const uint32_t use = static_cast<uint32_t>(it >> 1);
+                // this accumulator's previous tile is fully drained ...
+                if (!wait_bounded(acc_empty_bar(x), (use & 1u) ^ 1u, abort_flag, p.status, 0x200u | x)) break;
+                // ... and the previous tile (other accumulator) has given back the shared columns
+                if (it > 0 && !wait_bounded(ovl_free_bar(x ^ 1), (static_cast<uint32_t>(it - 1) >> 1) & 1u, abort_flag,
+                                            p.status, 0x900u | x))
+                    break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + x * kAccStride;
+                for (int kt = 0; kt < k_tiles; ++kt) {
+                    const uint32_t sf_buf = gi & 1u;
+                    if (!no_sf_wait) {
+                        // the copy warps waited for this stage's loads, so their barrier covers A and B too
+                        if (!wait_bounded(sf_ready_bar(sf_buf), (gi >> 1) & 1u, abort_flag, p.status, 0x500u | sf_buf)) {
+                            ok = false;
+                            break;
+                        }
+                    } else if (!wait_bounded(full_bar(stage), phase, abort_flag, p.status, 0x300u | stage)) {
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    if (trace) SOL_TRACE(6, gi);
+                    const uint64_t a_desc = desc_hi | (a_lo0 + static_cast<uint32_t>(stage) * kStageLo);
+                    const uint64_t b_desc = desc_hi | (b_lo0 + static_cast<uint32_t>(stage) * kStageLo);
+                    const uint32_t sfa_t = tmem_base + kSfCol + sf_buf * kSfBufCols;
+                    const uint32_t sfb_t = sfa_t + 16;
+                    if (elected && !no_mma) {
+                        if (kt + 1 < k_tiles || tail_mmas == kMmasPerStage) {
+                            ptx::mma_nvfp4_pair(d_tmem, a_desc, b_desc, idesc, sfa_t, sfb_t, kt != 0);
+                            ptx::mma_nvfp4_pair(d_tmem, a_desc + 2, b_desc + 2, idesc, sfa_t + 4, sfb_t + 8, 1);
+                            ptx::mma_nvfp4_pair(d_tmem, a_desc + 4, b_desc + 4, idesc, sfa_t + 8, sfb_t + 16, 1);
+                            ptx::mma_nvfp4_pair(d_tmem, a_desc + 6, b_desc + 6, idesc, sfa_t + 12, sfb_t + 24, 1);
+                        } else {
+                            for (int j = 0; j < tail_mmas; ++j)  // ragged K: fewer than four 32-byte slices are valid
+                                ptx::mma_nvfp4_pair(d_tmem, a_desc + 2u * j, b_desc + 2u * j, idesc, sfa_t + 4 * j,
+                                                    sfb_t + 8 * j, (kt | j) != 0);
+                        }
+                    }
+                    if (elected) ptx::tc_commit_pair_mcast(empty_bar(stage), 3);  // frees the stage in both CTAs
+                    if (trace) SOL_TRACE(3, gi);
+                    ++gi;
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (ok && elected) ptx::tc_commit_pair_mcast(acc_full_bar(x), 3);
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 2 + kEpiWarpsFp4) {
+        // ------------------------------------------------------------ scale-factor copy warps (even CTA)
+        // Copy w of a k-tile (0..11) is part w%3 (scales of A, of B rows 0..127, of B rows 128..255)
+        // of MMA w/3; each has its own warp because tcgen05.cp blocks its issuer for ~100 cycles.
+        if (leader && !(kTuning && (p.dbg & kDbgNoSfCopy))) {
+            const bool elected = ptx::elect_one();
+            const int w = warp - (2 + kEpiWarpsFp4);
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t gi = 0;
+            bool ok = true;
+            for (int t = pair; ok && t < total_tiles; t += num_pairs) {
+                for (int kt = 0; kt < k_tiles; ++kt) {
+                    if (!wait_bounded(full_bar(stage), phase, abort_flag, p.status, 0x600u | stage)) {
+                        ok = false;
+                        break;
+                    }
+                    if (gi >= 2) {
+                        const uint32_t g2 = gi - 2;  // last k-tile whose MMAs read this TMEM buffer
+                        if (!wait_bounded(empty_bar(g2 % kStages), (g2 / kStages) & 1u, abort_flag, p.status,
+                                          0x700u | (g2 % kStages))) {
+                            ok = false;
+                            break;
+                        }
+                    }
+                    ptx::tc_fence_after_sync();
+                    const int nmma = (kt + 1 < k_tiles) ? kMmasPerStage : tail_mmas;
+                    const uint32_t sf_buf = gi & 1u;
+                    if (elected) {
+                        const uint32_t ssf = smem_base + stage * kStageBytes + kABytes + kBBytes;
+                        const uint32_t sf_t = tmem_base + kSfCol + sf_buf * kSfBufCols;
+                        {
+                            const int j = w / 3, part = w % 3;
+                            if (j < nmma) {
+                                // part 0: A chunk j -> columns 4j; part 1/2: B row chunk 0/1, k chunk j -> columns 16 + 8j (+4)
+                                const uint32_t src = part == 0 ? ssf + j * 512 : ssf + kSfaBytes + (part - 1) * 2048 + j * 512;
+                                const uint32_t dst = part == 0 ? sf_t + 4 * j : sf_t + 16 + 8 * j + 4 * (part - 1);
+                                ptx::tc_copy_sf_pair(dst, ptx::smem_desc_sf(src));
+                            }
+                        }
+                        ptx::tc_commit_pair(sf_ready_bar(sf_buf));
+                    }
+                    ++gi;
+                    if (++stage == kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+        const int e = warp - 2;
+        const int quad = warp & 3;   // TMEM lanes [32*quad, 32*quad+32)
+        const int half = e >> 2;     // which of the quadrant's two warps
+        const uint32_t sbuf = epi_base + e * kEpiBufBytes;
+        const float alpha = __fmul_rn(__ldg(p.ts_a), __ldg(p.ts_b));
+        for (int t = pair, it = 0; t < total_tiles; t += num_pairs, ++it) {
+            int mt, nt;
+            tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
+            const int m0 = mt * 2 * kBM + static_cast<int>(rank) * kBM + quad * 32, n0 = nt * kBN;
+            const int x = it & 1;
+            if (!wait_bounded(acc_full_bar(x), (static_cast<uint32_t>(it) >> 1) & 1u, abort_flag, p.status, 0x400u | x)) break;
+            ptx::tc_fence_after_sync();
+            const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + x * kAccStride;
+            const uint32_t ovl_bar = ptx::map_to_cta(ovl_free_bar(x), 0);
+            const uint32_t done_bar = ptx::map_to_cta(acc_empty_bar(x), 0);
+            // 64-column units: accumulator A shares its units 2,3 with the next tile, accumulator B its units 0,1
+            const int first = x == 0 ? 2 + half : half;
+            const int second = x == 0 ? half : 2 + half;
+            if (kTuning && (p.dbg & kDbgNoEpilogue)) {
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) {
+                    ptx::mbar_arrive_cluster(ovl_bar);
+                    ptx::mbar_arrive_cluster(done_bar);
+                }
+                continue;
+            }
+            epilogue_chunk(&tm_y, p, t_acc + first * 64, m0, n0 + first * 64, alpha, sbuf, lane,
+                           [&] { ptx::mbar_arrive_cluster(ovl_bar); });
+            epilogue_chunk(&tm_y, p, t_acc + second * 64, m0, n0 + second * 64, alpha, sbuf, lane,
+                           [&] { ptx::mbar_arrive_cluster(done_bar); });
+        }
+        if (lane == 0) ptx::tma_store_wait_all<0>();
+    }
+
+    // ---------------------------------------------------------------- teardown
+    if (*abort_flag) __nanosleep(2000000);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();  // neither CTA frees TMEM or exits while its partner may still touch it
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace
+
+sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
+                                  const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
+                                  int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev) {
+    const uint64_t chunks_k = static_cast<uint64_t>(ceil_div(K, 64));
+    CUtensorMap tm_a, tm_b, tm_y, tm_sfa, tm_sfb;
+    if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, xq, K / 2, M, K / 2, 128, kBM,
+                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, wq, K / 2, N, K / 2, 128, kBN / 2,
+                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, N, M, ldy * 2, 64, 32,
+                      CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_tmap_sf(&tm_sfa, xsf, chunks_k, static_cast<uint64_t>(ceil_div(M, 128)), 1) ||
+        !make_tmap_sf(&tm_sfb, wsf, chunks_k, static_cast<uint64_t>(ceil_div(N, 128)), 2))
+        return SOL_ERR_CUDA;
+    Params p{};
+    p.sfa = static_cast<const uint8_t *>(xsf);
+    p.sfb = static_cast<const uint8_t *>(wsf);
+    p.ts_a = xts;
+    p.ts_b = wts;
+    p.bias = static_cast<const uint16_t *>(bias);
+    p.status = device_status_word();
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+#ifdef SOL_TUNING
+    if (const char *e = getenv("SOL_DBG")) p.dbg = static_cast<uint32_t>(atoi(e));
+#endif
+    static bool configured[64] = {};
+    if (dev->device < 64 && !configured[dev->device]) {
+        if (cudaFuncSetAttribute(gemm_pair_fp4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
+            cudaSuccess)
+            return SOL_ERR_CUDA;
+        configured[dev->device] = true;
+    }
+    p.m_tiles = static_cast<int>(ceil_div(p.M, 2 * kBM));
+    p.n_tiles = static_cast<int>(ceil_div(p.N, kBN));
+    const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
+    const int max_pairs = dev->sm_count / 2;
+    const int pairs = static_cast<int>(tiles < max_pairs ? tiles : max_pairs);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs), 1, 1);
+    cfg.blockDim = dim3(kThreadsFp4, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, gemm_pair_fp4_kernel, tm_a, tm_b, tm_y, tm_sfa, tm_sfb, p) != cudaSuccess) {
+        cudaGetLastError();
+        return SOL_ERR_CUDA;
+    }
+    return SOL_OK;
+}
+
+}  // namespace gemm
+}  // namespace sol
+
+#ifdef SOL_TUNING
+extern "C" int sol_debug_trace256(long long *host_out) {
+    return cudaMemcpyFromSymbol(host_out, sol::gemm::g_trace, sizeof(sol::gemm::g_trace)) == cudaSuccess ? 0 : 1;
+}
+#endif
