@@ -2,7 +2,7 @@
 //
 // Q(x) = S * Pi_FP4(x / S) with S = E4M3 block scale * FP32 tensor scale T (paper Section 2).
 // Both kernels are streaming codecs bound by HBM bandwidth: 16-byte loads, many loads in
-// flight per thread, packed 4-byte nibble stores, scale bytes staged in shared memory and
+// flight per thread, packed 8-byte nibble stores, scale bytes staged in shared memory and
 // written as whole 512-byte chunks of the layout the tensor core consumes.
 #include "sol_internal.h"
 
@@ -11,16 +11,27 @@ namespace {
 
 constexpr int kQuantThreads = 256;
 constexpr int kTileRows = 128;     // rows per block = one row tile of the chunked scale layout
-constexpr int kTileK = 256;        // elements along K per block = 4 scale chunks = 32 vectors of 8
-constexpr int kRowsPerWarp = kTileRows / (kQuantThreads / 32);  // 16
-constexpr int kBatch = 8;          // independent 16-byte loads in flight per thread
+constexpr int kTileK = 256;        // elements along K per block = 4 scale chunks = 16 scale blocks
+constexpr int kBlocksPerThread = kTileRows * (kTileK / 16) / kQuantThreads;  // 8 scale blocks of 16 elements
+constexpr int kBatch = 4;          // scale blocks (2 x 16-byte loads each) in flight per thread
+
+// max(|a|, |b|) per BF16 half (the sign bits of the result are garbage and masked off later)
+__device__ __forceinline__ uint32_t absmax2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 
 __device__ __forceinline__ uint32_t abs_max_bits(const uint4 &v) {
-    // packed per-halfword max of |bf16| bit patterns (magnitudes order like unsigned integers)
-    uint32_t a = __vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu);
-    uint32_t b = __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu);
-    a = __vmaxu2(a, b);
-    return max(a & 0xFFFFu, a >> 16);
+    // per-halfword max of |bf16| bit patterns (magnitudes order like unsigned integers)
+    const uint32_t m = absmax2(absmax2(v.x, v.y), absmax2(v.z, v.w)) & 0x7FFF7FFFu;
+    return max(m & 0xFFFFu, m >> 16);
+}
+
+__device__ __forceinline__ uint32_t abs_max_bits(const uint4 &u, const uint4 &v) {
+    const uint32_t m = absmax2(absmax2(absmax2(u.x, u.y), absmax2(u.z, u.w)),
+                               absmax2(absmax2(v.x, v.y), absmax2(v.z, v.w))) & 0x7FFF7FFFu;
+    return max(m & 0xFFFFu, m >> 16);
 }
 
 __device__ __forceinline__ uint32_t f32_to_e4m3_sat(float v) {
@@ -53,18 +64,27 @@ __device__ __forceinline__ uint32_t pack_e2m1x8(float y0, float y1, float y2, fl
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-// One block quantizes a 128-row x 256-element tile.  Lane l of a warp owns the 8 elements
-// [8l, 8l+8) of the tile's K range; lanes 2b and 2b+1 share scale block b.
+__device__ __forceinline__ uint32_t quantize8(const uint4 &v, float rcp) {
+    return pack_e2m1x8(__fmul_rn(bf16_lo(v.x), rcp), __fmul_rn(bf16_hi(v.x), rcp), __fmul_rn(bf16_lo(v.y), rcp),
+                       __fmul_rn(bf16_hi(v.y), rcp), __fmul_rn(bf16_lo(v.z), rcp), __fmul_rn(bf16_hi(v.z), rcp),
+                       __fmul_rn(bf16_lo(v.w), rcp), __fmul_rn(bf16_hi(v.w), rcp));
+}
+
+// One block quantizes a 128-row x 256-element tile.  A thread owns whole scale blocks (16
+// elements = two 16-byte loads, one 8-byte store, one scale byte), so the scale arithmetic runs
+// once per 16 elements: the kernel has to stay under ~8 instructions per element to be bound
+// by HBM rather than by instruction issue.  Thread t works on scale block t%16 of rows
+// t/16 + 16*i; a warp reads two 512-byte row segments per step.
 template <bool kSwizzled>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
                 const float *__restrict__ tscale, uint8_t *__restrict__ q, uint8_t *__restrict__ sf) {
     __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kTileK / 16)];  // 2 KB = 4 chunks
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = threadIdx.x & 15;   // scale block inside the tile
+    const int r0 = threadIdx.x >> 4;  // first row inside the tile
     const int64_t row0 = static_cast<int64_t>(blockIdx.y) * kTileRows;
-    const int64_t k0 = static_cast<int64_t>(blockIdx.x) * kTileK;
-    const int64_t k = k0 + lane * 8;
+    const int64_t k = static_cast<int64_t>(blockIdx.x) * kTileK + b * 16;
     const bool k_ok = k < K;
 
     if (kSwizzled) {
@@ -77,40 +97,36 @@ quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t
     const int64_t nb = K >> 4;
 
 #pragma unroll 1
-    for (int batch = 0; batch < kRowsPerWarp / kBatch; ++batch) {
-        uint4 v[kBatch];
+    for (int batch = 0; batch < kBlocksPerThread / kBatch; ++batch) {
+        uint4 lo[kBatch], hi[kBatch];
 #pragma unroll
         for (int i = 0; i < kBatch; ++i) {
-            const int64_t r = row0 + warp * kRowsPerWarp + batch * kBatch + i;
-            v[i] = make_uint4(0, 0, 0, 0);
-            if (k_ok && r < rows) v[i] = __ldcs(reinterpret_cast<const uint4 *>(x + r * ld + k));
+            const int64_t r = row0 + r0 + 16 * (batch * kBatch + i);
+            lo[i] = hi[i] = make_uint4(0, 0, 0, 0);
+            if (k_ok && r < rows) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(x + r * ld + k);
+                lo[i] = __ldcs(src);
+                hi[i] = __ldcs(src + 1);
+            }
         }
 #pragma unroll
         for (int i = 0; i < kBatch; ++i) {
-            const int rl = warp * kRowsPerWarp + batch * kBatch + i;  // row inside the tile
+            const int rl = r0 + 16 * (batch * kBatch + i);  // row inside the tile
             const int64_t r = row0 + rl;
-            uint32_t mb = abs_max_bits(v[i]);
-            mb = max(mb, __shfl_xor_sync(0xFFFFFFFFu, mb, 1));
-            const float a = __uint_as_float(mb << 16);
+            const float a = __uint_as_float(abs_max_bits(lo[i], hi[i]) << 16);
             const float sv = __fdiv_rn(a, c);
             const uint32_t sb = f32_to_e4m3_sat(sv);
             const float d = __fmul_rn(e4m3_to_f32(sb), T);
             const float rcp = sb ? __frcp_rn(d) : 0.0f;
-            const uint32_t packed = pack_e2m1x8(
-                __fmul_rn(bf16_lo(v[i].x), rcp), __fmul_rn(bf16_hi(v[i].x), rcp),
-                __fmul_rn(bf16_lo(v[i].y), rcp), __fmul_rn(bf16_hi(v[i].y), rcp),
-                __fmul_rn(bf16_lo(v[i].z), rcp), __fmul_rn(bf16_hi(v[i].z), rcp),
-                __fmul_rn(bf16_lo(v[i].w), rcp), __fmul_rn(bf16_hi(v[i].w), rcp));
+            uint2 packed;
+            packed.x = quantize8(lo[i], rcp);
+            packed.y = quantize8(hi[i], rcp);
             if (k_ok && r < rows) {
-                __stcs(reinterpret_cast<uint32_t *>(q + r * (K >> 1) + (k >> 1)), packed);
-                if ((lane & 1) == 0) {
-                    const int b = lane >> 1;  // scale block inside the tile, 0..15
-                    if (kSwizzled) {
-                        sf_tile[(b >> 2) * 512 + (rl & 31) * 16 + (rl >> 5) * 4 + (b & 3)] =
-                            static_cast<uint8_t>(sb);
-                    } else {
-                        sf[r * nb + (k >> 4)] = static_cast<uint8_t>(sb);
-                    }
+                __stcs(reinterpret_cast<uint2 *>(q + r * (K >> 1) + (k >> 1)), packed);
+                if (kSwizzled) {
+                    sf_tile[(b >> 2) * 512 + (rl & 31) * 16 + (rl >> 5) * 4 + (b & 3)] = static_cast<uint8_t>(sb);
+                } else {
+                    sf[r * nb + (k >> 4)] = static_cast<uint8_t>(sb);
                 }
             }
         }
@@ -142,10 +158,12 @@ amax_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t vecs_per_row, 
     int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (ld == vecs_per_row * 8) {
         const uint4 *p = reinterpret_cast<const uint4 *>(x);
-        for (; i + 3 * stride < total; i += 4 * stride) {
-            uint4 a = __ldcs(p + i), b = __ldcs(p + i + stride), c = __ldcs(p + i + 2 * stride),
-                  d = __ldcs(p + i + 3 * stride);
-            m = max(m, max(max(abs_max_bits(a), abs_max_bits(b)), max(abs_max_bits(c), abs_max_bits(d))));
+        for (; i + 7 * stride < total; i += 8 * stride) {  // eight independent 16-byte loads in flight
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldcs(p + i + u * stride);
+#pragma unroll
+            for (int u = 0; u < 8; u += 2) m = max(m, abs_max_bits(v[u], v[u + 1]));
         }
         for (; i < total; i += stride) m = max(m, abs_max_bits(__ldcs(p + i)));
     } else {
@@ -177,7 +195,7 @@ sol_status_t launch_amax(const void *x, int64_t rows, int64_t K, int64_t ld, flo
                          cudaStream_t stream, const DeviceInfo *dev) {
     if (cudaMemsetAsync(tscale_out, 0, sizeof(float), stream) != cudaSuccess) return SOL_ERR_CUDA;
     const int64_t vecs = rows * (K / 8);
-    int64_t blocks = ceil_div(vecs, 256 * 4);
+    int64_t blocks = ceil_div(vecs, 256 * 8);
     const int64_t cap = static_cast<int64_t>(dev->sm_count) * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
