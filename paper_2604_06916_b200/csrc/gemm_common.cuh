@@ -53,7 +53,9 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
                                              uint32_t *status, uint32_t code) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    while (!ptx::mbar_try_wait(bar, parity)) {
+    // long hardware suspends: a CTA has ~20 warps that mostly wait, and warps that poll in a tight loop
+    // take issue slots from the few that have work (the epilogue at a tile boundary, above all)
+    while (!ptx::mbar_try_wait_suspend(bar, parity, 200000u)) {
         if (*abort_flag) return false;
         if (clock64() - t0 > kWaitLimitCycles) {
             *abort_flag = 1;

@@ -428,6 +428,7 @@ sol_status_t launch_pair_bf16(const void *x, const void *w, const void *bias, vo
     return launch_pair<Kind::kBf16, kBN, 6>(tm_a, tm_b, tm_y, tm_a, tm_a, p, stream, dev);
 }
 
+#ifdef SOL_TUNING  // the 256 x 192 NVFP4 pair tile is kept for A/B timing only; the product uses gemm_pair_fp4.cu
 sol_status_t launch_pair_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
                                const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
                                int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev) {
@@ -463,6 +464,7 @@ sol_status_t launch_pair_nvfp4(const void *xq, const void *xsf, const float *xts
 #endif
     return launch_pair<Kind::kNvfp4, kBN, 5>(tm_a, tm_b, tm_y, tm_sfa, tm_sfb, p, stream, dev);
 }
+#endif
 
 }  // namespace gemm
 }  // namespace sol

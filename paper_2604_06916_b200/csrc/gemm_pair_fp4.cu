@@ -7,14 +7,17 @@
 // per flop (38 KB per CTA per k-tile = 74 B/clk, against the SM's 128 B/clk ingest port).
 //
 // TMEM does not hold two 256-column accumulators plus the scale factors, so the two accumulators
-// overlap: A = columns [0,256), B = [160,416), scale-factor buffers 2 x 48 columns at [416,512).
-// Tiles alternate between A and B.  The epilogue drains the shared columns [160,256) first and
+// overlap: A = columns [0,256), B = [96,352), scale-factor buffers 3 x 48 columns at [352,496).
+// Tiles alternate between A and B.  The epilogue drains the shared columns [96,256) first and
 // signals `ovl_free`; the MMAs of the next tile start then, while the rest of the tile is still
-// being converted and stored.  Eight epilogue warps (two per TMEM lane quadrant) halve that wait.
+// being converted and stored.  Eight epilogue warps (two per TMEM lane quadrant) shorten that wait.
+// Three scale-factor buffers are needed, not two: tcgen05.cp executes in the tensor pipe in issue
+// order, so a copy for k-tile i that must wait for the MMAs of k-tile i-2 lands behind the MMAs of
+// k-tile i-1 and k-tile i cannot be issued until those have run -- a bubble on every k-tile.
 //
 // Warps per CTA: 0 = TMA producer (A, B); 1 = TMEM owner, MMA issuer in the even CTA;
-// 2..9 = epilogue; 10..21 = scale-factor copy warps (even CTA; tcgen05.cp blocks its warp for
-// ~100 cycles, so each of the twelve copies of a k-tile has its own warp); 22 = TMA producer (scales).
+// 2..9 = epilogue; 10..13 = scale-factor copy warps (even CTA; tcgen05.cp blocks its warp for
+// ~100 cycles, so the copies stay off the MMA thread); 14 = TMA producer (scales).
 // No multicast loads; every mbarrier wait is bounded.
 #include "gemm_common.cuh"
 
@@ -32,55 +35,46 @@ constexpr int kSfaBytes = 2048;                // 4 k-chunks x 512 bytes
 constexpr int kSfbBytes = 4096;                // 2 row chunks x 4 k-chunks x 512 bytes
 constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 38 912
 constexpr int kSfBufCols = 48;                 // per k-tile: 4 MMAs x (4 columns of A + 8 of B)
-constexpr int kAccStride = 160;                // accumulator B starts here; [160,256) is shared
-constexpr int kSfCol = 416;
+constexpr int kAccStride = 96;                 // accumulator B starts here; [96,256) is shared
+constexpr int kSfBufs = 3;
+constexpr int kSfCol = kAccStride + kBN;       // 352
 constexpr int kEpiWarpsFp4 = 8;
-constexpr int kSfCopyWarps = 12;
+constexpr int kSfCopyWarps = 4;                // one per MMA of a k-tile: three tcgen05.cp each
 constexpr int kWarps = 2 + kEpiWarpsFp4 + kSfCopyWarps + 1;
 constexpr int kThreadsFp4 = 32 * kWarps;       // 544
 constexpr int kEpiBytes = kEpiWarpsFp4 * kEpiBufBytes;
-constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 256 + 1024;
-static_assert(kSfCol + 2 * kSfBufCols <= kTmemCols && kAccStride + kBN <= kSfCol, "TMEM budget");
+constexpr int kBiasBytes = kEpiWarpsFp4 * 256;  // per epilogue warp: BF16 bias of its two 64-column chunks
+constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kBiasBytes + 256 + 1024;
+static_assert(kSfCol + kSfBufs * kSfBufCols <= kTmemCols, "TMEM budget");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
-// One 64-column chunk of this warp's 32 accumulator rows: TMEM -> fma(acc, alpha, bias) -> BF16 ->
-// swizzled staging buffer -> TMA store.  `release()` runs as soon as the TMEM loads have completed.
-template <class Release>
-__device__ __forceinline__ void epilogue_chunk(const CUtensorMap *tm_y, const Params &p, uint32_t t_chunk, int m0,
-                                               int nc, float alpha, uint32_t sbuf, int lane, Release release) {
+// Converts one 64-column chunk held in registers: fma(acc, alpha, bias) -> BF16 -> swizzled staging
+// buffer -> TMA store (32 rows x 64 columns, clipped at the matrix edge).
+__device__ __forceinline__ void epilogue_store(const CUtensorMap *tm_y, const Params &p, const uint32_t (&lo)[32],
+                                               const uint32_t (&hi)[32], int m0, int nc, float alpha, uint32_t sbuf,
+                                               uint32_t sbias, int lane) {
     if (lane == 0) ptx::tma_store_wait_read<0>();  // the previous store of this warp has left the staging buffer
     __syncwarp();
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        uint32_t acc[32];
-        ptx::tmem_ld_32x32(t_chunk + h * 32, acc);
-        ptx::tmem_ld_wait();
-        if (h == 1) {  // both halves of the chunk have left TMEM
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) release();
-        }
-        const int nb = nc + h * 32;
+    for (int g = 0; g < 8; ++g) {
+        uint32_t bw[4];  // 8 bias values of columns nc + 8g .. (same address in every lane: a broadcast read)
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(bw[0]), "=r"(bw[1]), "=r"(bw[2]), "=r"(bw[3])
+                     : "r"(sbias + g * 16));
+        uint32_t o[4];
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            uint4 bb = make_uint4(0, 0, 0, 0);
-            if (p.bias != nullptr && nb + g * 8 < p.N) bb = __ldg(reinterpret_cast<const uint4 *>(p.bias + nb + g * 8));
-            const uint32_t bw[4] = {bb.x, bb.y, bb.z, bb.w};
-            uint32_t o[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float y0 = fmaf(__uint_as_float(acc[g * 8 + 2 * e]), alpha, __uint_as_float(bw[e] << 16));
-                const float y1 =
-                    fmaf(__uint_as_float(acc[g * 8 + 2 * e + 1]), alpha, __uint_as_float(bw[e] & 0xFFFF0000u));
-                __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
-                o[e] = *reinterpret_cast<uint32_t *>(&pk);
-            }
-            const uint32_t chunk16 = static_cast<uint32_t>(h * 4 + g) ^ (lane & 7u);  // 128-byte swizzle
-            const uint32_t dst = sbuf + lane * 128 + chunk16 * 16;
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]),
-                         "r"(o[3])
-                         : "memory");
+        for (int e = 0; e < 4; ++e) {
+            const uint32_t a0 = g < 4 ? lo[g * 8 + 2 * e] : hi[(g - 4) * 8 + 2 * e];
+            const uint32_t a1 = g < 4 ? lo[g * 8 + 2 * e + 1] : hi[(g - 4) * 8 + 2 * e + 1];
+            const float y0 = fmaf(__uint_as_float(a0), alpha, __uint_as_float(bw[e] << 16));
+            const float y1 = fmaf(__uint_as_float(a1), alpha, __uint_as_float(bw[e] & 0xFFFF0000u));
+            __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
+            o[e] = *reinterpret_cast<uint32_t *>(&pk);
         }
+        const uint32_t chunk16 = static_cast<uint32_t>(g) ^ (lane & 7u);  // 128-byte swizzle
+        const uint32_t dst = sbuf + lane * 128 + chunk16 * 16;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3])
+                     : "memory");
     }
     ptx::fence_proxy_async_smem();
     __syncwarp();
@@ -99,16 +93,18 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
 
     const uint32_t epi_base = smem_base + kStages * kStageBytes;
-    const uint32_t bar_base = epi_base + kEpiBytes;
-    uint8_t *bar_gen = smem_gen + kStages * kStageBytes + kEpiBytes;
+    const uint32_t bias_base = epi_base + kEpiBytes;
+    const uint32_t bar_base = bias_base + kBiasBytes;
+    uint8_t *bar_gen = smem_gen + kStages * kStageBytes + kEpiBytes + kBiasBytes;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
     auto acc_full_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
     auto acc_empty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 2 + s); };
     auto ovl_free_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 4 + s); };
     auto sf_ready_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 6 + s); };
-    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * (2 * kStages + 8));
-    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * (2 * kStages + 8) + 4);
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * (2 * kStages + 6 + kSfBufs));
+    volatile uint32_t *abort_flag =
+        reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * (2 * kStages + 6 + kSfBufs) + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();
@@ -127,8 +123,8 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             ptx::mbar_init(acc_full_bar(s), 1);
             ptx::mbar_init(acc_empty_bar(s), 2 * kEpiWarpsFp4);
             ptx::mbar_init(ovl_free_bar(s), 2 * kEpiWarpsFp4);
-            ptx::mbar_init(sf_ready_bar(s), kSfCopyWarps);
         }
+        for (int s = 0; s < kSfBufs; ++s) ptx::mbar_init(sf_ready_bar(s), kSfCopyWarps);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tm_a);
@@ -228,6 +224,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             int stage = 0;
             uint32_t phase = 0;
             uint32_t gi = 0;
+            uint32_t sf_buf = 0, sf_phase = 0;  // scale-factor buffer ring
             bool ok = true;
             for (int t = pair, it = 0; ok && t < total_tiles; t += num_pairs, ++it) {
                 const int x = it & 1;
@@ -239,12 +236,12 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                                             p.status, 0x900u | x))
                     break;
                 ptx::tc_fence_after_sync();
+                if (trace) SOL_TRACE(8, it);
                 const uint32_t d_tmem = tmem_base + x * kAccStride;
                 for (int kt = 0; kt < k_tiles; ++kt) {
-                    const uint32_t sf_buf = gi & 1u;
                     if (!no_sf_wait) {
                         // the copy warps waited for this stage's loads, so their barrier covers A and B too
-                        if (!wait_bounded(sf_ready_bar(sf_buf), (gi >> 1) & 1u, abort_flag, p.status, 0x500u | sf_buf)) {
+                        if (!wait_bounded(sf_ready_bar(sf_buf), sf_phase, abort_flag, p.status, 0x500u | sf_buf)) {
                             ok = false;
                             break;
                         }
@@ -273,25 +270,33 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     if (elected) ptx::tc_commit_pair_mcast(empty_bar(stage), 3);  // frees the stage in both CTAs
                     if (trace) SOL_TRACE(3, gi);
                     ++gi;
+                    if (++sf_buf == kSfBufs) {
+                        sf_buf = 0;
+                        sf_phase ^= 1u;
+                    }
                     if (++stage == kStages) {
                         stage = 0;
                         phase ^= 1u;
                     }
                 }
                 if (ok && elected) ptx::tc_commit_pair_mcast(acc_full_bar(x), 3);
+                if (trace) SOL_TRACE(7, it);
             }
         }
         __syncwarp();
     } else if (warp >= 2 + kEpiWarpsFp4) {
         // ------------------------------------------------------------ scale-factor copy warps (even CTA)
-        // Copy w of a k-tile (0..11) is part w%3 (scales of A, of B rows 0..127, of B rows 128..255)
-        // of MMA w/3; each has its own warp because tcgen05.cp blocks its issuer for ~100 cycles.
+        // tcgen05.cp blocks its issuing warp for ~100 cycles, so the twelve copies of a k-tile are
+        // spread over four warps and kept off the MMA thread; the third TMEM buffer hides their latency.
         if (leader && !(kTuning && (p.dbg & kDbgNoSfCopy))) {
             const bool elected = ptx::elect_one();
             const int w = warp - (2 + kEpiWarpsFp4);
             int stage = 0;
             uint32_t phase = 0;
             uint32_t gi = 0;
+            uint32_t sf_buf = 0;
+            int old_stage = kStages - kSfBufs;  // smem stage of k-tile gi - kSfBufs, the last reader of this buffer
+            uint32_t old_phase = 1;             // parity its `empty` barrier shows once those MMAs are done
             bool ok = true;
             for (int t = pair; ok && t < total_tiles; t += num_pairs) {
                 for (int kt = 0; kt < k_tiles; ++kt) {
@@ -299,32 +304,31 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                         ok = false;
                         break;
                     }
-                    if (gi >= 2) {
-                        const uint32_t g2 = gi - 2;  // last k-tile whose MMAs read this TMEM buffer
-                        if (!wait_bounded(empty_bar(g2 % kStages), (g2 / kStages) & 1u, abort_flag, p.status,
-                                          0x700u | (g2 % kStages))) {
-                            ok = false;
-                            break;
-                        }
+                    if (gi >= kSfBufs &&
+                        !wait_bounded(empty_bar(old_stage), old_phase, abort_flag, p.status, 0x700u | old_stage)) {
+                        ok = false;
+                        break;
                     }
                     ptx::tc_fence_after_sync();
+                    if (kTuning && (p.dbg & kDbgTrace) && w == 0) SOL_TRACE(4, gi);
                     const int nmma = (kt + 1 < k_tiles) ? kMmasPerStage : tail_mmas;
-                    const uint32_t sf_buf = gi & 1u;
                     if (elected) {
                         const uint32_t ssf = smem_base + stage * kStageBytes + kABytes + kBBytes;
                         const uint32_t sf_t = tmem_base + kSfCol + sf_buf * kSfBufCols;
-                        {
-                            const int j = w / 3, part = w % 3;
-                            if (j < nmma) {
-                                // part 0: A chunk j -> columns 4j; part 1/2: B row chunk 0/1, k chunk j -> columns 16 + 8j (+4)
-                                const uint32_t src = part == 0 ? ssf + j * 512 : ssf + kSfaBytes + (part - 1) * 2048 + j * 512;
-                                const uint32_t dst = part == 0 ? sf_t + 4 * j : sf_t + 16 + 8 * j + 4 * (part - 1);
-                                ptx::tc_copy_sf_pair(dst, ptx::smem_desc_sf(src));
-                            }
+                        if (w < nmma) {  // warp w: the scales of MMA w -- A chunk, then the two B row chunks
+                            ptx::tc_copy_sf_pair(sf_t + 4 * w, ptx::smem_desc_sf(ssf + w * 512));
+                            ptx::tc_copy_sf_pair(sf_t + 16 + 8 * w, ptx::smem_desc_sf(ssf + kSfaBytes + w * 512));
+                            ptx::tc_copy_sf_pair(sf_t + 20 + 8 * w, ptx::smem_desc_sf(ssf + kSfaBytes + 2048 + w * 512));
                         }
                         ptx::tc_commit_pair(sf_ready_bar(sf_buf));
                     }
+                    if (kTuning && (p.dbg & kDbgTrace) && w == 0) SOL_TRACE(5, gi);
                     ++gi;
+                    if (++sf_buf == kSfBufs) sf_buf = 0;
+                    if (++old_stage == kStages) {
+                        old_stage = 0;
+                        old_phase ^= 1u;
+                    }
                     if (++stage == kStages) {
                         stage = 0;
                         phase ^= 1u;
@@ -339,20 +343,33 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         const int quad = warp & 3;   // TMEM lanes [32*quad, 32*quad+32)
         const int half = e >> 2;     // which of the quadrant's two warps
         const uint32_t sbuf = epi_base + e * kEpiBufBytes;
+        const uint32_t sbias = bias_base + e * 256;
         const float alpha = __fmul_rn(__ldg(p.ts_a), __ldg(p.ts_b));
         for (int t = pair, it = 0; t < total_tiles; t += num_pairs, ++it) {
             int mt, nt;
             tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
             const int m0 = mt * 2 * kBM + static_cast<int>(rank) * kBM + quad * 32, n0 = nt * kBN;
             const int x = it & 1;
+            // 64-column units of the accumulator.  A (base 0) shares its columns [96,256) with the next
+            // tile: units 2, 3 and the upper half of unit 1; B (base 96) its columns [0,160): units 0, 1 and
+            // the lower half of unit 2.  Each warp takes one fully shared unit first and one other unit.
+            const int first = x == 0 ? 2 + half : half;
+            const int second = x == 0 ? half : 2 + half;
+            {   // stage this warp's 2 x 64 bias values in shared memory while the main loop is still running
+                const int unit = lane < 16 ? first : second;
+                const int col = n0 + unit * 64 + (lane & 15) * 4;
+                uint2 bv = make_uint2(0, 0);
+                if (p.bias != nullptr && col < p.N) bv = __ldg(reinterpret_cast<const uint2 *>(p.bias + col));
+                __syncwarp();  // the previous tile's reads of the staging area are done
+                asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sbias + lane * 8), "r"(bv.x), "r"(bv.y) : "memory");
+                __syncwarp();
+            }
             if (!wait_bounded(acc_full_bar(x), (static_cast<uint32_t>(it) >> 1) & 1u, abort_flag, p.status, 0x400u | x)) break;
             ptx::tc_fence_after_sync();
+            if (kTuning && (p.dbg & kDbgTrace) && warp == 2) SOL_TRACE(9, it);
             const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + x * kAccStride;
             const uint32_t ovl_bar = ptx::map_to_cta(ovl_free_bar(x), 0);
             const uint32_t done_bar = ptx::map_to_cta(acc_empty_bar(x), 0);
-            // 64-column units: accumulator A shares its units 2,3 with the next tile, accumulator B its units 0,1
-            const int first = x == 0 ? 2 + half : half;
-            const int second = x == 0 ? half : 2 + half;
             if (kTuning && (p.dbg & kDbgNoEpilogue)) {
                 ptx::tc_fence_before_sync();
                 __syncwarp();
@@ -362,10 +379,32 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 }
                 continue;
             }
-            epilogue_chunk(&tm_y, p, t_acc + first * 64, m0, n0 + first * 64, alpha, sbuf, lane,
-                           [&] { ptx::mbar_arrive_cluster(ovl_bar); });
-            epilogue_chunk(&tm_y, p, t_acc + second * 64, m0, n0 + second * 64, alpha, sbuf, lane,
-                           [&] { ptx::mbar_arrive_cluster(done_bar); });
+            // The shared columns leave TMEM first and go straight back to the MMA warp; the arithmetic
+            // runs from registers afterwards.  A warp whose second unit is partly shared also fetches
+            // that half before it releases.
+            const bool early = half == x;                 // second unit holds no shared columns
+            const uint32_t t1 = t_acc + first * 64, t2 = t_acc + second * 64;
+            const uint32_t shared_half = x == 0 ? 32u : 0u;  // A: upper half of unit 1, B: lower half of unit 2
+            uint32_t a_lo[32], a_hi[32], b_sh[32], b_ot[32];
+            ptx::tmem_ld_32x32(t1, a_lo);
+            ptx::tmem_ld_32x32(t1 + 32, a_hi);
+            if (!early) ptx::tmem_ld_32x32(t2 + shared_half, b_sh);
+            ptx::tmem_ld_wait();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(ovl_bar);
+            if (kTuning && (p.dbg & kDbgTrace) && warp == 2) SOL_TRACE(10, it);
+            epilogue_store(&tm_y, p, a_lo, a_hi, m0, n0 + first * 64, alpha, sbuf, sbias, lane);
+            if (early) ptx::tmem_ld_32x32(t2 + shared_half, b_sh);
+            ptx::tmem_ld_32x32(t2 + (shared_half ^ 32u), b_ot);
+            ptx::tmem_ld_wait();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(done_bar);
+            if (x == 0)  // b_sh is the upper half
+                epilogue_store(&tm_y, p, b_ot, b_sh, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
+            else
+                epilogue_store(&tm_y, p, b_sh, b_ot, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();
     }
