@@ -30,7 +30,10 @@ NOMINAL_BF16_TFLOPS = 2250.0    # vendor dense BF16 peak
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (None until a capture of the current kernel exists)
-NCU_TRAFFIC = {"gemm": None, "quantize": None}
+# ncu (profiles/gemm_pair_and_quantizer_flux_d_proj.md), d_proj launch: GEMM 69.1 MB read + 172.7 MB
+# written for 295.5 MB algorithmic (Y partly still dirty in L2 at kernel end); quantizer 226.5 + 26.5 MB
+# for 290.2 MB algorithmic.  Scaled to all six layers by the algorithmic bytes (traffic is proportional).
+NCU_TRAFFIC_RATIO = {"gemm": (69.09 + 172.67) / 295.5, "quantize": (226.53 + 26.51) / 290.2}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -280,6 +283,8 @@ def run_ours(args):
     gemm_tflops = flops / (tot["gemm"] * 1e-3) / 1e12
     fp4_peak = peaks["bf16_tflops_sustained"] * (NOMINAL_FP4_TFLOPS / NOMINAL_BF16_TFLOPS)
     quant_bytes = sum(l.M * l.K * 2 + l.M * l.K // 2 + B.scale_bytes(l.M, l.K) for l in layers)
+    gemm_bytes = sum(l.M * l.K // 2 + B.scale_bytes(l.M, l.K) + l.N * l.K // 2 + B.scale_bytes(l.N, l.K) + 2 * l.N +
+                     2 * l.M * l.N for l in layers)
 
     # ---- end to end: pinned HOST activations in, HOST outputs back, copies inside the timed region,
     # through the host-buffer entry point of the C ABI, all six layers per step
@@ -332,12 +337,14 @@ def run_ours(args):
         "gemm_only_tflops": gemm_tflops, "gemm_pct_of_nominal_fp4_peak": 100.0 * gemm_tflops / NOMINAL_FP4_TFLOPS,
         "quantizer_gbs": quant_bytes / (tot["quant"] * 1e-3) / 1e9,
         "quantizer_pct_of_8tbs": 100.0 * quant_bytes / (tot["quant"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-        "roofline": {"bound": "tensor", "kernel": "gemm_pair_kernel<nvfp4>", "achieved": gemm_tflops, "peak": fp4_peak,
-                     "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak, "traffic": NCU_TRAFFIC.get("gemm"),
+        "roofline": {"bound": "tensor", "kernel": "gemm_pair_fp4_kernel", "achieved": gemm_tflops, "peak": fp4_peak,
+                     "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak, "traffic": int(NCU_TRAFFIC_RATIO["gemm"] * gemm_bytes),
+                     "traffic_unit": "bytes per step (six launches), d_proj ncu capture scaled by algorithmic bytes",
                      "peak_source": f"{peak_src} sustained bf16 {peaks['bf16_tflops_sustained']} TF x 4 (nominal fp4:bf16)"},
         "roofline_quantizer": {"bound": "hbm", "kernel": "quantize_kernel", "achieved": quant_bytes / (tot["quant"] * 1e-3) / 1e9,
                                "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                               "frac": quant_bytes / (tot["quant"] * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get("quantize"),
+                               "frac": quant_bytes / (tot["quant"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                               "traffic": int(NCU_TRAFFIC_RATIO["quantize"] * quant_bytes),
                                "peak_source": peak_src},
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": kernels_per_layer * len(layers) * args.steps,
