@@ -225,6 +225,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             uint32_t phase = 0;
             uint32_t gi = 0;
             uint32_t sf_buf = 0, sf_phase = 0;  // scale-factor buffer ring
+            bool sf_seen = false;
             bool ok = true;
             for (int t = pair, it = 0; ok && t < total_tiles; t += num_pairs, ++it) {
                 const int x = it & 1;
@@ -240,8 +241,10 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 const uint32_t d_tmem = tmem_base + x * kAccStride;
                 for (int kt = 0; kt < k_tiles; ++kt) {
                     if (!no_sf_wait) {
-                        // the copy warps waited for this stage's loads, so their barrier covers A and B too
-                        if (!wait_bounded(sf_ready_bar(sf_buf), sf_phase, abort_flag, p.status, 0x500u | sf_buf)) {
+                        // the copy warps waited for this stage's loads, so their barrier covers A and B too;
+                        // `sf_seen`: the previous k-tile already saw this barrier complete (peek below)
+                        if (!sf_seen &&
+                            !wait_bounded(sf_ready_bar(sf_buf), sf_phase, abort_flag, p.status, 0x500u | sf_buf)) {
                             ok = false;
                             break;
                         }
@@ -267,13 +270,17 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                                                     sfb_t + 8 * j, (kt | j) != 0);
                         }
                     }
-                    if (elected) ptx::tc_commit_pair_mcast(empty_bar(stage), 3);  // frees the stage in both CTAs
+                    // next k-tile's scale-factor buffer (it may belong to the next tile)
+                    const uint32_t nb = sf_buf + 1 == kSfBufs ? 0u : sf_buf + 1;
+                    const uint32_t np = sf_buf + 1 == kSfBufs ? sf_phase ^ 1u : sf_phase;
+                    // commit frees the stage in both CTAs; the peek tells whether the next buffer is ready
+                    bool seen = false;
+                    if (elected) seen = ptx::tc_commit_pair_mcast_and_peek(empty_bar(stage), 3, sf_ready_bar(nb), np);
+                    sf_seen = __any_sync(0xFFFFFFFFu, seen) != 0;  // keeps the loop warp-uniform
                     if (trace) SOL_TRACE(3, gi);
                     ++gi;
-                    if (++sf_buf == kSfBufs) {
-                        sf_buf = 0;
-                        sf_phase ^= 1u;
-                    }
+                    sf_buf = nb;
+                    sf_phase = np;
                     if (++stage == kStages) {
                         stage = 0;
                         phase ^= 1u;

@@ -281,6 +281,21 @@ __device__ __forceinline__ void tc_commit_pair_mcast(uint32_t bar, uint16_t mask
                  ::"r"(bar), "h"(mask)
                  : "memory");
 }
+// Multicast commit, with a non-blocking test of another barrier started before it: the test's
+// result is only read after the commit has been issued, so its latency hides behind the commit.
+__device__ __forceinline__ bool tc_commit_pair_mcast_and_peek(uint32_t bar, uint16_t mask, uint32_t peek_bar,
+                                                              uint32_t peek_parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%3], %4;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "h"(mask), "r"(peek_bar), "r"(peek_parity)
+        : "memory");
+    return done != 0;
+}
 __device__ __forceinline__ void tc_copy_sf_pair(uint32_t taddr, uint64_t s_desc) {
     asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(s_desc) : "memory");
 }
