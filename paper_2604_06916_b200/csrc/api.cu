@@ -251,9 +251,7 @@ sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *
     uint8_t *xq = ws;
     uint8_t *xsf = xq + align256(sol_nvfp4_data_bytes(M, K));
     float *xts = reinterpret_cast<float *>(xsf + align256(sol_nvfp4_scale_bytes(M, K, SOL_SF_SWIZZLED_128x4)));
-    st = launch_amax(x_bf16, M, K, ldx, xts, s, dev);
-    if (st != SOL_OK) return st;
-    st = launch_quantize(x_bf16, M, K, ldx, xts, xq, xsf, SOL_SF_SWIZZLED_128x4, s);
+    st = launch_amax_quantize(x_bf16, M, K, ldx, xts, xq, xsf, SOL_SF_SWIZZLED_128x4, s, dev);
     if (st != SOL_OK) return st;
     return launch_gemm_nvfp4(xq, xsf, xts, wq, wsf, w_tscale, bias_bf16, y_bf16, M, N, K, ldy, s, dev);
 }

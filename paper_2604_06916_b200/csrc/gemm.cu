@@ -268,7 +268,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CU
         // ------------------------------------------------------------ epilogue (warps 2..5)
         const int quad = warp & 3;  // TMEM lanes [32*quad, 32*quad+32) are this warp's
         const uint32_t epi_warp = epi_base + (warp - 2) * 2 * kEpiBufBytes;
-        const float alpha = C::kFp4 ? __fmul_rn(__ldg(p.ts_a), __ldg(p.ts_b)) : 1.0f;
+        const float alpha = C::kFp4 ? __fmul_rn(__ldcg(p.ts_a), __ldcg(p.ts_b)) : 1.0f;
         int it = 0;
         uint32_t buf = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++it) {

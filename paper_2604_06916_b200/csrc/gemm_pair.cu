@@ -102,6 +102,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     ptx::cluster_sync();  // both CTAs' barriers and TMEM exist before anything crosses the pair
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_smem;
+    ptx::grid_dependency_wait();  // set-up above overlaps the previous kernel; its results are read below
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer: A and B tiles (both CTAs)
@@ -330,7 +331,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
         const int quad = warp & 3;
         const uint32_t epi_warp = epi_base + (warp - 2) * 2 * kEpiBufBytes;
-        const float alpha = C::kFp4 ? __fmul_rn(__ldg(p.ts_a), __ldg(p.ts_b)) : 1.0f;
+        const float alpha = C::kFp4 ? __fmul_rn(__ldcg(p.ts_a), __ldcg(p.ts_b)) : 1.0f;
         int it = 0;
         uint32_t buf = 0;
         for (int t = pair; t < total_tiles; t += num_pairs, ++it) {
@@ -391,13 +392,15 @@ sol_status_t launch_pair(const CUtensorMap &tm_a, const CUtensorMap &tm_b, const
     cfg.blockDim = dim3(C::kThreads, 1, 1);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_y, tm_sfa, tm_sfb, p) != cudaSuccess) {
         cudaGetLastError();
         return SOL_ERR_CUDA;

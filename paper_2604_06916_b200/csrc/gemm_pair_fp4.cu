@@ -142,6 +142,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     ptx::cluster_sync();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_smem;
+    ptx::grid_dependency_wait();  // set-up above overlaps the previous kernel; its results are read below
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer: A and B tiles (both CTAs)
@@ -351,7 +352,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         const int half = e >> 2;     // which of the quadrant's two warps
         const uint32_t sbuf = epi_base + e * kEpiBufBytes;
         const uint32_t sbias = bias_base + e * 256;
-        const float alpha = __fmul_rn(__ldg(p.ts_a), __ldg(p.ts_b));
+        const float alpha = __fmul_rn(__ldcg(p.ts_a), __ldcg(p.ts_b));
         for (int t = pair, it = 0; t < total_tiles; t += num_pairs, ++it) {
             int mt, nt;
             tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
@@ -473,13 +474,15 @@ sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *
     cfg.blockDim = dim3(kThreadsFp4, 1, 1);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, gemm_pair_fp4_kernel, tm_a, tm_b, tm_y, tm_sfa, tm_sfb, p) != cudaSuccess) {
         cudaGetLastError();
         return SOL_ERR_CUDA;

@@ -61,6 +61,16 @@ __device__ __forceinline__ uint32_t pack_e2m1x8(float y0, float y1, float y2, fl
     return out;
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
+// start while its predecessor in the stream is still draining; it must not touch global memory
+// before grid_dependency_wait() returns (a no-op when there is nothing to wait for).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+__device__ __forceinline__ float tensor_scale_from_amax(float a) {
+    return (a == 0.0f) ? 1.0f : __fdiv_rn(a, 2688.0f);
+}
+
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
@@ -75,10 +85,13 @@ __device__ __forceinline__ uint32_t quantize8(const uint4 &v, float rcp) {
 // once per 16 elements: the kernel has to stay under ~8 instructions per element to be bound
 // by HBM rather than by instruction issue.  Thread t works on scale block t%16 of rows
 // t/16 + 16*i; a warp reads two 512-byte row segments per step.
+// With `amax` set the tensor scale is derived here from the amax word the reduction left (the
+// bit pattern of max|x| as FP32) and block (0,0) publishes it in `tscale_out` for the GEMM.
 template <bool kSwizzled>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
-                const float *__restrict__ tscale, uint8_t *__restrict__ q, uint8_t *__restrict__ sf) {
+                const float *tscale, const float *amax, float *tscale_out, uint8_t *__restrict__ q,
+                uint8_t *__restrict__ sf) {
     __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kTileK / 16)];  // 2 KB = 4 chunks
 
     const int b = threadIdx.x & 15;   // scale block inside the tile
@@ -92,7 +105,10 @@ quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t
         __syncthreads();
     }
 
-    const float T = __ldg(tscale);
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const float T = amax != nullptr ? tensor_scale_from_amax(*amax) : *tscale;
+    if (tscale_out != nullptr && threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0) *tscale_out = T;
     const float c = __fmul_rn(6.0f, T);
     const int64_t nb = K >> 4;
 
@@ -152,6 +168,7 @@ quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t
 __global__ void __launch_bounds__(256)
 amax_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t vecs_per_row, int64_t ld,
             uint32_t *__restrict__ out_bits) {
+    grid_launch_dependents();
     uint32_t m = 0;
     const int64_t total = rows * vecs_per_row;
     const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
@@ -185,39 +202,72 @@ amax_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t vecs_per_row, 
 
 // In place: amax bits -> T = amax / (6 * 448), or 1 for an all-zero tensor.
 __global__ void tensor_scale_kernel(float *t) {
-    const float a = *t;
-    *t = (a == 0.0f) ? 1.0f : __fdiv_rn(a, 2688.0f);
+    *t = tensor_scale_from_amax(*t);
 }
 
 }  // namespace
 
-sol_status_t launch_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *tscale_out,
-                         cudaStream_t stream, const DeviceInfo *dev) {
-    if (cudaMemsetAsync(tscale_out, 0, sizeof(float), stream) != cudaSuccess) return SOL_ERR_CUDA;
+namespace {
+
+sol_status_t launch_amax_bits(const void *x, int64_t rows, int64_t K, int64_t ld, uint32_t *bits_out,
+                              cudaStream_t stream, const DeviceInfo *dev) {
+    if (cudaMemsetAsync(bits_out, 0, sizeof(uint32_t), stream) != cudaSuccess) return SOL_ERR_CUDA;
     const int64_t vecs = rows * (K / 8);
     int64_t blocks = ceil_div(vecs, 256 * 8);
     const int64_t cap = static_cast<int64_t>(dev->sm_count) * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     amax_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
-        static_cast<const uint16_t *>(x), rows, K / 8, ld, reinterpret_cast<uint32_t *>(tscale_out));
+        static_cast<const uint16_t *>(x), rows, K / 8, ld, bits_out);
+    return launch_status();
+}
+
+// The quantizer is launched as a programmatic dependent of whatever kernel precedes it in the
+// stream: its blocks may become resident while that kernel drains, and wait in hardware before
+// their first global access.
+sol_status_t launch_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale,
+                                const float *amax, float *tscale_out, void *q, void *sf,
+                                sol_sf_layout_t layout, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ceil_div(K, kTileK)), static_cast<unsigned>(ceil_div(rows, kTileRows)));
+    cfg.blockDim = dim3(kQuantThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    auto kern = layout == SOL_SF_SWIZZLED_128x4 ? quantize_kernel<true> : quantize_kernel<false>;
+    if (cudaLaunchKernelEx(&cfg, kern, static_cast<const uint16_t *>(x), rows, K, ld, tscale, amax, tscale_out,
+                           static_cast<uint8_t *>(q), static_cast<uint8_t *>(sf)) != cudaSuccess) {
+        cudaGetLastError();
+        return SOL_ERR_CUDA;
+    }
+    return launch_status();
+}
+
+}  // namespace
+
+sol_status_t launch_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *tscale_out,
+                         cudaStream_t stream, const DeviceInfo *dev) {
+    sol_status_t st = launch_amax_bits(x, rows, K, ld, reinterpret_cast<uint32_t *>(tscale_out), stream, dev);
+    if (st != SOL_OK) return st;
     tensor_scale_kernel<<<1, 1, 0, stream>>>(tscale_out);
     return launch_status();
 }
 
 sol_status_t launch_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale,
                              void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream) {
-    dim3 grid(static_cast<unsigned>(ceil_div(K, kTileK)), static_cast<unsigned>(ceil_div(rows, kTileRows)));
-    if (layout == SOL_SF_SWIZZLED_128x4) {
-        quantize_kernel<true><<<grid, kQuantThreads, 0, stream>>>(
-            static_cast<const uint16_t *>(x), rows, K, ld, tscale, static_cast<uint8_t *>(q),
-            static_cast<uint8_t *>(sf));
-    } else {
-        quantize_kernel<false><<<grid, kQuantThreads, 0, stream>>>(
-            static_cast<const uint16_t *>(x), rows, K, ld, tscale, static_cast<uint8_t *>(q),
-            static_cast<uint8_t *>(sf));
-    }
-    return launch_status();
+    return launch_quantize_ex(x, rows, K, ld, tscale, nullptr, nullptr, q, sf, layout, stream);
+}
+
+sol_status_t launch_amax_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,
+                                  void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream,
+                                  const DeviceInfo *dev) {
+    sol_status_t st = launch_amax_bits(x, rows, K, ld, reinterpret_cast<uint32_t *>(scale_words + 1), stream, dev);
+    if (st != SOL_OK) return st;
+    return launch_quantize_ex(x, rows, K, ld, nullptr, scale_words + 1, scale_words, q, sf, layout, stream);
 }
 
 }  // namespace sol

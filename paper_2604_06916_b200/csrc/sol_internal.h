@@ -37,6 +37,11 @@ sol_status_t launch_amax(const void *x, int64_t rows, int64_t K, int64_t ld, flo
                          cudaStream_t stream, const DeviceInfo *dev);
 sol_status_t launch_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale,
                              void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream);
+// Per-tensor scale and quantizer in two kernels: scale_words[1] receives max|x| (as FP32 bits),
+// the quantizer derives T from it and publishes T in scale_words[0].
+sol_status_t launch_amax_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,
+                                  void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream,
+                                  const DeviceInfo *dev);
 sol_status_t launch_gemm_bf16(const void *x, const void *w, const void *bias, void *y, int64_t M,
                               int64_t N, int64_t K, int64_t ldx, int64_t ldw, int64_t ldy,
                               cudaStream_t stream, const DeviceInfo *dev);

@@ -74,9 +74,7 @@ sol_status_t nvfp4_quantize_linear_static(const void *x_bf16, int64_t ldx, const
     // The array keeps whatever the previous call left in it.  Nothing below relies on old contents:
     // the amax step zeroes the scale word it accumulates into, and the quantizer writes every byte of
     // the data and scale regions it hands to the GEMM, padding included.
-    st = launch_amax(x_bf16, M, K, ldx, xts, s, dev);
-    if (st != SOL_OK) return st;
-    st = launch_quantize(x_bf16, M, K, ldx, xts, xq, xsf, SOL_SF_SWIZZLED_128x4, s);
+    st = launch_amax_quantize(x_bf16, M, K, ldx, xts, xq, xsf, SOL_SF_SWIZZLED_128x4, s, dev);
     if (st != SOL_OK) return st;
     return launch_gemm_nvfp4(xq, xsf, xts, wq, wsf, w_tscale, bias_bf16, y_bf16, M, N, K, ldy, s, dev);
 }
