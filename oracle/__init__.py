@@ -61,6 +61,8 @@ def _load():
     L.oracle_bf16_linear.argtypes = [u16p, i64, u16p, i64, u16p, i64, i64, i64p, i64, f64p]
     L.oracle_f64_to_bf16_array.restype, L.oracle_f64_to_bf16_array.argtypes = None, [f64p, i64, u16p]
     L.oracle_num_threads.restype, L.oracle_num_threads.argtypes = ctypes.c_int, []
+    L.oracle_lora_merge.restype = None
+    L.oracle_lora_merge.argtypes = [u16p, i64, u16p, i64, u16p, i64, i64, i64, i64, f32, u16p]
     _lib = L
     return L
 
@@ -199,6 +201,28 @@ def bf16_linear(x_bits, w_bits, bias_bits=None, rows=None) -> np.ndarray:
         raise MemoryError("oracle_bf16_linear")
     del keep
     return Y
+
+
+# ----------------------------------------------------------------- weight refresh
+def lora_merge(w_bits: np.ndarray, a_bits: np.ndarray, b_bits: np.ndarray, scaling) -> np.ndarray:
+    """W' = bf16(W + s * B A) in the fixed binary32 order; W [N, K], A [r, K], B [N, r] as BF16 bits."""
+    w, a, b = _c(w_bits, np.uint16), _c(a_bits, np.uint16), _c(b_bits, np.uint16)
+    N, K = w.shape
+    r = a.shape[0]
+    if a.shape != (r, K) or b.shape != (N, r):
+        raise ValueError("shapes: W [N, K], A [r, K], B [N, r]")
+    out = np.empty((N, K), np.uint16)
+    _load().oracle_lora_merge(_p(w, ctypes.c_uint16), K, _p(a, ctypes.c_uint16), K, _p(b, ctypes.c_uint16), r,
+                              N, K, r, np.float32(scaling), _p(out, ctypes.c_uint16))
+    return out
+
+
+def requantize_lora(w_bits, a_bits, b_bits, scaling):
+    """Merge, then the weight quantizer: (W' bits, packed nibbles, row-major scales, T)."""
+    merged = lora_merge(w_bits, a_bits, b_bits, scaling)
+    T = tensor_scale(merged)
+    q, sf = quantize(merged, T)
+    return merged, q, sf, T
 
 
 def round_bf16(y: np.ndarray) -> np.ndarray:

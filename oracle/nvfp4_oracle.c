@@ -26,7 +26,9 @@
  * Pins (tests/test_oracle_*.py): closed-form tables, exhaustive E2M1/E4M3
  * rounding against an exact-rational brute force written separately in Python,
  * hand-worked block, exact round trips, metamorphic invariants, integer-exact
- * tiny matmuls.  Not pinned: byte-for-byte agreement with NVIDIA Transformer
+ * tiny matmuls; for the adapter merge: integer-exact cases, agreement with an FP64 library
+ * product up to the last BF16 place, two hand-worked cases that fix the order and the
+ * single rounding of the final multiply-add.  Not pinned: byte-for-byte agreement with NVIDIA Transformer
  * Engine's quantizer (the paper's backend; not available) -- "parity with
  * Transformer Engine unpinned".
  */
@@ -279,6 +281,32 @@ int oracle_bf16_linear(const uint16_t *x, int64_t ldx, const uint16_t *w, int64_
     free(A);
     free(B);
     return 0;
+}
+
+/* ------------------------------------------------------------------ weight refresh (LoRA merge) */
+
+/* The policy is trained through rank-r adapters (Section 4.1: r = 32, alpha = 64) and its
+ * weights are re-quantized into the NVFP4 engine after every update (Section 3.4,
+ * Appendix B.2).  The paper does not say how the adapters reach the engine; the reading taken
+ * here is the usual merge
+ *     W'[n][k] = W[n][k] + s * sum_j B[n][j] * A[j][k],      s = alpha / r,
+ * with W [N, K], A [r, K] ("down"), B [N, r] ("up") in BF16 and W' rounded to BF16, after
+ * which W' goes through the weight quantizer above.  Because W' decides quantized codes, its
+ * arithmetic is fixed as a sequence in IEEE binary32:
+ *     acc = 0;  for j = 0 .. r-1 in this order:  acc = fma(B[n][j], A[j][k], acc)
+ *     W'  = bf16_rne( fma(s, acc, W[n][k]) )
+ * (each fma rounds once; the BF16 products are exact in binary32).  `out` is dense [N, K]. */
+void oracle_lora_merge(const uint16_t *w, int64_t ldw, const uint16_t *a, int64_t lda, const uint16_t *b,
+                       int64_t ldb, int64_t N, int64_t K, int64_t r, float s, uint16_t *out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t k = 0; k < K; ++k) {
+            float acc = 0.0f;
+            for (int64_t j = 0; j < r; ++j)
+                acc = fmaf(oracle_bf16_to_f32(b[n * ldb + j]), oracle_bf16_to_f32(a[j * lda + k]), acc);
+            const float merged = fmaf(s, acc, oracle_bf16_to_f32(w[n * ldw + k]));
+            out[n * K + k] = oracle_f64_to_bf16((double)merged);  /* widening is exact: one rounding */
+        }
 }
 
 void oracle_f64_to_bf16_array(const double *y, int64_t n, uint16_t *out) {
