@@ -286,6 +286,50 @@ def run_ours(args):
     gemm_bytes = sum(l.M * l.K // 2 + B.scale_bytes(l.M, l.K) + l.N * l.K // 2 + B.scale_bytes(l.N, l.K) + 2 * l.N +
                      2 * l.M * l.N for l in layers)
 
+    # ---- weight refresh after a policy update: merge the rank-32 adapters of every targeted projection
+    # and re-quantize it.  FLUX targets to_q/k/v/out: 19 double blocks x 4 + 38 single blocks x 3 = 190
+    # matrices of 3072 x 3072.  Timed on 19 distinct matrices (359 MB of base weights, larger than L2)
+    # with one merged-weight scratch buffer, as a refresh loop would run it.
+    refresh = None
+    if world == 1:
+        RN = RK = 3072
+        n_mat, n_total = 19, 190
+        mats = []
+        for i in range(n_mat):
+            gen = torch.Generator(device=dev).manual_seed(9000 + i)
+            Wm = (torch.randn(RN, RK, generator=gen, device=dev) * RK ** -0.5).to(torch.bfloat16)
+            La, Lb = workloads.make_lora(RN, RK, i, dev)
+            mats.append((Wm, La, Lb))
+        plan = B.LoraRefreshPlan(mats, workloads.LORA_ALPHA / workloads.LORA_RANK)
+        refresh_pass = plan.run
+
+        def passes_ms(n):
+            refresh_pass()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n):
+                refresh_pass()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / n
+
+        t_refresh = passes_ms(50) / n_mat
+        B.sol_last_device_status()
+        fma = RN * RK * workloads.LORA_RANK
+        sm_mhz = 1965.0                                    # the part's maximum SM clock
+        alu_peak = 148 * 128 * 2 * sm_mhz * 1e6 / 1e12     # FP32 FMA issue: 128 lanes per SM per clock
+        refresh = {
+            "matrices_per_update": n_total, "shape": [RN, RK], "rank": workloads.LORA_RANK,
+            "us_per_matrix": t_refresh * 1e3, "ms_per_update": t_refresh * n_total,
+            "elements_per_s": RN * RK / (t_refresh * 1e-3),
+            "roofline": {"bound": "alu", "kernel": "lora_merge_kernel", "achieved": 2.0 * fma / (t_refresh * 1e-3) / 1e12,
+                         "peak": alu_peak, "unit": "TFLOP/s (fp32)", "frac": 2.0 * fma / (t_refresh * 1e-3) / 1e12 / alu_peak,
+                         "traffic": None,
+                         "note": "nvfp4_requantize_lora_batch (memset, merge, quantizer per matrix) against the FP32 issue peak "
+                                 "148 SM x 128 FMA/clk x 1965 MHz (maximum SM clock); the merge's chain order rules tensor cores out"},
+        }
+        del mats, plan
+
     # ---- end to end: pinned HOST activations in, HOST outputs back, copies inside the timed region,
     # through the host-buffer entry point of the C ABI, all six layers per step
     host_x = {}
@@ -346,6 +390,8 @@ def run_ours(args):
                                "frac": quant_bytes / (tot["quant"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
                                "traffic": int(NCU_TRAFFIC_RATIO["quantize"] * quant_bytes),
                                "peak_source": peak_src},
+        "stack_tflops_caller_supplied_scale": flops / ((tot["quant"] + tot["gemm"]) * 1e-3) / 1e12,
+        "weight_refresh": refresh,
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": kernels_per_layer * len(layers) * args.steps,
         "bf16_vs_torch_matmul_note": "MEASURED_PEAKS bf16 (torch.matmul 8192^3): %.0f burst / %.0f sustained TF" % (

@@ -109,6 +109,44 @@ sol_status_t nvfp4_quantize_weight(const void *w_bf16, int64_t N, int64_t K, int
                                    sol_sf_layout_t layout, void *stream);
 
 /*
+ * Weight refresh: merge rank-r adapters into the base weights and quantize the result, the step
+ * that follows every policy update (Section 3.4, Appendix B.2; Section 4.1: r = 32, alpha = 64,
+ * so scaling = alpha / r = 2).  The paper does not spell the merge out; this is the usual
+ *     W'[n][k] = bf16_rne( fma(scaling, acc, W[n][k]) ),
+ *     acc = 0;  acc = fma(B[n][j], A[j][k], acc)  for j = 0 .. r-1 in this order   (IEEE binary32)
+ * followed by nvfp4_quantize_weight's mapping applied to W'.
+ *   w_bf16      [N, K] BF16, pitch ldw; not modified (training keeps base and adapters apart)
+ *   lora_a      [r, K] BF16, pitch lda ("down" projection)
+ *   lora_b      [N, r] BF16, pitch ldb ("up" projection); 1 <= r <= 64
+ *   merged_bf16 [N, K] BF16, dense; receives W' (also the scratch the quantizer reads back)
+ *   q_out, sf_out, layout: as for nvfp4_quantize_weight
+ *   tensor_scale_out  TWO floats (device): [0] receives T of W'; [1] is scratch (it is left holding
+ *                     max|W'|, the value T was derived from)
+ * Three launches on the stream: clear the scratch word, the merge kernel, the quantizer.
+ */
+sol_status_t nvfp4_requantize_lora(const void *w_bf16, int64_t ldw, const void *lora_a, int64_t lda,
+                                   const void *lora_b, int64_t ldb, int64_t N, int64_t K, int64_t r,
+                                   float scaling, void *merged_bf16, void *q_out, void *sf_out,
+                                   float *tensor_scale_out, sol_sf_layout_t layout, void *stream);
+
+/*
+ * The same for `count` matrices of one shape (all targeted projections of a model after a policy
+ * update), in one call.  One matrix is ~20 us of GPU work, so launches are shared: matrices are
+ * processed in groups of up to min(merged_matrices, 8), three launches per group.  The six lists
+ * are HOST arrays of `count` DEVICE pointers; matrix i uses w_list[i] [N, K], a_list[i] [r, K],
+ * b_list[i] [N, r] (all dense) and writes q_list[i], sf_list[i], ts_list[i] (two floats each).
+ *   merged_bf16      device scratch for `merged_matrices` (>= 1) dense [N, K] BF16 matrices, reused
+ *                    group after group in stream order (contents undefined afterwards); a scratch
+ *                    that fits L2 keeps the merged weights out of HBM
+ * Everything is validated before the first launch.
+ */
+sol_status_t nvfp4_requantize_lora_batch(int64_t count, const void *const *w_list, const void *const *a_list,
+                                         const void *const *b_list, void *const *q_list, void *const *sf_list,
+                                         float *const *ts_list, int64_t N, int64_t K, int64_t r, float scaling,
+                                         void *merged_bf16, int64_t merged_matrices, sol_sf_layout_t layout,
+                                         void *stream);
+
+/*
  * Block-scaled FP4 GEMM with BF16 output (the NVFP4 linear the rollout runs, Section 3.4):
  *     acc[m,n] = sum_b sx[m,b] * sw[n,b] * sum_{k in b} qx[m,k] * qw[n,k]      (FP32 accumulate)
  *     Y[m,n]   = bf16_rne( fma(acc, Tx*Tw, bias[n]) )

@@ -22,6 +22,7 @@ EXPORTS = [
     "sol_nvfp4_linear_workspace_bytes", "sol_amax_bf16", "nvfp4_quantize", "nvfp4_quantize_weight",
     "nvfp4_linear", "bf16_linear", "nvfp4_quantize_linear", "sol_last_device_status",
     "sol_nvfp4_static_scratch_bytes", "nvfp4_quantize_linear_static", "nvfp4_quantize_linear_host",
+    "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch",
 ]
 
 _lib = None
@@ -64,6 +65,12 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_quantize_linear_static.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp]
     L.nvfp4_quantize_linear_host.restype = i32
     L.nvfp4_quantize_linear_host.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, vp, sz, vp]
+    L.nvfp4_requantize_lora.restype = i32
+    L.nvfp4_requantize_lora.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, ctypes.c_float, vp, vp, vp, vp,
+                                        i32, vp]
+    L.nvfp4_requantize_lora_batch.restype = i32
+    L.nvfp4_requantize_lora_batch.argtypes = [i64, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_float, vp, i64,
+                                              i32, vp]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -142,6 +149,76 @@ def nvfp4_quantize_weight(w: torch.Tensor, layout: int = SF_SWIZZLED_128x4):
     _check(lib().nvfp4_quantize_weight(_ptr(w), N, K, w.stride(0), _ptr(q), _ptr(sf), _ptr(ts), layout, _stream()),
            "nvfp4_quantize_weight")
     return q, sf, ts
+
+
+def nvfp4_requantize_lora(w: torch.Tensor, lora_a: torch.Tensor, lora_b: torch.Tensor, scaling: float,
+                          layout: int = SF_SWIZZLED_128x4, merged: torch.Tensor | None = None, out=None):
+    """Merge adapters (W + scaling * B A, BF16) and quantize: (merged W', nibbles, scales, T).
+
+    ``out`` = (q, sf, ts) supplies the output buffers; ts holds two floats (T and the entry
+    point's scratch word), the returned T is a view of its first element.
+    """
+    _need_2d_bf16(w, "w")
+    _need_2d_bf16(lora_a, "lora_a")
+    _need_2d_bf16(lora_b, "lora_b")
+    N, K = w.shape
+    r = lora_a.shape[0]
+    if lora_a.shape[1] != K or tuple(lora_b.shape) != (N, r):
+        raise ValueError("shapes: w [N, K], lora_a [r, K], lora_b [N, r]")
+    if merged is None:
+        merged = torch.empty((N, K), dtype=torch.bfloat16, device=w.device)
+    if out is None:
+        q, sf = _alloc_q(N, K, layout, w.device)
+        ts2 = torch.empty(2, dtype=torch.float32, device=w.device)
+    else:
+        q, sf, ts2 = out
+        if ts2.numel() < 2:
+            raise ValueError("ts must hold two floats")
+    _check(lib().nvfp4_requantize_lora(_ptr(w), w.stride(0), _ptr(lora_a), lora_a.stride(0), _ptr(lora_b),
+                                       lora_b.stride(0), N, K, r, float(scaling), _ptr(merged), _ptr(q),
+                                       _ptr(sf), _ptr(ts2), layout, _stream()), "nvfp4_requantize_lora")
+    return merged, q, sf, ts2[:1]
+
+
+class LoraRefreshPlan:
+    """Pointer lists for nvfp4_requantize_lora_batch, built once for a set of same-shaped matrices.
+
+    ``items`` = [(w, lora_a, lora_b), ...]; the outputs (q, sf, ts) are allocated here and kept in
+    ``outputs``; ``run()`` re-quantizes all of them with one call into the library, ``group``
+    matrices per launch (the merged-weight scratch holds that many).
+    """
+
+    def __init__(self, items, scaling: float, layout: int = SF_SWIZZLED_128x4, group: int = 8):
+        if not items:
+            raise ValueError("no matrices")
+        N, K = items[0][0].shape
+        r = items[0][1].shape[0]
+        for w, a, b in items:
+            for t, name in ((w, "w"), (a, "lora_a"), (b, "lora_b")):
+                _need_2d_bf16(t, name)
+                if not t.is_contiguous():
+                    raise ValueError(f"{name} must be dense")
+            if tuple(w.shape) != (N, K) or tuple(a.shape) != (r, K) or tuple(b.shape) != (N, r):
+                raise ValueError("all matrices of a plan share one shape")
+        dev = items[0][0].device
+        self.items = list(items)
+        self.N, self.K, self.r, self.scaling, self.layout = N, K, r, float(scaling), layout
+        self.group = max(1, min(group, len(items)))
+        self.merged = torch.empty((self.group, N, K), dtype=torch.bfloat16, device=dev)
+        self.outputs = []
+        for _ in items:
+            q, sf = _alloc_q(N, K, layout, dev)
+            self.outputs.append((q, sf, torch.empty(2, dtype=torch.float32, device=dev)))
+        n = len(items)
+        arr = ctypes.c_void_p * n
+        self._lists = [arr(*[t[i].data_ptr() for t in items]) for i in range(3)] + \
+                      [arr(*[o[i].data_ptr() for o in self.outputs]) for i in range(3)]
+
+    def run(self):
+        _check(lib().nvfp4_requantize_lora_batch(len(self.items), *self._lists, self.N, self.K, self.r,
+                                                 self.scaling, _ptr(self.merged), self.group, self.layout, _stream()),
+               "nvfp4_requantize_lora_batch")
+        return self.outputs
 
 
 def nvfp4_linear(xq, xsf, x_tscale, wq, wsf, w_tscale, bias=None, out: torch.Tensor | None = None):

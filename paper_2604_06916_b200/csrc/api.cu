@@ -190,6 +190,88 @@ sol_status_t nvfp4_quantize_weight(const void *w_bf16, int64_t N, int64_t K, int
     return launch_quantize(w_bf16, N, K, ldw, tensor_scale_out, q_out, sf_out, layout, s);
 }
 
+static sol_status_t check_requantize_lora(const void *w, const void *a, const void *b, const void *merged,
+                                          const void *q, const void *sf, const float *ts, int64_t ldw, int64_t lda,
+                                          int64_t ldb, int64_t N, int64_t K, int64_t r, sol_sf_layout_t layout) {
+    if (w == nullptr || a == nullptr || b == nullptr || merged == nullptr || q == nullptr || sf == nullptr ||
+        ts == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(N, K) || ldw < K || lda < K || r < 1 || r > lora_max_rank() || ldb < r || N > 65535LL * 64)
+        return SOL_ERR_BAD_SHAPE;
+    if (layout != SOL_SF_ROW_MAJOR && layout != SOL_SF_SWIZZLED_128x4) return SOL_ERR_BAD_LAYOUT;
+    if (!aligned16(w) || !aligned16(a) || !aligned16(merged) || !aligned16(q) || !aligned16(sf) || ldw % 8 != 0 ||
+        lda % 8 != 0 || (reinterpret_cast<uintptr_t>(b) & 1u) || (reinterpret_cast<uintptr_t>(ts) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    return SOL_OK;
+}
+
+sol_status_t nvfp4_requantize_lora(const void *w_bf16, int64_t ldw, const void *lora_a, int64_t lda,
+                                   const void *lora_b, int64_t ldb, int64_t N, int64_t K, int64_t r, float scaling,
+                                   void *merged_bf16, void *q_out, void *sf_out, float *tensor_scale_out,
+                                   sol_sf_layout_t layout, void *stream) {
+    sol_status_t st = check_requantize_lora(w_bf16, lora_a, lora_b, merged_bf16, q_out, sf_out, tensor_scale_out, ldw,
+                                            lda, ldb, N, K, r, layout);
+    if (st != SOL_OK) return st;
+    const DeviceInfo *dev = nullptr;
+    st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    MergeGroup mg = {};
+    mg.w[0] = static_cast<const uint16_t *>(w_bf16);
+    mg.a[0] = static_cast<const uint16_t *>(lora_a);
+    mg.b[0] = static_cast<const uint16_t *>(lora_b);
+    mg.out[0] = static_cast<uint16_t *>(merged_bf16);
+    mg.scale_words[0] = tensor_scale_out;
+    st = launch_lora_merge(mg, 1, ldw, lda, ldb, N, K, r, scaling, s);
+    if (st != SOL_OK) return st;
+    return launch_quantize_from_amax(merged_bf16, N, K, K, tensor_scale_out, q_out, sf_out, layout, s);
+}
+
+sol_status_t nvfp4_requantize_lora_batch(int64_t count, const void *const *w_list, const void *const *a_list,
+                                         const void *const *b_list, void *const *q_list, void *const *sf_list,
+                                         float *const *ts_list, int64_t N, int64_t K, int64_t r, float scaling,
+                                         void *merged_bf16, int64_t merged_matrices, sol_sf_layout_t layout,
+                                         void *stream) {
+    if (count < 0 || merged_matrices < 1) return SOL_ERR_BAD_SHAPE;
+    if (count == 0) return SOL_OK;
+    if (w_list == nullptr || a_list == nullptr || b_list == nullptr || q_list == nullptr || sf_list == nullptr ||
+        ts_list == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    // validate every matrix before the first launch: an error status means nothing was launched
+    for (int64_t i = 0; i < count; ++i) {
+        const sol_status_t st = check_requantize_lora(w_list[i], a_list[i], b_list[i], merged_bf16, q_list[i],
+                                                      sf_list[i], ts_list[i], K, K, r, N, K, r, layout);
+        if (st != SOL_OK) return st;
+    }
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int64_t group = merged_matrices < kMaxGroup ? merged_matrices : kMaxGroup;
+    for (int64_t i0 = 0; i0 < count; i0 += group) {
+        const int n = static_cast<int>(count - i0 < group ? count - i0 : group);
+        MergeGroup mg = {};
+        QuantGroup qg = {};
+        for (int i = 0; i < n; ++i) {
+            uint16_t *merged = static_cast<uint16_t *>(merged_bf16) + static_cast<int64_t>(i) * N * K;
+            mg.w[i] = static_cast<const uint16_t *>(w_list[i0 + i]);
+            mg.a[i] = static_cast<const uint16_t *>(a_list[i0 + i]);
+            mg.b[i] = static_cast<const uint16_t *>(b_list[i0 + i]);
+            mg.out[i] = merged;
+            mg.scale_words[i] = ts_list[i0 + i];
+            qg.x[i] = merged;
+            qg.scale_words[i] = ts_list[i0 + i];
+            qg.q[i] = static_cast<uint8_t *>(q_list[i0 + i]);
+            qg.sf[i] = static_cast<uint8_t *>(sf_list[i0 + i]);
+        }
+        st = launch_lora_merge(mg, n, K, K, r, N, K, r, scaling, s);
+        if (st != SOL_OK) return st;
+        st = launch_quantize_group(qg, n, N, K, layout, s);
+        if (st != SOL_OK) return st;
+    }
+    return SOL_OK;
+}
+
 static sol_status_t check_linear_common(const void *bias, const void *y, int64_t M, int64_t N, int64_t K,
                                         int64_t ldy) {
     if (!shape_ok(M, K) || N <= 0 || N % 8 != 0 || N > (1LL << 24) || ldy < N) return SOL_ERR_BAD_SHAPE;

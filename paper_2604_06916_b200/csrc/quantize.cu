@@ -88,10 +88,9 @@ __device__ __forceinline__ uint32_t quantize8(const uint4 &v, float rcp) {
 // With `amax` set the tensor scale is derived here from the amax word the reduction left (the
 // bit pattern of max|x| as FP32) and block (0,0) publishes it in `tscale_out` for the GEMM.
 template <bool kSwizzled>
-__global__ void __launch_bounds__(kQuantThreads)
-quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
-                const float *tscale, const float *amax, float *tscale_out, uint8_t *__restrict__ q,
-                uint8_t *__restrict__ sf) {
+__device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
+                                              const float *tscale, const float *amax, float *tscale_out,
+                                              uint8_t *__restrict__ q, uint8_t *__restrict__ sf) {
     __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kTileK / 16)];  // 2 KB = 4 chunks
 
     const int b = threadIdx.x & 15;   // scale block inside the tile
@@ -162,6 +161,23 @@ quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t
             }
         }
     }
+}
+
+template <bool kSwizzled>
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
+                const float *tscale, const float *amax, float *tscale_out, uint8_t *__restrict__ q,
+                uint8_t *__restrict__ sf) {
+    quantize_tile<kSwizzled>(x, rows, K, ld, tscale, amax, tscale_out, q, sf);
+}
+
+// The same over a group of equally shaped dense tensors, one per blockIdx.z, each with its own
+// amax word (the weight refresh quantizes several merged matrices per launch).
+template <bool kSwizzled>
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_group_kernel(const __grid_constant__ QuantGroup g, int64_t rows, int64_t K) {
+    const int z = blockIdx.z;
+    quantize_tile<kSwizzled>(g.x[z], rows, K, K, nullptr, g.scale_words[z] + 1, g.scale_words[z], g.q[z], g.sf[z]);
 }
 
 // max |x| over the tensor as the bit pattern of the FP32 value (BF16 magnitude << 16).
@@ -262,12 +278,37 @@ sol_status_t launch_quantize(const void *x, int64_t rows, int64_t K, int64_t ld,
     return launch_quantize_ex(x, rows, K, ld, tscale, nullptr, nullptr, q, sf, layout, stream);
 }
 
+sol_status_t launch_quantize_from_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,
+                                       void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream) {
+    return launch_quantize_ex(x, rows, K, ld, nullptr, scale_words + 1, scale_words, q, sf, layout, stream);
+}
+
+sol_status_t launch_quantize_group(const QuantGroup &g, int count, int64_t rows, int64_t K, sol_sf_layout_t layout,
+                                   cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ceil_div(K, kTileK)), static_cast<unsigned>(ceil_div(rows, kTileRows)),
+                       static_cast<unsigned>(count));
+    cfg.blockDim = dim3(kQuantThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    auto kern = layout == SOL_SF_SWIZZLED_128x4 ? quantize_group_kernel<true> : quantize_group_kernel<false>;
+    if (cudaLaunchKernelEx(&cfg, kern, g, rows, K) != cudaSuccess) {
+        cudaGetLastError();
+        return SOL_ERR_CUDA;
+    }
+    return launch_status();
+}
+
 sol_status_t launch_amax_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,
                                   void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream,
                                   const DeviceInfo *dev) {
     sol_status_t st = launch_amax_bits(x, rows, K, ld, reinterpret_cast<uint32_t *>(scale_words + 1), stream, dev);
     if (st != SOL_OK) return st;
-    return launch_quantize_ex(x, rows, K, ld, nullptr, scale_words + 1, scale_words, q, sf, layout, stream);
+    return launch_quantize_from_amax(x, rows, K, ld, scale_words, q, sf, layout, stream);
 }
 
 }  // namespace sol

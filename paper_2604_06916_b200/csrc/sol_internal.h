@@ -42,6 +42,31 @@ sol_status_t launch_quantize(const void *x, int64_t rows, int64_t K, int64_t ld,
 sol_status_t launch_amax_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,
                                   void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream,
                                   const DeviceInfo *dev);
+// Quantizer that derives T from max|x| left in scale_words[1] (FP32 bits) and publishes T in scale_words[0].
+sol_status_t launch_quantize_from_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,
+                                       void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream);
+// Groups of equally shaped matrices handled by one launch (blockIdx.z picks the matrix).
+constexpr int kMaxGroup = 8;
+struct MergeGroup {
+    const uint16_t *w[kMaxGroup];   // base weights [N, K], pitch ldw
+    const uint16_t *a[kMaxGroup];   // adapter down factors [r, K], pitch lda
+    const uint16_t *b[kMaxGroup];   // adapter up factors [N, r], pitch ldb
+    uint16_t *out[kMaxGroup];       // merged weights, dense [N, K]
+    float *scale_words[kMaxGroup];  // [0]: T (written by the quantizer), [1]: max|W'| as FP32 bits
+};
+struct QuantGroup {
+    const uint16_t *x[kMaxGroup];   // dense [rows, K]
+    float *scale_words[kMaxGroup];
+    uint8_t *q[kMaxGroup];
+    uint8_t *sf[kMaxGroup];
+};
+// Adapter merge W' = bf16(W + s * B A) for `count` matrices: zeroes each scale_words[i][1], then
+// accumulates max|W'| into it as FP32 bits.
+sol_status_t launch_lora_merge(const MergeGroup &g, int count, int64_t ldw, int64_t lda, int64_t ldb, int64_t N,
+                               int64_t K, int64_t r, float s, cudaStream_t stream);
+sol_status_t launch_quantize_group(const QuantGroup &g, int count, int64_t rows, int64_t K, sol_sf_layout_t layout,
+                                   cudaStream_t stream);
+int lora_max_rank();
 sol_status_t launch_gemm_bf16(const void *x, const void *w, const void *bias, void *y, int64_t M,
                               int64_t N, int64_t K, int64_t ldx, int64_t ldw, int64_t ldy,
                               cudaStream_t stream, const DeviceInfo *dev);

@@ -119,6 +119,24 @@ def make_layer(cfg: Config, index: int, device="cpu", M: int | None = None, with
     return X, W, bias
 
 
+LORA_RANK = 32    # Section 4.1: rank 32, alpha 64 in every experiment
+LORA_ALPHA = 64.0
+
+
+def make_lora(N: int, K: int, seed: int, device="cpu", rank: int = LORA_RANK):
+    """Adapter factors of a trained policy, (A bf16 [rank, K], B bf16 [N, rank]).
+
+    A keeps its Gaussian init (sigma = 1/rank, the usual default); B starts at zero and drifts
+    during training, modelled as N(0, 0.02^2) so that (alpha/rank) * B A perturbs a weight of
+    sigma K^-1/2 by a few per cent and moves most of its BF16 bits.
+    """
+    gen = torch.Generator(device=device)
+    gen.manual_seed(77_000 + seed)
+    A = (_normal((rank, K), gen, device) * (1.0 / rank)).to(torch.bfloat16)
+    B = (_normal((N, rank), gen, device) * 0.02).to(torch.bfloat16)
+    return A, B
+
+
 def to_bits(t: torch.Tensor):
     """bf16 tensor -> numpy uint16 bit patterns (host)."""
     import numpy as np
