@@ -409,6 +409,27 @@ def run_only(args):
     from paper_2604_06916_b200 import binding as B
     from paper_2604_06916_b200 import workloads
 
+    if args.only == "weight_refresh":
+        # eight FLUX attention projections (3072 x 3072, rank-32 adapters) through the batched entry
+        n = 3072
+        mats = []
+        for i in range(8):
+            gen = torch.Generator(device="cuda").manual_seed(9000 + i)
+            Wm = (torch.randn(n, n, generator=gen, device="cuda") * n ** -0.5).to(torch.bfloat16)
+            mats.append((Wm,) + workloads.make_lora(n, n, i, "cuda"))
+        plan = B.LoraRefreshPlan(mats, workloads.LORA_ALPHA / workloads.LORA_RANK)
+        times = []
+        for it in range(args.warmup + args.steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            plan.run()
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                times.append(e0.elapsed_time(e1))
+        B.sol_last_device_status()
+        print(json.dumps({"only": "weight_refresh", "matrices": 8, "us_per_matrix": 1e3 * sum(times) / len(times) / 8}))
+        return
     cfg = workloads.CONFIGS[args.workload]
     index = [l.name for l in cfg.layers].index(args.only)
     l = cfg.layers[index]
@@ -439,7 +460,7 @@ def run_only(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload")
+    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh'")
     ap.add_argument("--rows", type=int, default=0, help="profile mode: override M")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
