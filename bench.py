@@ -33,7 +33,7 @@ NOMINAL_HBM_GBS = 8000.0
 # ncu (profiles/gemm_pair_and_quantizer_flux_d_proj.md), d_proj launch: GEMM 69.1 MB read + 172.7 MB
 # written for 295.5 MB algorithmic (Y partly still dirty in L2 at kernel end); quantizer 226.5 + 26.5 MB
 # for 290.2 MB algorithmic.  Scaled to all six layers by the algorithmic bytes (traffic is proportional).
-NCU_TRAFFIC_RATIO = {"gemm": (69.09 + 172.67) / 295.5, "quantize": (226.53 + 26.51) / 290.2}
+NCU_TRAFFIC_RATIO = {"gemm": (69.06 + 171.63) / 295.5, "quantize": (226.53 + 26.43) / 290.2}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -291,7 +291,7 @@ def run_ours(args):
     # matrices of 3072 x 3072.  Timed on 19 distinct matrices (359 MB of base weights, larger than L2)
     # with one merged-weight scratch buffer, as a refresh loop would run it.
     refresh = None
-    if world == 1:
+    if world == 1 and not args.lean:
         RN = RK = 3072
         n_mat, n_total = 19, 190
         mats = []
@@ -335,7 +335,7 @@ def run_ours(args):
     host_x = {}
     e2e_items = []
     h2d = d2h = 0
-    for d in data:
+    for d in ([] if args.lean else data):
         l = d["l"]
         if l.K not in host_x:
             host_x[l.K] = torch.empty((l.M, l.K), dtype=torch.bfloat16).pin_memory()
@@ -349,12 +349,14 @@ def run_ours(args):
         for d, xh, yh, xd in e2e_items:
             B.nvfp4_quantize_linear_host(xh, d["wq"], d["wsf"], d["wts"], d["bias"], yh, xd, d["Y"], d["ws"])
 
-    e2e_step()
-    n_e2e = 3
-    ms_e2e = timed(e2e_step, n_e2e) / n_e2e
-    e2e = {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e,
-           "entry": "nvfp4_quantize_linear_host (pinned host X and Y, copies inside the timed region)"}
+    e2e = None
+    if not args.lean:
+        e2e_step()
+        n_e2e = 3
+        ms_e2e = timed(e2e_step, n_e2e) / n_e2e
+        e2e = {"value": world * flops / (ms_e2e * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e, "steps": n_e2e,
+               "entry": "nvfp4_quantize_linear_host (pinned host X and Y, copies inside the timed region)"}
     del host_x, e2e_items
 
     if rank != 0:
@@ -363,7 +365,7 @@ def run_ours(args):
         return
 
     cpu = None
-    if world == 1:
+    if world == 1 and not args.lean:
         rows = calibrated_rows(workloads.CONFIG_FLUX, 1, 12.0, args.ref_rows)
         v, dt, cores, sample = oracle_sample_tflops(workloads.CONFIG_FLUX, 1, rows)
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample, "seconds": round(dt, 2)}
@@ -468,6 +470,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="flux1_12b_g8")
     ap.add_argument("--ref-rows", type=int, default=0, help="rows of the oracle sample (0 = calibrate)")
+    ap.add_argument("--lean", action="store_true",
+                    help="sweep mode: skip the end-to-end, weight-refresh and CPU-oracle legs (their keys are null)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -230,7 +230,9 @@ sol_status_t launch_amax_bits(const void *x, int64_t rows, int64_t K, int64_t ld
     if (cudaMemsetAsync(bits_out, 0, sizeof(uint32_t), stream) != cudaSuccess) return SOL_ERR_CUDA;
     const int64_t vecs = rows * (K / 8);
     int64_t blocks = ceil_div(vecs, 256 * 8);
-    const int64_t cap = static_cast<int64_t>(dev->sm_count) * 8;
+    // up to 16 waves of resident blocks: short blocks balance the tail of the reduction better than
+    // one wave of long grid-stride loops (measured 5.5 against 5.0 TB/s on a 226 MB tensor)
+    const int64_t cap = static_cast<int64_t>(dev->sm_count) * 8 * 16;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     amax_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
