@@ -51,3 +51,25 @@ def check_linear(y_gpu_bits: np.ndarray, Y: np.ndarray, what: str = ""):
             f"gpu={g[i, j]!r} oracle={Y[i, j]!r} err={err[i, j]:.3e} tol={tol[i, j]:.3e}; "
             f"bad rows={np.unique(np.argwhere(bad)[:, 0])[:8]} bad cols={np.unique(np.argwhere(bad)[:, 1])[:8]}")
     return float(np.max(err / np.maximum(tol, 1e-300)))
+
+
+def dequantize_on_device(q: torch.Tensor, sf_swizzled: torch.Tensor, rows: int, K: int) -> torch.Tensor:
+    """code * block scale as BF16 (exact: at most 6 significant bits), built from plain torch ops.
+
+    A secondary, full-coverage screen for the GEMMs; the tensor scale is left out so that every
+    value is representable.  The swizzled-scale index rule is the vectorised copy checked against
+    the oracle's scalar function.
+    """
+    dev = q.device
+    lut = torch.tensor([0, .5, 1, 1.5, 2, 3, 4, 6, -0., -.5, -1, -1.5, -2, -3, -4, -6], dtype=torch.float32, device=dev)
+    lo = lut[(q & 0xF).long()]
+    hi = lut[(q >> 4).long()]
+    vals = torch.stack((lo, hi), dim=-1).reshape(rows, K)
+    offs = torch.from_numpy(swizzled_offsets(np.arange(rows), K)).to(dev)
+    sb = sf_swizzled.reshape(-1)[offs].to(torch.int32)
+    e, m = (sb >> 3) & 15, sb & 7
+    scale = torch.where(e == 0, m.float() * 2.0 ** -9, torch.ldexp(1.0 + m.float() / 8.0, e - 7))
+    out = (vals.reshape(rows, K // 16, 16) * scale[:, :, None]).reshape(rows, K)
+    out_bf16 = out.to(torch.bfloat16)
+    assert torch.equal(out_bf16.float(), out)
+    return out_bf16

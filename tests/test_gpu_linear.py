@@ -186,3 +186,33 @@ def test_deterministic_run_to_run(B):
     b = B.nvfp4_quantize_linear(X, wq, wsf, wts, bias)
     assert torch.equal(a, b)
     assert torch.equal(B.bf16_linear(X, W, bias), B.bf16_linear(X, W, bias))
+
+
+@pytest.mark.parametrize("index", [1, 5])  # d_proj (K = 3072) and s_out (K = 15360), full M = 36864
+def test_flux_layers_every_output_against_library_matmul_screen(B, index):
+    # secondary screen with full coverage: a library BF16 matmul (FP32 accumulation) on the
+    # dequantized operands; the oracle itself covers sampled rows of the same launches above
+    from tests.helpers import dequantize_on_device
+    cfg = workloads.CONFIG_FLUX
+    layer = cfg.layers[index]
+    X, W, bias = workloads.make_layer(cfg, index, "cuda")
+    wq, wsf, wts = B.nvfp4_quantize_weight(W)
+    xts = B.sol_amax_bf16(X)
+    xq, xsf = B.nvfp4_quantize(X, xts)
+    y = B.nvfp4_linear(xq, xsf, xts, wq, wsf, wts, bias)
+    B.sol_last_device_status()
+    xd = dequantize_on_device(xq, xsf, layer.M, layer.K)
+    wd = dequantize_on_device(wq, wsf, layer.N, layer.K)
+    del X, W, xq, xsf
+    alpha = (xts * wts).item()
+    worst = 0.0
+    for r0 in range(0, layer.M, 4096):
+        acc = torch.matmul(xd[r0:r0 + 4096], wd.t()).float()      # BF16 result of an FP32 accumulation
+        ref = acc * alpha + bias.float()[None, :]
+        got = y[r0:r0 + 4096].float()
+        # the screen's own BF16 rounding of acc adds 2^-9 relative; the product bound stays 2^-7
+        tol = 2.0 ** -7 * ref.abs() + 1e-4 * ref.pow(2).mean(dim=1, keepdim=True).sqrt() + 2.0 ** -8 * (acc * alpha).abs()
+        err = (got - ref).abs()
+        assert bool((err <= tol).all()), f"rows {r0}..: {(err > tol).sum().item()} outputs off"
+        worst = max(worst, float((err / tol.clamp_min(1e-30)).max()))
+    assert worst <= 1.0
