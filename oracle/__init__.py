@@ -61,6 +61,8 @@ def _load():
     L.oracle_bf16_linear.argtypes = [u16p, i64, u16p, i64, u16p, i64, i64, i64p, i64, f64p]
     L.oracle_f64_to_bf16_array.restype, L.oracle_f64_to_bf16_array.argtypes = None, [f64p, i64, u16p]
     L.oracle_num_threads.restype, L.oracle_num_threads.argtypes = ctypes.c_int, []
+    L.oracle_gelu_tanh.restype, L.oracle_gelu_tanh.argtypes = ctypes.c_double, [ctypes.c_double]
+    L.oracle_gelu_tanh_array.restype, L.oracle_gelu_tanh_array.argtypes = None, [f64p, i64, f64p]
     L.oracle_lora_merge.restype = None
     L.oracle_lora_merge.argtypes = [u16p, i64, u16p, i64, u16p, i64, i64, i64, i64, f32, u16p]
     _lib = L
@@ -201,6 +203,31 @@ def bf16_linear(x_bits, w_bits, bias_bits=None, rows=None) -> np.ndarray:
         raise MemoryError("oracle_bf16_linear")
     del keep
     return Y
+
+
+# ----------------------------------------------------------------- linear with quantized output
+ACT_NONE, ACT_GELU_TANH = 0, 1
+
+
+def gelu_tanh(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.empty_like(x)
+    _load().oracle_gelu_tanh_array(_p(x, ctypes.c_double), x.size, _p(out, ctypes.c_double))
+    return out
+
+
+def nvfp4_linear_quantized(qx, sfx, Tx, qw, sfw, Tw, bias_bits, act: int, T_out, rows=None):
+    """The NVFP4 linear followed by an activation and the activation quantizer of the NEXT linear.
+
+    H = act(Y) with Y the FP64 linear; h = H rounded once to BF16 (what an unfused pipeline would
+    store); (q, sf) = quantize(h, T_out) with a caller-supplied T_out.  Returns (H as FP64, h bits,
+    packed nibbles, row-major scales).
+    """
+    Y = nvfp4_linear(qx, sfx, Tx, qw, sfw, Tw, bias_bits, rows=rows)
+    H = gelu_tanh(Y) if act == ACT_GELU_TANH else Y
+    h = round_bf16(H)
+    q, sf = quantize(h, T_out)
+    return H, h, q, sf
 
 
 # ----------------------------------------------------------------- weight refresh

@@ -283,6 +283,20 @@ int oracle_bf16_linear(const uint16_t *x, int64_t ldx, const uint16_t *w, int64_
     return 0;
 }
 
+/* ------------------------------------------------------------------ activation between two linears */
+
+/* GELU in its tanh form, the activation of the DiT feed-forward blocks whose linears the rollout
+ * runs in NVFP4 (the paper does not restate it):
+ *     gelu(x) = x/2 * (1 + tanh( sqrt(2/pi) * (x + 0.044715 x^3) )),   evaluated in FP64. */
+double oracle_gelu_tanh(double x) {
+    const double c = 0.79788456080286535588;  /* sqrt(2/pi) */
+    return 0.5 * x * (1.0 + tanh(c * (x + 0.044715 * x * x * x)));
+}
+
+void oracle_gelu_tanh_array(const double *x, int64_t n, double *out) {
+    for (int64_t i = 0; i < n; ++i) out[i] = oracle_gelu_tanh(x[i]);
+}
+
 /* ------------------------------------------------------------------ weight refresh (LoRA merge) */
 
 /* The policy is trained through rank-r adapters (Section 4.1: r = 32, alpha = 64) and its
