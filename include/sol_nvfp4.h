@@ -59,6 +59,7 @@ typedef enum {
 } sol_status_t;
 
 typedef enum { SOL_SF_ROW_MAJOR = 0, SOL_SF_SWIZZLED_128x4 = 1 } sol_sf_layout_t;
+typedef enum { SOL_ACT_NONE = 0, SOL_ACT_GELU_TANH = 1 } sol_activation_t;
 
 /* Static, human-readable name of a status (host pointer, never NULL). */
 const char *sol_status_string(sol_status_t status);
@@ -160,6 +161,31 @@ sol_status_t nvfp4_linear(const void *xq, const void *xsf, const float *x_tscale
                           const void *wq, const void *wsf, const float *w_tscale,
                           const void *bias_bf16, void *y_bf16, int64_t M, int64_t N, int64_t K,
                           int64_t ldy, void *stream);
+
+/*
+ * The NVFP4 linear with its output already quantized for the NEXT NVFP4 linear: between two
+ * rollout linears (Section 3.4) the activations never exist in BF16 in memory, which removes the
+ * 2 B/element store, the amax pass and the 2.56 B/element quantizer pass of the next layer.
+ *     y[m,n] = fma(acc[m,n], Tx*Tw, bias[n])                     (as nvfp4_linear, FP32)
+ *     h[m,n] = bf16_rne( act(y[m,n]) )       act = identity or GELU (tanh form), FP32
+ *     (hq, hsf) = the activation quantizer of nvfp4_quantize applied to h along N with T = *out_tscale
+ * The two-level scale needs T before the first output exists, so T is the caller's: a calibrated
+ * value or the one derived from the previous step's amax_out (a value too small only saturates
+ * more blocks at 6*448*T).
+ *   out_tscale  one float (device), > 0
+ *   hq_out      packed nibbles [M, N/2];  hsf_out  scales, SOL_SF_SWIZZLED_128x4 layout of an [M, N]
+ *               tensor, sol_nvfp4_scale_bytes(M, N, ...) bytes, padding rows written as 0
+ *   amax_out    nullable; one device word holding max|h| as an FP32 value, updated with an atomic
+ *               max (a running maximum: the caller zeroes it to start a new window)
+ *   N % 64 == 0.  GELU is evaluated in FP32 with the hardware tanh (absolute error of tanh about
+ *   2^-11): far below the BF16 rounding and the FP4 grid that follow, but h can differ from an exactly
+ *   evaluated GELU in its last BF16 place more often than the GEMM's accumulation order alone causes.
+ */
+sol_status_t nvfp4_linear_quantized_out(const void *xq, const void *xsf, const float *x_tscale, const void *wq,
+                                        const void *wsf, const float *w_tscale, const void *bias_bf16,
+                                        sol_activation_t activation, const float *out_tscale, void *hq_out,
+                                        void *hsf_out, float *amax_out, int64_t M, int64_t N, int64_t K,
+                                        void *stream);
 
 /*
  * BF16 linear, the full-precision stage-2 reference (Section 3.4):

@@ -22,7 +22,7 @@ EXPORTS = [
     "sol_nvfp4_linear_workspace_bytes", "sol_amax_bf16", "nvfp4_quantize", "nvfp4_quantize_weight",
     "nvfp4_linear", "bf16_linear", "nvfp4_quantize_linear", "sol_last_device_status",
     "sol_nvfp4_static_scratch_bytes", "nvfp4_quantize_linear_static", "nvfp4_quantize_linear_host",
-    "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch",
+    "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch", "nvfp4_linear_quantized_out",
 ]
 
 _lib = None
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_requantize_lora_batch.restype = i32
     L.nvfp4_requantize_lora_batch.argtypes = [i64, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_float, vp, i64,
                                               i32, vp]
+    L.nvfp4_linear_quantized_out.restype = i32
+    L.nvfp4_linear_quantized_out.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, i64, i64, i64, vp]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -230,6 +232,23 @@ def nvfp4_linear(xq, xsf, x_tscale, wq, wsf, w_tscale, bias=None, out: torch.Ten
     _check(lib().nvfp4_linear(_ptr(xq), _ptr(xsf), _ptr(x_tscale), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
                               _ptr(out), M, N, K, out.stride(0), _stream()), "nvfp4_linear")
     return out
+
+
+ACT_NONE, ACT_GELU_TANH = 0, 1
+
+
+def nvfp4_linear_quantized_out(xq, xsf, x_tscale, wq, wsf, w_tscale, bias, activation: int, out_tscale,
+                               amax_out: torch.Tensor | None = None, out=None):
+    """NVFP4 linear whose output leaves as (nibbles [M, N/2], swizzled scales) for the next linear."""
+    M, K = xq.shape[0], xq.shape[1] * 2
+    N = wq.shape[0]
+    if out is None:
+        out = _alloc_q(M, N, SF_SWIZZLED_128x4, xq.device)
+    hq, hsf = out
+    _check(lib().nvfp4_linear_quantized_out(_ptr(xq), _ptr(xsf), _ptr(x_tscale), _ptr(wq), _ptr(wsf), _ptr(w_tscale),
+                                            _ptr(bias), activation, _ptr(out_tscale), _ptr(hq), _ptr(hsf),
+                                            _ptr(amax_out), M, N, K, _stream()), "nvfp4_linear_quantized_out")
+    return hq, hsf
 
 
 def bf16_linear(x, w, bias=None, out: torch.Tensor | None = None):

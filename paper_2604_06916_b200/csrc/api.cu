@@ -1,6 +1,7 @@
 // C-ABI entry points: argument validation, size queries, device checks, TMA descriptor
 // encoding.  Every compute step runs in the kernels of quantize.cu and gemm.cu.
 #include "sol_internal.h"
+#include "gemm_common.cuh"
 
 #include <mutex>
 
@@ -309,6 +310,29 @@ sol_status_t bf16_linear(const void *x_bf16, const void *w_bf16, const void *bia
     if (st != SOL_OK) return st;
     return launch_gemm_bf16(x_bf16, w_bf16, bias_bf16, y_bf16, M, N, K, ldx, ldw, ldy,
                             static_cast<cudaStream_t>(stream), dev);
+}
+
+sol_status_t nvfp4_linear_quantized_out(const void *xq, const void *xsf, const float *x_tscale, const void *wq,
+                                        const void *wsf, const float *w_tscale, const void *bias_bf16,
+                                        sol_activation_t activation, const float *out_tscale, void *hq_out,
+                                        void *hsf_out, float *amax_out, int64_t M, int64_t N, int64_t K, void *stream) {
+    if (xq == nullptr || xsf == nullptr || x_tscale == nullptr || wq == nullptr || wsf == nullptr ||
+        w_tscale == nullptr || out_tscale == nullptr || hq_out == nullptr || hsf_out == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(M, K) || N <= 0 || N % 64 != 0 || N > (1LL << 24)) return SOL_ERR_BAD_SHAPE;
+    if (activation != SOL_ACT_NONE && activation != SOL_ACT_GELU_TANH) return SOL_ERR_BAD_LAYOUT;
+    if (!aligned16(xq) || !aligned16(xsf) || !aligned16(wq) || !aligned16(wsf) || !aligned16(hq_out) ||
+        !aligned16(hsf_out) || (bias_bf16 != nullptr && !aligned16(bias_bf16)) ||
+        (reinterpret_cast<uintptr_t>(x_tscale) & 3u) || (reinterpret_cast<uintptr_t>(w_tscale) & 3u) ||
+        (reinterpret_cast<uintptr_t>(out_tscale) & 3u) || (reinterpret_cast<uintptr_t>(amax_out) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return gemm::launch_pair256_nvfp4_quant_out(xq, xsf, x_tscale, wq, wsf, w_tscale, bias_bf16,
+                                                activation == SOL_ACT_GELU_TANH ? 1 : 0, out_tscale, hq_out, hsf_out,
+                                                reinterpret_cast<uint32_t *>(amax_out), M, N, K,
+                                                static_cast<cudaStream_t>(stream), dev);
 }
 
 sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,

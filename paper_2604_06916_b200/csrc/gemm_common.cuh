@@ -47,6 +47,10 @@ struct Params {
     uint32_t dbg;
     int M, N, K;
     int m_tiles, n_tiles;
+    // quantized-output epilogue (NVFP4 pair kernel only): Y leaves as the next linear's Q(X)
+    uint8_t *sf_out;        // scales of the output, chunked layout for an [M, N] tensor
+    const float *ts_out;    // tensor scale T of the output (caller supplied)
+    uint32_t *amax_out;     // running max |h| as FP32 bits (atomicMax), or null
 };
 
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
@@ -148,6 +152,11 @@ sol_status_t launch_pair_bf16(const void *x, const void *w, const void *bias, vo
 sol_status_t launch_pair_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
                                const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
                                int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev);
+sol_status_t launch_pair256_nvfp4_quant_out(const void *xq, const void *xsf, const float *xts, const void *wq,
+                                            const void *wsf, const float *wts, const void *bias, int act,
+                                            const float *ts_out, void *hq, void *hsf, uint32_t *amax_out,
+                                            int64_t M, int64_t N, int64_t K, cudaStream_t stream,
+                                            const DeviceInfo *dev);
 sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
                                   const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
                                   int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev);

@@ -20,6 +20,7 @@
 // ~100 cycles, so the copies stay off the MMA thread); 14 = TMA producer (scales).
 // No multicast loads; every mbarrier wait is bounded.
 #include "gemm_common.cuh"
+#include "quant_math.cuh"
 
 namespace sol {
 namespace gemm {
@@ -84,6 +85,88 @@ __device__ __forceinline__ void epilogue_store(const CUtensorMap *tm_y, const Pa
     }
 }
 
+// Output modes of the kernel: BF16 Y, or Y passed through an activation and quantized for the next
+// linear (packed E2M1 + E4M3 block scales along N, with a caller-supplied tensor scale).
+enum : int { kOutBf16 = 0, kOutQuant = 1, kOutQuantGelu = 2 };
+
+// tanh-form GELU, 0.5 y (1 + tanh(u)), u = sqrt(2/pi) y (1 + 0.044715 y^2), with the hardware tanh
+// (one special-function op per element; the epilogue is bound by that unit, and the exact form
+// y / (1 + exp(-2u)) needs two).  tanh.approx is good to ~2^-11, far inside the BF16 rounding and
+// the FP4 grid that follow.
+__device__ __forceinline__ float gelu_tanh(float y) {
+    const float u = y * fmaf(0.79788456080286536f * 0.044715f, y * y, 0.79788456080286536f);
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+    const float hy = 0.5f * y;
+    return fmaf(hy, t, hy);
+}
+
+// The same 64-column chunk, but leaving as the next linear's quantized activations: h = bf16(act(
+// fma(acc, alpha, bias))), then per 16 columns the block scale and sixteen nibbles in the
+// quantizer's FP32 sequence.  A row's 64 columns are 32 bytes of nibbles (staged, one TMA store
+// of 32 rows x 32 bytes per chunk) and the four scale bytes of one (row, k-chunk) slot of the
+// chunked scale layout (one 4-byte store).  `amax2` collects max|h| per BF16 half.
+template <int kOut>
+__device__ __forceinline__ void epilogue_quant_store(const CUtensorMap *tm_q, const Params &p, const uint32_t (&lo)[32],
+                                                     const uint32_t (&hi)[32], int m0, int quad_in_tile, int row_tile,
+                                                     int nc, float alpha, float Tq, float c6T, uint32_t sbuf,
+                                                     uint32_t sbias, int lane, uint32_t &amax2) {
+    if (lane == 0) ptx::tma_store_wait_read<0>();
+    __syncwarp();
+    uint32_t sfw = 0;
+#pragma unroll
+    for (int blk = 0; blk < 4; ++blk) {
+        uint32_t hw[8];  // sixteen BF16 values of h
+        uint32_t bm = 0;
+#pragma unroll
+        for (int g2 = 0; g2 < 2; ++g2) {
+            const int g = blk * 2 + g2;
+            uint32_t bw[4];
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(bw[0]), "=r"(bw[1]), "=r"(bw[2]), "=r"(bw[3])
+                         : "r"(sbias + g * 16));
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t a0 = g < 4 ? lo[g * 8 + 2 * e] : hi[(g - 4) * 8 + 2 * e];
+                const uint32_t a1 = g < 4 ? lo[g * 8 + 2 * e + 1] : hi[(g - 4) * 8 + 2 * e + 1];
+                float y0 = fmaf(__uint_as_float(a0), alpha, __uint_as_float(bw[e] << 16));
+                float y1 = fmaf(__uint_as_float(a1), alpha, __uint_as_float(bw[e] & 0xFFFF0000u));
+                if (kOut == kOutQuantGelu) {
+                    y0 = gelu_tanh(y0);
+                    y1 = gelu_tanh(y1);
+                }
+                __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
+                const uint32_t w = *reinterpret_cast<uint32_t *>(&pk);
+                hw[g2 * 4 + e] = w;
+                bm = qmath::absmax2(bm, w);
+            }
+        }
+        amax2 = qmath::absmax2(amax2, bm);
+        bm &= 0x7FFF7FFFu;
+        const float a = __uint_as_float(max(bm & 0xFFFFu, bm >> 16) << 16);
+        float rcp;
+        const uint32_t sb = qmath::block_scale(a, c6T, Tq, rcp);
+        sfw |= sb << (8 * blk);
+        const uint32_t q0 = qmath::quantize8(hw[0], hw[1], hw[2], hw[3], rcp);
+        const uint32_t q1 = qmath::quantize8(hw[4], hw[5], hw[6], hw[7], rcp);
+        asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sbuf + lane * 32 + blk * 8), "r"(q0), "r"(q1) : "memory");
+    }
+    const bool unit_ok = nc < p.N && !(kTuning && (p.dbg & kDbgNoStore));
+    if (unit_ok && row_tile * 128 < p.M) {
+        // rows past M inside the last 128-row chunk are padding and read as 0
+        if (m0 + lane >= p.M) sfw = 0;
+        const int64_t chunk = static_cast<int64_t>(row_tile) * (p.N >> 6) + (nc >> 6);
+        *reinterpret_cast<uint32_t *>(p.sf_out + chunk * 512 + lane * 16 + quad_in_tile * 4) = sfw;
+    }
+    ptx::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        if (unit_ok && m0 < p.M) ptx::tma_store_2d(tm_q, nc >> 1, m0, sbuf);
+        ptx::tma_store_commit();
+    }
+}
+
+template <int kOut>
 __global__ void __launch_bounds__(kThreadsFp4, 1)
 gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                      const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_sfa,
@@ -353,10 +436,14 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         const uint32_t sbuf = epi_base + e * kEpiBufBytes;
         const uint32_t sbias = bias_base + e * 256;
         const float alpha = __fmul_rn(__ldcg(p.ts_a), __ldcg(p.ts_b));
+        const float Tq = kOut != kOutBf16 ? __ldcg(p.ts_out) : 1.0f;
+        const float c6T = __fmul_rn(6.0f, Tq);
+        uint32_t amax2 = 0;
         for (int t = pair, it = 0; t < total_tiles; t += num_pairs, ++it) {
             int mt, nt;
             tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
             const int m0 = mt * 2 * kBM + static_cast<int>(rank) * kBM + quad * 32, n0 = nt * kBN;
+            const int row_tile = mt * 2 + static_cast<int>(rank);
             const int x = it & 1;
             // 64-column units of the accumulator.  A (base 0) shares its columns [96,256) with the next
             // tile: units 2, 3 and the upper half of unit 1; B (base 96) its columns [0,160): units 0, 1 and
@@ -402,19 +489,38 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(ovl_bar);
             if (kTuning && (p.dbg & kDbgTrace) && warp == 2) SOL_TRACE(10, it);
-            epilogue_store(&tm_y, p, a_lo, a_hi, m0, n0 + first * 64, alpha, sbuf, sbias, lane);
+            if (kOut == kOutBf16)
+                epilogue_store(&tm_y, p, a_lo, a_hi, m0, n0 + first * 64, alpha, sbuf, sbias, lane);
+            else
+                epilogue_quant_store<kOut>(&tm_y, p, a_lo, a_hi, m0, quad, row_tile, n0 + first * 64, alpha, Tq, c6T,
+                                           sbuf, sbias, lane, amax2);
             if (early) ptx::tmem_ld_32x32(t2 + shared_half, b_sh);
             ptx::tmem_ld_32x32(t2 + (shared_half ^ 32u), b_ot);
             ptx::tmem_ld_wait();
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(done_bar);
-            if (x == 0)  // b_sh is the upper half
-                epilogue_store(&tm_y, p, b_ot, b_sh, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
-            else
-                epilogue_store(&tm_y, p, b_sh, b_ot, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
+            if (kOut == kOutBf16) {
+                if (x == 0)  // b_sh is the upper half
+                    epilogue_store(&tm_y, p, b_ot, b_sh, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
+                else
+                    epilogue_store(&tm_y, p, b_sh, b_ot, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
+            } else {
+                if (x == 0)
+                    epilogue_quant_store<kOut>(&tm_y, p, b_ot, b_sh, m0, quad, row_tile, n0 + second * 64, alpha, Tq,
+                                               c6T, sbuf, sbias + 128, lane, amax2);
+                else
+                    epilogue_quant_store<kOut>(&tm_y, p, b_sh, b_ot, m0, quad, row_tile, n0 + second * 64, alpha, Tq,
+                                               c6T, sbuf, sbias + 128, lane, amax2);
+            }
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();
+        if (kOut != kOutBf16 && p.amax_out != nullptr) {
+            amax2 &= 0x7FFF7FFFu;
+            uint32_t m = max(amax2 & 0xFFFFu, amax2 >> 16);
+            m = __reduce_max_sync(0xFFFFFFFFu, m);
+            if (lane == 0 && m) atomicMax(p.amax_out, m << 16);
+        }
     }
 
     // ---------------------------------------------------------------- teardown
@@ -430,20 +536,27 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
 
 }  // namespace
 
-sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
-                                  const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
-                                  int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev) {
+namespace {
+
+sol_status_t launch_pair256(int out_mode, const void *xq, const void *xsf, const float *xts, const void *wq,
+                            const void *wsf, const float *wts, const void *bias, void *y, int64_t ldy,
+                            const float *ts_out, void *hsf, uint32_t *amax_out, int64_t M, int64_t N, int64_t K,
+                            cudaStream_t stream, const DeviceInfo *dev) {
     const uint64_t chunks_k = static_cast<uint64_t>(ceil_div(K, 64));
     CUtensorMap tm_a, tm_b, tm_y, tm_sfa, tm_sfb;
-    if (!make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, xq, K / 2, M, K / 2, 128, kBM,
-                      CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, wq, K / 2, N, K / 2, 128, kBN / 2,
-                      CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, N, M, ldy * 2, 64, 32,
-                      CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_tmap_sf(&tm_sfa, xsf, chunks_k, static_cast<uint64_t>(ceil_div(M, 128)), 1) ||
-        !make_tmap_sf(&tm_sfb, wsf, chunks_k, static_cast<uint64_t>(ceil_div(N, 128)), 2))
-        return SOL_ERR_CUDA;
+    bool ok = make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, xq, K / 2, M, K / 2, 128, kBM,
+                           CU_TENSOR_MAP_SWIZZLE_128B) &&
+              make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, wq, K / 2, N, K / 2, 128, kBN / 2,
+                           CU_TENSOR_MAP_SWIZZLE_128B) &&
+              make_tmap_sf(&tm_sfa, xsf, chunks_k, static_cast<uint64_t>(ceil_div(M, 128)), 1) &&
+              make_tmap_sf(&tm_sfb, wsf, chunks_k, static_cast<uint64_t>(ceil_div(N, 128)), 2);
+    if (out_mode == kOutBf16)
+        ok = ok && make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, N, M, ldy * 2, 64, 32,
+                                CU_TENSOR_MAP_SWIZZLE_128B);
+    else  // packed nibbles [M, N/2]: boxes of 32 rows x 32 bytes (64 columns)
+        ok = ok && make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, y, N / 2, M, N / 2, 32, 32,
+                                CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (!ok) return SOL_ERR_CUDA;
     Params p{};
     p.sfa = static_cast<const uint8_t *>(xsf);
     p.sfb = static_cast<const uint8_t *>(wsf);
@@ -454,15 +567,19 @@ sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *
     p.M = static_cast<int>(M);
     p.N = static_cast<int>(N);
     p.K = static_cast<int>(K);
+    p.sf_out = static_cast<uint8_t *>(hsf);
+    p.ts_out = ts_out;
+    p.amax_out = amax_out;
 #ifdef SOL_TUNING
     if (const char *e = getenv("SOL_DBG")) p.dbg = static_cast<uint32_t>(atoi(e));
 #endif
-    static bool configured[64] = {};
-    if (dev->device < 64 && !configured[dev->device]) {
-        if (cudaFuncSetAttribute(gemm_pair_fp4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
-            cudaSuccess)
+    auto kern = out_mode == kOutBf16 ? gemm_pair_fp4_kernel<kOutBf16>
+                : out_mode == kOutQuant ? gemm_pair_fp4_kernel<kOutQuant> : gemm_pair_fp4_kernel<kOutQuantGelu>;
+    static bool configured[3][64] = {};
+    if (dev->device < 64 && !configured[out_mode][dev->device]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return SOL_ERR_CUDA;
-        configured[dev->device] = true;
+        configured[out_mode][dev->device] = true;
     }
     p.m_tiles = static_cast<int>(ceil_div(p.M, 2 * kBM));
     p.n_tiles = static_cast<int>(ceil_div(p.N, kBN));
@@ -483,11 +600,29 @@ sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, gemm_pair_fp4_kernel, tm_a, tm_b, tm_y, tm_sfa, tm_sfb, p) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_y, tm_sfa, tm_sfb, p) != cudaSuccess) {
         cudaGetLastError();
         return SOL_ERR_CUDA;
     }
     return SOL_OK;
+}
+
+}  // namespace
+
+sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
+                                  const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
+                                  int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev) {
+    return launch_pair256(kOutBf16, xq, xsf, xts, wq, wsf, wts, bias, y, ldy, nullptr, nullptr, nullptr, M, N, K,
+                          stream, dev);
+}
+
+sol_status_t launch_pair256_nvfp4_quant_out(const void *xq, const void *xsf, const float *xts, const void *wq,
+                                            const void *wsf, const float *wts, const void *bias, int act,
+                                            const float *ts_out, void *hq, void *hsf, uint32_t *amax_out,
+                                            int64_t M, int64_t N, int64_t K, cudaStream_t stream,
+                                            const DeviceInfo *dev) {
+    return launch_pair256(act == 1 ? kOutQuantGelu : kOutQuant, xq, xsf, xts, wq, wsf, wts, bias, hq, 0, ts_out, hsf,
+                          amax_out, M, N, K, stream, dev);
 }
 
 }  // namespace gemm

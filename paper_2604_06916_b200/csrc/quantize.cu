@@ -4,6 +4,7 @@
 // Both kernels are streaming codecs bound by HBM bandwidth: 16-byte loads, many loads in
 // flight per thread, packed 8-byte nibble stores, scale bytes staged in shared memory and
 // written as whole 512-byte chunks of the layout the tensor core consumes.
+#include "quant_math.cuh"
 #include "sol_internal.h"
 
 namespace sol {
@@ -15,12 +16,12 @@ constexpr int kTileK = 256;        // elements along K per block = 4 scale chunk
 constexpr int kBlocksPerThread = kTileRows * (kTileK / 16) / kQuantThreads;  // 8 scale blocks of 16 elements
 constexpr int kBatch = 4;          // scale blocks (2 x 16-byte loads each) in flight per thread
 
-// max(|a|, |b|) per BF16 half (the sign bits of the result are garbage and masked off later)
-__device__ __forceinline__ uint32_t absmax2(uint32_t a, uint32_t b) {
-    uint32_t d;
-    asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
-}
+using qmath::absmax2;
+using qmath::bf16_hi;
+using qmath::bf16_lo;
+using qmath::e4m3_to_f32;
+using qmath::f32_to_e4m3_sat;
+using qmath::pack_e2m1x8;
 
 __device__ __forceinline__ uint32_t abs_max_bits(const uint4 &v) {
     // per-halfword max of |bf16| bit patterns (magnitudes order like unsigned integers)
@@ -34,33 +35,6 @@ __device__ __forceinline__ uint32_t abs_max_bits(const uint4 &u, const uint4 &v)
     return max(m & 0xFFFFu, m >> 16);
 }
 
-__device__ __forceinline__ uint32_t f32_to_e4m3_sat(float v) {
-    uint16_t packed;
-    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(packed) : "f"(0.0f), "f"(v));
-    return packed & 0xFFu;
-}
-
-__device__ __forceinline__ float e4m3_to_f32(uint32_t code) {
-    uint32_t e = (code >> 3) & 15u, m = code & 7u;
-    if (e == 0) return __uint2float_rn(m) * 0x1p-9f;
-    return __uint_as_float(((e + 120u) << 23) | (m << 20));
-}
-
-// Eight FP32 values -> eight E2M1 nibbles (element 0 in the lowest nibble).
-__device__ __forceinline__ uint32_t pack_e2m1x8(float y0, float y1, float y2, float y3, float y4,
-                                                float y5, float y6, float y7) {
-    uint32_t out;
-    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
-        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
-        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
-        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
-        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
-        "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
-        : "=r"(out)
-        : "f"(y0), "f"(y1), "f"(y2), "f"(y3), "f"(y4), "f"(y5), "f"(y6), "f"(y7));
-    return out;
-}
-
 // Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
 // start while its predecessor in the stream is still draining; it must not touch global memory
 // before grid_dependency_wait() returns (a no-op when there is nothing to wait for).
@@ -71,13 +45,8 @@ __device__ __forceinline__ float tensor_scale_from_amax(float a) {
     return (a == 0.0f) ? 1.0f : __fdiv_rn(a, 2688.0f);
 }
 
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
-
 __device__ __forceinline__ uint32_t quantize8(const uint4 &v, float rcp) {
-    return pack_e2m1x8(__fmul_rn(bf16_lo(v.x), rcp), __fmul_rn(bf16_hi(v.x), rcp), __fmul_rn(bf16_lo(v.y), rcp),
-                       __fmul_rn(bf16_hi(v.y), rcp), __fmul_rn(bf16_lo(v.z), rcp), __fmul_rn(bf16_hi(v.z), rcp),
-                       __fmul_rn(bf16_lo(v.w), rcp), __fmul_rn(bf16_hi(v.w), rcp));
+    return qmath::quantize8(v.x, v.y, v.z, v.w, rcp);
 }
 
 // One block quantizes a 128-row x 256-element tile.  A thread owns whole scale blocks (16

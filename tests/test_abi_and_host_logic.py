@@ -88,6 +88,24 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.nvfp4_quantize_linear(p, 64, p, p, p, None, p, 4, 8, 64, 8, p + 16, 1 << 20, None) == ALIGN
     assert L.nvfp4_quantize_linear_static(p, 4096, p, p, p, None, p, 1 << 20, 8, 4096, 8, None) == WS
     assert L.nvfp4_quantize_linear_static(None, 64, p, p, p, None, p, 4, 8, 64, 8, None) == NULLP
+    # weight refresh
+    assert L.nvfp4_requantize_lora(p, 64, p, 64, p, 32, 8, 64, 32, 2.0, None, p, p, p, 1, None) == NULLP
+    assert L.nvfp4_requantize_lora(p, 64, p, 64, p, 32, 8, 64, 65, 2.0, p, p, p, p, 1, None) == SHAPE   # rank > 64
+    assert L.nvfp4_requantize_lora(p, 64, p, 64, p, 16, 8, 64, 32, 2.0, p, p, p, p, 1, None) == SHAPE   # ldb < r
+    assert L.nvfp4_requantize_lora(p, 64, p, 64, p + 1, 32, 8, 64, 32, 2.0, p, p, p, p, 1, None) == ALIGN
+    assert L.nvfp4_requantize_lora(p, 64, p, 64, p, 32, 8, 64, 32, 2.0, p, p, p, p, 7, None) == LAYOUT
+    lst = (ctypes.c_void_p * 2)(p, p)
+    bad = (ctypes.c_void_p * 2)(p, None)
+    assert L.nvfp4_requantize_lora_batch(0, None, None, None, None, None, None, 8, 64, 32, 2.0, p, 1, 1, None) == 0
+    assert L.nvfp4_requantize_lora_batch(2, lst, lst, lst, lst, lst, None, 8, 64, 32, 2.0, p, 1, 1, None) == NULLP
+    assert L.nvfp4_requantize_lora_batch(2, lst, bad, lst, lst, lst, lst, 8, 64, 32, 2.0, p, 1, 1, None) == NULLP
+    assert L.nvfp4_requantize_lora_batch(2, lst, lst, lst, lst, lst, lst, 8, 64, 32, 2.0, p, 0, 1, None) == SHAPE
+    assert L.nvfp4_requantize_lora_batch(-1, lst, lst, lst, lst, lst, lst, 8, 64, 32, 2.0, p, 1, 1, None) == SHAPE
+    # linear with quantized output
+    assert L.nvfp4_linear_quantized_out(p, p, p, p, p, p, None, 0, None, p, p, None, 4, 64, 64, None) == NULLP
+    assert L.nvfp4_linear_quantized_out(p, p, p, p, p, p, None, 0, p, p, p, None, 4, 96, 64, None) == SHAPE   # N % 64
+    assert L.nvfp4_linear_quantized_out(p, p, p, p, p, p, None, 5, p, p, p, None, 4, 64, 64, None) == LAYOUT  # activation
+    assert L.nvfp4_linear_quantized_out(p, p, p, p, p, p, None, 0, p, p + 8, p, None, 4, 64, 64, None) == ALIGN
 
 
 def test_binding_refuses_to_run_without_the_library(tmp_path):
