@@ -506,6 +506,34 @@ def run_only(args):
         B.sol_last_device_status()
         print(json.dumps({"only": "weight_refresh", "matrices": 8, "us_per_matrix": 1e3 * sum(times) / len(times) / 8}))
         return
+    if args.only == "mlp_pair":
+        # FLUX feed-forward pair with the intermediate kept in NVFP4 (GELU in the first GEMM's epilogue)
+        cfg = workloads.CONFIGS[args.workload]
+        names = [l.name for l in cfg.layers]
+        i1, i2 = names.index("d_mlp_in"), names.index("d_mlp_out")
+        M = args.rows if args.rows > 0 else cfg.layers[i1].M
+        X, W1, b1 = workloads.make_layer(cfg, i1, "cuda", M=M)
+        _, W2, b2 = workloads.make_layer(cfg, i2, "cuda", M=128)
+        w1 = B.nvfp4_quantize_weight(W1)
+        w2 = B.nvfp4_quantize_weight(W2)
+        xts = B.sol_amax_bf16(X)
+        xq, xsf = B.nvfp4_quantize(X, xts)
+        t_out = torch.full((1,), 0.01, dtype=torch.float32, device="cuda")
+        amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+        Y2 = torch.empty((M, W2.shape[0]), dtype=torch.bfloat16, device="cuda")
+        times = []
+        for it in range(args.warmup + args.steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            hq, hsf = B.nvfp4_linear_quantized_out(xq, xsf, xts, *w1, b1, B.ACT_GELU_TANH, t_out, amax_out=amax)
+            B.nvfp4_linear(hq, hsf, t_out, *w2, b2, out=Y2)
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                times.append(e0.elapsed_time(e1))
+        B.sol_last_device_status()
+        print(json.dumps({"only": "mlp_pair", "M": M, "ms": sum(times) / len(times)}))
+        return
     cfg = workloads.CONFIGS[args.workload]
     index = [l.name for l in cfg.layers].index(args.only)
     l = cfg.layers[index]
@@ -536,7 +564,7 @@ def run_only(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh'")
+    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair'")
     ap.add_argument("--rows", type=int, default=0, help="profile mode: override M")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
