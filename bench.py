@@ -396,6 +396,21 @@ def run_ours(args):
                             "counted; fused = nvfp4_linear_quantized_out (GELU, calibrated T) feeding nvfp4_linear"}
         del xq, xsf, hq, hsf
 
+    # ---- stage-1 selection and rank metrics at the paper's sizes (48 prompts per epoch, N = 96, K = 24):
+    # two launches of one block per prompt, a few microseconds each (launch latency, not throughput)
+    selection = None
+    if world == 1 and not args.lean:
+        gen = torch.Generator(device=dev).manual_seed(123)
+        r_ref = torch.randn(48, 96, generator=gen, device=dev)
+        r_proxy = (r_ref + 0.25 * torch.randn(48, 96, generator=gen, device=dev)).contiguous()
+        seeds = torch.randint(0, 2 ** 62, (48, 96), device=dev, dtype=torch.int64, generator=gen)
+        t_sel = loop_ms(lambda: B.solrl_select_contrastive(r_proxy, 24, seeds))
+        t_rank = loop_ms(lambda: B.solrl_rank_consistency(r_ref, r_proxy, 4))
+        _, m = B.solrl_rank_consistency(r_ref, r_proxy, 4)
+        selection = {"prompts": 48, "candidates": 96, "kept": 24, "select_us": t_sel * 1e3, "rank_metrics_us": t_rank * 1e3,
+                     "synthetic_mean_tau_rho_top4_bottom4": [round(float(x), 4) for x in m.mean(dim=0).tolist()],
+                     "note": "includes the Python binding's output allocation; synthetic proxy = reference + N(0, 0.25^2)"}
+
     # ---- end to end: pinned HOST activations in, HOST outputs back, copies inside the timed region,
     # through the host-buffer entry point of the C ABI, all six layers per step
     host_x = {}
@@ -467,7 +482,7 @@ def run_ours(args):
                                "traffic": int(NCU_TRAFFIC_RATIO["quantize"] * quant_bytes),
                                "peak_source": peak_src},
         "stack_tflops_caller_supplied_scale": world * flops / (ms_static / args.steps * 1e-3) / 1e12,
-        "weight_refresh": refresh, "mlp_pair_nvfp4_intermediate": mlp_pair,
+        "weight_refresh": refresh, "mlp_pair_nvfp4_intermediate": mlp_pair, "stage1_selection": selection,
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": kernels_per_layer * len(layers) * args.steps,
         "bf16_vs_torch_matmul_note": "MEASURED_PEAKS bf16 (torch.matmul 8192^3): %.0f burst / %.0f sustained TF" % (

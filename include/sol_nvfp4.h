@@ -222,6 +222,34 @@ sol_status_t nvfp4_quantize_linear_host(const void *x_host, int64_t ldx, const v
                                         void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Stage-1 selection (Section 3.4; Section 4.1 "Rollout Generation": N = 96 candidates per prompt,
+ * the 12 best and 12 worst kept, their initial noises preserved) and the group-standardised
+ * advantages of the GRPO equation in Section 2, A_i = (R_i - mean) / population std.
+ *   rewards        [P, N] FP32 proxy rewards, finite; N <= 4096
+ *   seeds          [P, N] 64-bit noise seeds (nullable when seeds_out is null)
+ *   idx_out        [P, K] int32: K/2 best candidates in descending order of reward, then the K/2
+ *                  worst starting from the lowest; among equal rewards the lower index ranks higher
+ *   seeds_out      [P, K] the selected candidates' seeds (nullable)
+ *   advantages_out [P, N] FP32 (nullable); statistics in FP64; all zeros when the std is 0
+ *   K even, 0 < K <= N.  One block per prompt; indices and seeds are exact.
+ */
+sol_status_t solrl_select_contrastive(const float *rewards, const uint64_t *seeds, int64_t P, int64_t N, int64_t K,
+                                      int32_t *idx_out, uint64_t *seeds_out, float *advantages_out, void *stream);
+
+/*
+ * Rank consistency between reference and proxy rewards (appendix "Group-Relative Ranking
+ * Consistency"): per prompt
+ *   counts_out  [P, 4] int64: concordant minus discordant pairs (ties count 0), sum of squared
+ *               rank differences (ordinal ranks, ties to the lower index), candidates in both top-k
+ *               sets, candidates in both bottom-k sets -- all exact
+ *   metrics_out [P, 4] FP32 (nullable): Kendall tau-a = count / (N(N-1)/2), Spearman rho =
+ *               1 - 6 sum d^2 / (N(N^2-1)), top-k and bottom-k match rates
+ *   2 <= N <= 2048, 0 < k <= N.
+ */
+sol_status_t solrl_rank_consistency(const float *rewards_ref, const float *rewards_proxy, int64_t P, int64_t N,
+                                    int64_t k, int64_t *counts_out, float *metrics_out, void *stream);
+
+/*
  * (No counterpart in the paper: an addition for callers that cannot allocate device memory.)
  *
  * Same computation and result as nvfp4_quantize_linear, but without a workspace argument: the

@@ -23,6 +23,7 @@ EXPORTS = [
     "nvfp4_linear", "bf16_linear", "nvfp4_quantize_linear", "sol_last_device_status",
     "sol_nvfp4_static_scratch_bytes", "nvfp4_quantize_linear_static", "nvfp4_quantize_linear_host",
     "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch", "nvfp4_linear_quantized_out",
+    "solrl_select_contrastive", "solrl_rank_consistency",
 ]
 
 _lib = None
@@ -73,6 +74,10 @@ def lib() -> ctypes.CDLL:
                                               i32, vp]
     L.nvfp4_linear_quantized_out.restype = i32
     L.nvfp4_linear_quantized_out.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, i64, i64, i64, vp]
+    L.solrl_select_contrastive.restype = i32
+    L.solrl_select_contrastive.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, vp]
+    L.solrl_rank_consistency.restype = i32
+    L.solrl_rank_consistency.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -235,6 +240,39 @@ def nvfp4_linear(xq, xsf, x_tscale, wq, wsf, w_tscale, bias=None, out: torch.Ten
 
 
 ACT_NONE, ACT_GELU_TANH = 0, 1
+
+
+def solrl_select_contrastive(rewards: torch.Tensor, K: int, seeds: torch.Tensor | None = None,
+                             with_advantages: bool = True):
+    """[P, N] FP32 rewards -> (indices [P, K] int32, selected seeds or None, advantages [P, N] or None)."""
+    if rewards.dtype != torch.float32 or rewards.dim() != 2 or not rewards.is_contiguous():
+        raise ValueError("rewards must be a dense 2-D float32 tensor")
+    P, N = rewards.shape
+    idx = torch.empty((P, K), dtype=torch.int32, device=rewards.device)
+    sel = None
+    if seeds is not None:
+        if seeds.dtype != torch.int64 or tuple(seeds.shape) != (P, N) or not seeds.is_contiguous():
+            raise ValueError("seeds must be a dense [P, N] int64 tensor")
+        sel = torch.empty((P, K), dtype=torch.int64, device=rewards.device)
+    adv = torch.empty_like(rewards) if with_advantages else None
+    _check(lib().solrl_select_contrastive(_ptr(rewards), _ptr(seeds), P, N, K, _ptr(idx), _ptr(sel), _ptr(adv),
+                                          _stream()), "solrl_select_contrastive")
+    return idx, sel, adv
+
+
+def solrl_rank_consistency(ref: torch.Tensor, proxy: torch.Tensor, k: int):
+    """Per prompt: exact counts [P, 4] int64 and (tau, rho, top-k match, bottom-k match) [P, 4] FP32."""
+    for t in (ref, proxy):
+        if t.dtype != torch.float32 or t.dim() != 2 or not t.is_contiguous():
+            raise ValueError("rewards must be dense 2-D float32 tensors")
+    if ref.shape != proxy.shape:
+        raise ValueError("shapes differ")
+    P, N = ref.shape
+    counts = torch.empty((P, 4), dtype=torch.int64, device=ref.device)
+    metrics = torch.empty((P, 4), dtype=torch.float32, device=ref.device)
+    _check(lib().solrl_rank_consistency(_ptr(ref), _ptr(proxy), P, N, k, _ptr(counts), _ptr(metrics), _stream()),
+           "solrl_rank_consistency")
+    return counts, metrics
 
 
 def nvfp4_linear_quantized_out(xq, xsf, x_tscale, wq, wsf, w_tscale, bias, activation: int, out_tscale,

@@ -335,6 +335,37 @@ sol_status_t nvfp4_linear_quantized_out(const void *xq, const void *xsf, const f
                                                 static_cast<cudaStream_t>(stream), dev);
 }
 
+sol_status_t solrl_select_contrastive(const float *rewards, const uint64_t *seeds, int64_t P, int64_t N, int64_t K,
+                                      int32_t *idx_out, uint64_t *seeds_out, float *advantages_out, void *stream) {
+    if (rewards == nullptr || idx_out == nullptr || (seeds_out != nullptr && seeds == nullptr)) return SOL_ERR_NULL_POINTER;
+    if (P <= 0 || P > 0x7FFFFFFF || N <= 0 || N > selection_max_candidates() || K <= 0 || K % 2 != 0 || K > N)
+        return SOL_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(rewards) & 3u) || (reinterpret_cast<uintptr_t>(idx_out) & 3u) ||
+        (reinterpret_cast<uintptr_t>(seeds) & 7u) || (reinterpret_cast<uintptr_t>(seeds_out) & 7u) ||
+        (reinterpret_cast<uintptr_t>(advantages_out) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_select_contrastive(rewards, seeds, P, N, K, idx_out, seeds_out, advantages_out,
+                                     static_cast<cudaStream_t>(stream));
+}
+
+sol_status_t solrl_rank_consistency(const float *rewards_ref, const float *rewards_proxy, int64_t P, int64_t N,
+                                    int64_t k, int64_t *counts_out, float *metrics_out, void *stream) {
+    if (rewards_ref == nullptr || rewards_proxy == nullptr || counts_out == nullptr) return SOL_ERR_NULL_POINTER;
+    if (P <= 0 || P > 0x7FFFFFFF || N < 2 || 2 * N > selection_max_candidates() || k <= 0 || k > N)
+        return SOL_ERR_BAD_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(rewards_ref) & 3u) || (reinterpret_cast<uintptr_t>(rewards_proxy) & 3u) ||
+        (reinterpret_cast<uintptr_t>(counts_out) & 7u) || (reinterpret_cast<uintptr_t>(metrics_out) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_rank_consistency(rewards_ref, rewards_proxy, P, N, k, counts_out, metrics_out,
+                                   static_cast<cudaStream_t>(stream));
+}
+
 sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,
                                    const float *w_tscale, const void *bias_bf16, void *y_bf16, int64_t M,
                                    int64_t N, int64_t K, int64_t ldy, void *workspace, size_t workspace_bytes,

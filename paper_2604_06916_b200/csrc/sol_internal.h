@@ -67,6 +67,12 @@ sol_status_t launch_lora_merge(const MergeGroup &g, int count, int64_t ldw, int6
 sol_status_t launch_quantize_group(const QuantGroup &g, int count, int64_t rows, int64_t K, sol_sf_layout_t layout,
                                    cudaStream_t stream);
 int lora_max_rank();
+// Stage-1 selection and rank-consistency metrics (one block per prompt).
+sol_status_t launch_select_contrastive(const float *rewards, const uint64_t *seeds, int64_t P, int64_t N, int64_t K,
+                                       int32_t *idx_out, uint64_t *seeds_out, float *adv_out, cudaStream_t stream);
+sol_status_t launch_rank_consistency(const float *ref, const float *proxy, int64_t P, int64_t N, int64_t k,
+                                     int64_t *counts_out, float *metrics_out, cudaStream_t stream);
+int selection_max_candidates();
 sol_status_t launch_gemm_bf16(const void *x, const void *w, const void *bias, void *y, int64_t M,
                               int64_t N, int64_t K, int64_t ldx, int64_t ldw, int64_t ldy,
                               cudaStream_t stream, const DeviceInfo *dev);

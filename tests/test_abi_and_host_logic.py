@@ -101,6 +101,17 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.nvfp4_requantize_lora_batch(2, lst, bad, lst, lst, lst, lst, 8, 64, 32, 2.0, p, 1, 1, None) == NULLP
     assert L.nvfp4_requantize_lora_batch(2, lst, lst, lst, lst, lst, lst, 8, 64, 32, 2.0, p, 0, 1, None) == SHAPE
     assert L.nvfp4_requantize_lora_batch(-1, lst, lst, lst, lst, lst, lst, 8, 64, 32, 2.0, p, 1, 1, None) == SHAPE
+    # stage-1 selection and rank metrics
+    assert L.solrl_select_contrastive(None, None, 2, 8, 4, p, None, None, None) == NULLP
+    assert L.solrl_select_contrastive(p, None, 2, 8, 4, p, p, None, None) == NULLP      # seeds_out without seeds
+    assert L.solrl_select_contrastive(p, None, 2, 8, 5, p, None, None, None) == SHAPE   # odd K
+    assert L.solrl_select_contrastive(p, None, 2, 8, 10, p, None, None, None) == SHAPE  # K > N
+    assert L.solrl_select_contrastive(p, None, 2, 5000, 4, p, None, None, None) == SHAPE
+    assert L.solrl_select_contrastive(p + 2, None, 2, 8, 4, p, None, None, None) == ALIGN
+    assert L.solrl_rank_consistency(p, None, 2, 8, 4, p, None, None) == NULLP
+    assert L.solrl_rank_consistency(p, p, 2, 1, 1, p, None, None) == SHAPE
+    assert L.solrl_rank_consistency(p, p, 2, 8, 9, p, None, None) == SHAPE
+    assert L.solrl_rank_consistency(p, p, 2, 8, 4, p + 4, None, None) == ALIGN
     # linear with quantized output
     assert L.nvfp4_linear_quantized_out(p, p, p, p, p, p, None, 0, None, p, p, None, 4, 64, 64, None) == NULLP
     assert L.nvfp4_linear_quantized_out(p, p, p, p, p, p, None, 0, p, p, p, None, 4, 96, 64, None) == SHAPE   # N % 64
