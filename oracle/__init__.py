@@ -61,6 +61,14 @@ def _load():
     L.oracle_bf16_linear.argtypes = [u16p, i64, u16p, i64, u16p, i64, i64, i64p, i64, f64p]
     L.oracle_f64_to_bf16_array.restype, L.oracle_f64_to_bf16_array.argtypes = None, [f64p, i64, u16p]
     L.oracle_num_threads.restype, L.oracle_num_threads.argtypes = ctypes.c_int, []
+    L.oracle_e8m0_decode.restype, L.oracle_e8m0_decode.argtypes = ctypes.c_double, [ctypes.c_uint8]
+    L.oracle_mxfp4_quantize.restype, L.oracle_mxfp4_quantize.argtypes = None, [u16p, i64, i64, i64, u8p, u8p]
+    L.oracle_mx_sf_swizzled_offset.restype, L.oracle_mx_sf_swizzled_offset.argtypes = i64, [i64, i64, i64]
+    L.oracle_mx_sf_swizzled_bytes.restype, L.oracle_mx_sf_swizzled_bytes.argtypes = i64, [i64, i64]
+    L.oracle_mx_sf_swizzle.restype, L.oracle_mx_sf_swizzle.argtypes = None, [u8p, i64, i64, u8p]
+    L.oracle_mxfp4_dequantize.restype, L.oracle_mxfp4_dequantize.argtypes = None, [u8p, u8p, i64, i64, f64p]
+    L.oracle_mxfp4_linear.restype = ctypes.c_int
+    L.oracle_mxfp4_linear.argtypes = [u8p, u8p, u8p, u8p, u16p, i64, i64, i64p, i64, f64p]
     L.oracle_gelu_tanh.restype, L.oracle_gelu_tanh.argtypes = ctypes.c_double, [ctypes.c_double]
     L.oracle_gelu_tanh_array.restype, L.oracle_gelu_tanh_array.argtypes = None, [f64p, i64, f64p]
     L.oracle_lora_merge.restype = None
@@ -201,6 +209,62 @@ def bf16_linear(x_bits, w_bits, bias_bits=None, rows=None) -> np.ndarray:
                                     _p(Y, ctypes.c_double))
     if rc:
         raise MemoryError("oracle_bf16_linear")
+    del keep
+    return Y
+
+
+# ----------------------------------------------------------------- MXFP4
+def e8m0_decode(b: int) -> float:
+    return float(_load().oracle_e8m0_decode(int(b)))
+
+
+def mxfp4_quantize(x_bits: np.ndarray) -> tuple[np.ndarray, np.ndarray]:
+    """BF16 bits [rows, K] -> (packed nibbles [rows, K/2], E8M0 scales [rows, K/32])."""
+    x = _c(x_bits, np.uint16)
+    rows, K = x.shape
+    if K % 32:
+        raise ValueError("K must be a multiple of 32")
+    q = np.empty((rows, K // 2), np.uint8)
+    sf = np.empty((rows, K // 32), np.uint8)
+    _load().oracle_mxfp4_quantize(_p(x, ctypes.c_uint16), rows, K, K, _p(q, ctypes.c_uint8), _p(sf, ctypes.c_uint8))
+    return q, sf
+
+
+def mx_sf_swizzled_offset(r: int, kb: int, K: int) -> int:
+    return int(_load().oracle_mx_sf_swizzled_offset(r, kb, K))
+
+
+def mx_sf_swizzle(sf: np.ndarray, K: int) -> np.ndarray:
+    sf = _c(sf, np.uint8)
+    rows = sf.shape[0]
+    out = np.empty(int(_load().oracle_mx_sf_swizzled_bytes(rows, K)), np.uint8)
+    _load().oracle_mx_sf_swizzle(_p(sf, ctypes.c_uint8), rows, K, _p(out, ctypes.c_uint8))
+    return out
+
+
+def mxfp4_dequantize(q: np.ndarray, sf: np.ndarray) -> np.ndarray:
+    q, sf = _c(q, np.uint8), _c(sf, np.uint8)
+    rows, K = q.shape[0], q.shape[1] * 2
+    out = np.empty((rows, K), np.float64)
+    _load().oracle_mxfp4_dequantize(_p(q, ctypes.c_uint8), _p(sf, ctypes.c_uint8), rows, K, _p(out, ctypes.c_double))
+    return out
+
+
+def mxfp4_linear(qx, sfx, qw, sfw, bias_bits=None, rows=None) -> np.ndarray:
+    """Y = dequant(X) . dequant(W)^T + bias in FP64 for `rows` of X (all rows when None)."""
+    qx, sfx, qw, sfw = _c(qx, np.uint8), _c(sfx, np.uint8), _c(qw, np.uint8), _c(sfw, np.uint8)
+    M, K = qx.shape[0], qx.shape[1] * 2
+    N = qw.shape[0]
+    if qw.shape[1] * 2 != K:
+        raise ValueError("K mismatch")
+    keep, n_rows, rp = _rows(rows, M)
+    Y = np.empty((n_rows, N), np.float64)
+    b = _c(bias_bits, np.uint16) if bias_bits is not None else None
+    rc = _load().oracle_mxfp4_linear(_p(qx, ctypes.c_uint8), _p(sfx, ctypes.c_uint8), _p(qw, ctypes.c_uint8),
+                                     _p(sfw, ctypes.c_uint8), _p(b, ctypes.c_uint16) if b is not None else None,
+                                     N, K, rp, n_rows, _p(Y, ctypes.c_double))
+    if rc:
+        raise MemoryError("oracle_mxfp4_linear")
     del keep
     return Y
 

@@ -283,6 +283,100 @@ int oracle_bf16_linear(const uint16_t *x, int64_t ldx, const uint16_t *w, int64_
     return 0;
 }
 
+/* ------------------------------------------------------------------ MXFP4 (the other FP4 format of Section 2) */
+
+/* Section 2 names two block formats: NVFP4 above, and OCP MXFP4 -- 32 elements under one E8M0
+ * scale.  E8M0 is a bare biased exponent: byte b stands for 2^(b - 127) (0xFF is NaN, unused).
+ * Q(x) = S * Pi_FP4(x / S) with S a power of two and no tensor-level scale.  The reading taken for
+ * the scale is the OCP Microscaling rule: shared exponent = floor(log2(max|x|)) - 2 (2 = the
+ * exponent of E2M1's largest value 6 = 1.5 * 2^2), clamped to [-127, 127]; a block maximum in
+ * [4S, 8S) therefore has elements above 6S, which saturate.  Pi_FP4 is the same nearest-even,
+ * saturating projection as for NVFP4; x / S is exact (a power-of-two scaling). */
+double oracle_e8m0_decode(uint8_t b) { return ldexp(1.0, (int)b - 127); }
+
+void oracle_mxfp4_quantize(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, uint8_t *q, uint8_t *sf) {
+    const int64_t nb = K / 32;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t b = 0; b < nb; ++b) {
+            const uint16_t *xb = x + r * ld + b * 32;
+            double a = 0.0;
+            for (int k = 0; k < 32; ++k) {
+                double t = fabs((double)oracle_bf16_to_f32(xb[k]));
+                if (t > a) a = t;
+            }
+            int se = -127;
+            if (a > 0.0) {
+                int e;
+                (void)frexp(a, &e);      /* a in [2^(e-1), 2^e)  ->  floor(log2 a) = e - 1 */
+                se = (e - 1) - 2;
+                if (se < -127) se = -127;
+                if (se > 127) se = 127;
+            }
+            sf[r * nb + b] = (uint8_t)(se + 127);
+            for (int j = 0; j < 16; ++j) {
+                float y0 = (float)ldexp((double)oracle_bf16_to_f32(xb[2 * j]), -se);
+                float y1 = (float)ldexp((double)oracle_bf16_to_f32(xb[2 * j + 1]), -se);
+                q[r * (K / 2) + b * 16 + j] = (uint8_t)(oracle_e2m1_encode(y0) | (oracle_e2m1_encode(y1) << 4));
+            }
+        }
+    }
+}
+
+/* The same 512-byte chunks of 128 rows x 4 scales as for NVFP4; a chunk now spans 128 elements of K. */
+int64_t oracle_mx_sf_swizzled_offset(int64_t r, int64_t kb, int64_t K) {
+    int64_t chunks_k = (K / 32 + 3) / 4;
+    int64_t chunk = (r / 128) * chunks_k + kb / 4;
+    int64_t rr = r % 128;
+    return chunk * 512 + (rr % 32) * 16 + (rr / 32) * 4 + kb % 4;
+}
+
+int64_t oracle_mx_sf_swizzled_bytes(int64_t rows, int64_t K) {
+    return ((rows + 127) / 128) * ((K / 32 + 3) / 4) * 512;
+}
+
+void oracle_mx_sf_swizzle(const uint8_t *sf, int64_t rows, int64_t K, uint8_t *out) {
+    memset(out, 0, (size_t)oracle_mx_sf_swizzled_bytes(rows, K));
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t b = 0; b < K / 32; ++b)
+            out[oracle_mx_sf_swizzled_offset(r, b, K)] = sf[r * (K / 32) + b];
+}
+
+void oracle_mxfp4_dequantize(const uint8_t *q, const uint8_t *sf, int64_t rows, int64_t K, double *out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            uint8_t byte = q[r * (K / 2) + k / 2];
+            uint8_t code = (k & 1) ? (uint8_t)(byte >> 4) : (uint8_t)(byte & 0xF);
+            out[r * K + k] = oracle_e2m1_decode(code) * oracle_e8m0_decode(sf[r * (K / 32) + k / 32]);
+        }
+}
+
+static void matmul_nt_f64(const double *A, const double *B, const uint16_t *bias, int64_t n_rows, int64_t N,
+                          int64_t K, double *Y);
+
+/* MXFP4 linear: Y = dequant(X) . dequant(W)^T + bias in FP64 for the selected rows of X. */
+int oracle_mxfp4_linear(const uint8_t *q_x, const uint8_t *sf_x, const uint8_t *q_w, const uint8_t *sf_w,
+                        const uint16_t *bias, int64_t N, int64_t K, const int64_t *row_idx, int64_t n_rows,
+                        double *Y) {
+    double *A = (double *)malloc(sizeof(double) * (size_t)n_rows * (size_t)K);
+    double *B = (double *)malloc(sizeof(double) * (size_t)N * (size_t)K);
+    if (!A || !B) {
+        free(A);
+        free(B);
+        return 1;
+    }
+    for (int64_t i = 0; i < n_rows; ++i) {
+        int64_t r = row_idx ? row_idx[i] : i;
+        oracle_mxfp4_dequantize(q_x + r * (K / 2), sf_x + r * (K / 32), 1, K, A + i * K);
+    }
+    oracle_mxfp4_dequantize(q_w, sf_w, N, K, B);
+    matmul_nt_f64(A, B, bias, n_rows, N, K, Y);
+    free(A);
+    free(B);
+    return 0;
+}
+
 /* ------------------------------------------------------------------ activation between two linears */
 
 /* GELU in its tanh form, the activation of the DiT feed-forward blocks whose linears the rollout
