@@ -222,6 +222,27 @@ sol_status_t nvfp4_quantize_linear_host(const void *x_host, int64_t ldx, const v
                                         void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * MXFP4, the OCP format Section 2 sets beside NVFP4: 32 contiguous elements along K under one E8M0
+ * scale (a bare exponent: byte b = 2^(b-127)), no tensor-level scale.
+ *     scale = 2^(floor(log2 max|x|) - 2), exponent clamped to [-127, 127]; byte 0 for an all-zero block
+ *     nibble_k = E2M1_rne_sat(x_k / scale)    (the division is an exact power-of-two scaling)
+ * Storage: nibbles as for NVFP4; scales row-major [rows, K/32], or SOL_SF_SWIZZLED_128x4: the same
+ * 512-byte chunks of 128 rows x 4 scales (a chunk now spans 128 elements of K), chunk order
+ * [ceil(rows/128)][ceil(K/128)], padding 0.  sol_mxfp4_scale_bytes gives the buffer size.
+ */
+size_t sol_mxfp4_scale_bytes(int64_t rows, int64_t K, sol_sf_layout_t layout);
+sol_status_t mxfp4_quantize(const void *x_bf16, int64_t rows, int64_t K, int64_t ldx, void *q_out, void *sf_out,
+                            sol_sf_layout_t layout, void *stream);
+
+/*
+ * MXFP4 linear: Y[m,n] = bf16_rne( sum_b 2^(ex[m,b] + ew[n,b]) sum_{k in b} qx[m,k] qw[n,k] + bias[n] ),
+ * FP32 accumulation in the tensor core (kind::mxf4, two scales per row per K = 64 instruction).
+ * Operands as written by mxfp4_quantize with the chunked scale layout; otherwise as nvfp4_linear.
+ */
+sol_status_t mxfp4_linear(const void *xq, const void *xsf, const void *wq, const void *wsf, const void *bias_bf16,
+                          void *y_bf16, int64_t M, int64_t N, int64_t K, int64_t ldy, void *stream);
+
+/*
  * Stage-1 selection (Section 3.4; Section 4.1 "Rollout Generation": N = 96 candidates per prompt,
  * the 12 best and 12 worst kept, their initial noises preserved) and the group-standardised
  * advantages of the GRPO equation in Section 2, A_i = (R_i - mean) / population std.

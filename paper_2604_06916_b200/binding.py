@@ -23,7 +23,8 @@ EXPORTS = [
     "nvfp4_linear", "bf16_linear", "nvfp4_quantize_linear", "sol_last_device_status",
     "sol_nvfp4_static_scratch_bytes", "nvfp4_quantize_linear_static", "nvfp4_quantize_linear_host",
     "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch", "nvfp4_linear_quantized_out",
-    "solrl_select_contrastive", "solrl_rank_consistency",
+    "solrl_select_contrastive", "solrl_rank_consistency", "sol_mxfp4_scale_bytes", "mxfp4_quantize",
+    "mxfp4_linear",
 ]
 
 _lib = None
@@ -78,6 +79,9 @@ def lib() -> ctypes.CDLL:
     L.solrl_select_contrastive.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp, vp]
     L.solrl_rank_consistency.restype = i32
     L.solrl_rank_consistency.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
+    L.sol_mxfp4_scale_bytes.restype, L.sol_mxfp4_scale_bytes.argtypes = sz, [i64, i64, i32]
+    L.mxfp4_quantize.restype, L.mxfp4_quantize.argtypes = i32, [vp, i64, i64, i64, vp, vp, i32, vp]
+    L.mxfp4_linear.restype, L.mxfp4_linear.argtypes = i32, [vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -240,6 +244,36 @@ def nvfp4_linear(xq, xsf, x_tscale, wq, wsf, w_tscale, bias=None, out: torch.Ten
 
 
 ACT_NONE, ACT_GELU_TANH = 0, 1
+
+
+def mxfp4_scale_bytes(rows: int, K: int, layout: int = SF_SWIZZLED_128x4) -> int:
+    return int(lib().sol_mxfp4_scale_bytes(rows, K, layout))
+
+
+def mxfp4_quantize(x: torch.Tensor, layout: int = SF_SWIZZLED_128x4, out=None):
+    """BF16 [rows, K] -> (packed nibbles [rows, K/2], E8M0 scales in the given layout)."""
+    _need_2d_bf16(x, "x")
+    rows, K = x.shape
+    if out is None:
+        nbytes = mxfp4_scale_bytes(rows, K, layout)
+        if nbytes == 0:
+            raise ValueError("bad shape for mxfp4_quantize")
+        out = (torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device),
+               torch.empty(nbytes, dtype=torch.uint8, device=x.device))
+    q, sf = out
+    _check(lib().mxfp4_quantize(_ptr(x), rows, K, x.stride(0), _ptr(q), _ptr(sf), layout, _stream()), "mxfp4_quantize")
+    return q, sf
+
+
+def mxfp4_linear(xq, xsf, wq, wsf, bias=None, out: torch.Tensor | None = None):
+    """Y = dequant(X) . dequant(W)^T + bias in BF16 from MXFP4 operands (chunked scales)."""
+    M, K = xq.shape[0], xq.shape[1] * 2
+    N = wq.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=xq.device)
+    _check(lib().mxfp4_linear(_ptr(xq), _ptr(xsf), _ptr(wq), _ptr(wsf), _ptr(bias), _ptr(out), M, N, K, out.stride(0),
+                              _stream()), "mxfp4_linear")
+    return out
 
 
 def solrl_select_contrastive(rewards: torch.Tensor, K: int, seeds: torch.Tensor | None = None,

@@ -87,12 +87,12 @@ bool make_tmap_2d(CUtensorMap *out, CUtensorMapDataType dtype, uint32_t elem_byt
 }
 
 bool make_tmap_sf(CUtensorMap *out, const void *base, uint64_t chunks_k, uint64_t row_chunks,
-                  uint32_t box_row_chunks) {
+                  uint32_t box_row_chunks, uint32_t box_k_chunks) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
     cuuint64_t dims[3] = {128, chunks_k, row_chunks};
     cuuint64_t strides[2] = {512, 512 * chunks_k};
-    cuuint32_t box[3] = {128, 4, box_row_chunks};
+    cuuint32_t box[3] = {128, box_k_chunks, box_row_chunks};
     cuuint32_t estr[3] = {1, 1, 1};
     return fn(out, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -333,6 +333,40 @@ sol_status_t nvfp4_linear_quantized_out(const void *xq, const void *xsf, const f
                                                 activation == SOL_ACT_GELU_TANH ? 1 : 0, out_tscale, hq_out, hsf_out,
                                                 reinterpret_cast<uint32_t *>(amax_out), M, N, K,
                                                 static_cast<cudaStream_t>(stream), dev);
+}
+
+size_t sol_mxfp4_scale_bytes(int64_t rows, int64_t K, sol_sf_layout_t layout) {
+    if (!shape_ok(rows, K)) return 0;
+    if (layout == SOL_SF_ROW_MAJOR) return static_cast<size_t>(rows) * static_cast<size_t>(K / 32);
+    if (layout == SOL_SF_SWIZZLED_128x4)
+        return static_cast<size_t>(ceil_div(rows, 128)) * static_cast<size_t>(ceil_div(K, 128)) * 512;
+    return 0;
+}
+
+sol_status_t mxfp4_quantize(const void *x_bf16, int64_t rows, int64_t K, int64_t ldx, void *q_out, void *sf_out,
+                            sol_sf_layout_t layout, void *stream) {
+    if (x_bf16 == nullptr || q_out == nullptr || sf_out == nullptr) return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(rows, K) || ldx < K) return SOL_ERR_BAD_SHAPE;
+    if (layout != SOL_SF_ROW_MAJOR && layout != SOL_SF_SWIZZLED_128x4) return SOL_ERR_BAD_LAYOUT;
+    if (!aligned16(x_bf16) || !aligned16(q_out) || !aligned16(sf_out) || ldx % 8 != 0) return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_mxfp4_quantize(x_bf16, rows, K, ldx, q_out, sf_out, layout, static_cast<cudaStream_t>(stream));
+}
+
+sol_status_t mxfp4_linear(const void *xq, const void *xsf, const void *wq, const void *wsf, const void *bias_bf16,
+                          void *y_bf16, int64_t M, int64_t N, int64_t K, int64_t ldy, void *stream) {
+    if (xq == nullptr || xsf == nullptr || wq == nullptr || wsf == nullptr || y_bf16 == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    sol_status_t st = check_linear_common(bias_bf16, y_bf16, M, N, K, ldy);
+    if (st != SOL_OK) return st;
+    if (!aligned16(xq) || !aligned16(xsf) || !aligned16(wq) || !aligned16(wsf)) return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return gemm::launch_pair256_mxfp4(xq, xsf, wq, wsf, bias_bf16, y_bf16, M, N, K, ldy,
+                                      static_cast<cudaStream_t>(stream), dev);
 }
 
 sol_status_t solrl_select_contrastive(const float *rewards, const uint64_t *seeds, int64_t P, int64_t N, int64_t K,

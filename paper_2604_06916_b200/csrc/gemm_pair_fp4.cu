@@ -166,7 +166,9 @@ __device__ __forceinline__ void epilogue_quant_store(const CUtensorMap *tm_q, co
     }
 }
 
-template <int kOut>
+// kMx: MXFP4 operands (32-element blocks, E8M0 scales: a 512-byte scale chunk spans 128 elements of K,
+// so a k-tile has two chunks per 128 rows instead of four, and no tensor scales) -- BF16 output only.
+template <int kOut, bool kMx>
 __global__ void __launch_bounds__(kThreadsFp4, 1)
 gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                      const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_sfa,
@@ -196,6 +198,9 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     const int total_tiles = p.m_tiles * p.n_tiles;
     const int k_tiles = (p.K + kBK - 1) / kBK;
     const int tail_mmas = (p.K - (k_tiles - 1) * kBK + kMmaK - 1) / kMmaK;  // MMAs of the last k-tile (1..4)
+    constexpr int kSfChunksK = kMx ? 2 : 4;                  // scale chunks along K per stage and 128 rows
+    constexpr int kSfRowChunkBytes = kSfChunksK * 512;       // one 128-row chunk's scales of a stage
+    constexpr int kSfLoadBytes = 3 * kSfRowChunkBytes;       // A (one row chunk) + B (two)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -232,7 +237,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         const bool elected = ptx::elect_one();
         const uint32_t full0 = ptx::map_to_cta(full_bar(0), 0);  // the even CTA's barriers
         const bool sf_load = !(kTuning && (p.dbg & kDbgNoSfLoad));
-        const uint32_t tx = 2u * (kStageBytes - (sf_load ? 0 : kSfaBytes + kSfbBytes));
+        const uint32_t tx = 2u * (kABytes + kBBytes + (sf_load ? kSfLoadBytes : 0));
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -280,8 +285,8 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     }
                     const uint32_t ssfa = smem_base + stage * kStageBytes + kABytes + kBBytes;
                     if (elected) {
-                        ptx::tma_load_3d_pair(ssfa, &tm_sfa, 0, kt * 4, rca, full0 + 8u * stage);
-                        ptx::tma_load_3d_pair(ssfa + kSfaBytes, &tm_sfb, 0, kt * 4, rcb, full0 + 8u * stage);
+                        ptx::tma_load_3d_pair(ssfa, &tm_sfa, 0, kt * kSfChunksK, rca, full0 + 8u * stage);
+                        ptx::tma_load_3d_pair(ssfa + kSfaBytes, &tm_sfb, 0, kt * kSfChunksK, rcb, full0 + 8u * stage);
                     }
                     if (++stage == kStages) {
                         stage = 0;
@@ -296,8 +301,12 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         // The loop is warp-uniform so every operand lives in uniform registers; one elected lane issues.
         if (leader) {
             const bool elected = ptx::elect_one();
+            // E2M1 x E2M1, M = 256; scale format UE4M3 (0) or UE8M0 (1) in bit 23
             const uint32_t idesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(kBN >> 3) << 17) |
-                                   (static_cast<uint32_t>((2 * kBM) >> 4) << 24);  // E2M1 x E2M1, UE4M3, M=256
+                                   (kMx ? (1u << 23) : 0u) | (static_cast<uint32_t>((2 * kBM) >> 4) << 24);
+            // MXFP4: the odd instruction of a scale chunk takes bytes 2..3 of the scale columns (scale ids of
+            // A in bits 29..30, of B in bits 4..5)
+            constexpr uint32_t kSfIdHi = (2u << 29) | (2u << 4);
             const uint64_t desc_hi = ptx::smem_desc_sw128(0);
             const uint32_t a_lo0 = (smem_base & 0x3FFFFu) >> 4;
             const uint32_t b_lo0 = ((smem_base + kABytes) & 0x3FFFFu) >> 4;
@@ -343,7 +352,15 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     const uint32_t sfa_t = tmem_base + kSfCol + sf_buf * kSfBufCols;
                     const uint32_t sfb_t = sfa_t + 16;
                     if (elected && !no_mma) {
-                        if (kt + 1 < k_tiles || tail_mmas == kMmasPerStage) {
+                        if (kMx) {
+                            const int nm = (kt + 1 < k_tiles) ? kMmasPerStage : tail_mmas;
+#pragma unroll
+                            for (int j = 0; j < kMmasPerStage; ++j)
+                                if (j < nm)
+                                    ptx::mma_mxfp4_pair(d_tmem, a_desc + 2u * j, b_desc + 2u * j,
+                                                        idesc | ((j & 1) ? kSfIdHi : 0u), sfa_t + 4 * (j >> 1),
+                                                        sfb_t + 8 * (j >> 1), (kt | j) != 0);
+                        } else if (kt + 1 < k_tiles || tail_mmas == kMmasPerStage) {
                             ptx::mma_nvfp4_pair(d_tmem, a_desc, b_desc, idesc, sfa_t, sfb_t, kt != 0);
                             ptx::mma_nvfp4_pair(d_tmem, a_desc + 2, b_desc + 2, idesc, sfa_t + 4, sfb_t + 8, 1);
                             ptx::mma_nvfp4_pair(d_tmem, a_desc + 4, b_desc + 4, idesc, sfa_t + 8, sfb_t + 16, 1);
@@ -406,10 +423,13 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     if (elected) {
                         const uint32_t ssf = smem_base + stage * kStageBytes + kABytes + kBBytes;
                         const uint32_t sf_t = tmem_base + kSfCol + sf_buf * kSfBufCols;
-                        if (w < nmma) {  // warp w: the scales of MMA w -- A chunk, then the two B row chunks
+                        // warp w: scale chunk w of the stage (NVFP4: the scales of MMA w; MXFP4: of MMAs 2w and
+                        // 2w+1) -- the A chunk, then the two B row chunks
+                        if (w < (kMx ? (nmma + 1) / 2 : nmma)) {
                             ptx::tc_copy_sf_pair(sf_t + 4 * w, ptx::smem_desc_sf(ssf + w * 512));
                             ptx::tc_copy_sf_pair(sf_t + 16 + 8 * w, ptx::smem_desc_sf(ssf + kSfaBytes + w * 512));
-                            ptx::tc_copy_sf_pair(sf_t + 20 + 8 * w, ptx::smem_desc_sf(ssf + kSfaBytes + 2048 + w * 512));
+                            ptx::tc_copy_sf_pair(sf_t + 20 + 8 * w,
+                                                 ptx::smem_desc_sf(ssf + kSfaBytes + kSfRowChunkBytes + w * 512));
                         }
                         ptx::tc_commit_pair(sf_ready_bar(sf_buf));
                     }
@@ -435,7 +455,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         const int half = e >> 2;     // which of the quadrant's two warps
         const uint32_t sbuf = epi_base + e * kEpiBufBytes;
         const uint32_t sbias = bias_base + e * 256;
-        const float alpha = __fmul_rn(__ldcg(p.ts_a), __ldcg(p.ts_b));
+        const float alpha = kMx ? 1.0f : __fmul_rn(__ldcg(p.ts_a), __ldcg(p.ts_b));
         const float Tq = kOut != kOutBf16 ? __ldcg(p.ts_out) : 1.0f;
         const float c6T = __fmul_rn(6.0f, Tq);
         uint32_t amax2 = 0;
@@ -538,18 +558,19 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
 
 namespace {
 
-sol_status_t launch_pair256(int out_mode, const void *xq, const void *xsf, const float *xts, const void *wq,
+sol_status_t launch_pair256(int out_mode, bool mx, const void *xq, const void *xsf, const float *xts, const void *wq,
                             const void *wsf, const float *wts, const void *bias, void *y, int64_t ldy,
                             const float *ts_out, void *hsf, uint32_t *amax_out, int64_t M, int64_t N, int64_t K,
                             cudaStream_t stream, const DeviceInfo *dev) {
-    const uint64_t chunks_k = static_cast<uint64_t>(ceil_div(K, 64));
+    const uint64_t chunks_k = static_cast<uint64_t>(ceil_div(K, mx ? 128 : 64));
+    const uint32_t box_k = mx ? 2 : 4;
     CUtensorMap tm_a, tm_b, tm_y, tm_sfa, tm_sfb;
     bool ok = make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, xq, K / 2, M, K / 2, 128, kBM,
                            CU_TENSOR_MAP_SWIZZLE_128B) &&
               make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, wq, K / 2, N, K / 2, 128, kBN / 2,
                            CU_TENSOR_MAP_SWIZZLE_128B) &&
-              make_tmap_sf(&tm_sfa, xsf, chunks_k, static_cast<uint64_t>(ceil_div(M, 128)), 1) &&
-              make_tmap_sf(&tm_sfb, wsf, chunks_k, static_cast<uint64_t>(ceil_div(N, 128)), 2);
+              make_tmap_sf(&tm_sfa, xsf, chunks_k, static_cast<uint64_t>(ceil_div(M, 128)), 1, box_k) &&
+              make_tmap_sf(&tm_sfb, wsf, chunks_k, static_cast<uint64_t>(ceil_div(N, 128)), 2, box_k);
     if (out_mode == kOutBf16)
         ok = ok && make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, N, M, ldy * 2, 64, 32,
                                 CU_TENSOR_MAP_SWIZZLE_128B);
@@ -573,13 +594,16 @@ sol_status_t launch_pair256(int out_mode, const void *xq, const void *xsf, const
 #ifdef SOL_TUNING
     if (const char *e = getenv("SOL_DBG")) p.dbg = static_cast<uint32_t>(atoi(e));
 #endif
-    auto kern = out_mode == kOutBf16 ? gemm_pair_fp4_kernel<kOutBf16>
-                : out_mode == kOutQuant ? gemm_pair_fp4_kernel<kOutQuant> : gemm_pair_fp4_kernel<kOutQuantGelu>;
-    static bool configured[3][64] = {};
-    if (dev->device < 64 && !configured[out_mode][dev->device]) {
+    auto kern = mx ? gemm_pair_fp4_kernel<kOutBf16, true>
+                : out_mode == kOutBf16 ? gemm_pair_fp4_kernel<kOutBf16, false>
+                : out_mode == kOutQuant ? gemm_pair_fp4_kernel<kOutQuant, false>
+                                        : gemm_pair_fp4_kernel<kOutQuantGelu, false>;
+    static bool configured[4][64] = {};
+    const int slot = mx ? 3 : out_mode;
+    if (dev->device < 64 && !configured[slot][dev->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return SOL_ERR_CUDA;
-        configured[out_mode][dev->device] = true;
+        configured[slot][dev->device] = true;
     }
     p.m_tiles = static_cast<int>(ceil_div(p.M, 2 * kBM));
     p.n_tiles = static_cast<int>(ceil_div(p.N, kBN));
@@ -612,8 +636,15 @@ sol_status_t launch_pair256(int out_mode, const void *xq, const void *xsf, const
 sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
                                   const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
                                   int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev) {
-    return launch_pair256(kOutBf16, xq, xsf, xts, wq, wsf, wts, bias, y, ldy, nullptr, nullptr, nullptr, M, N, K,
-                          stream, dev);
+    return launch_pair256(kOutBf16, false, xq, xsf, xts, wq, wsf, wts, bias, y, ldy, nullptr, nullptr, nullptr, M, N,
+                          K, stream, dev);
+}
+
+sol_status_t launch_pair256_mxfp4(const void *xq, const void *xsf, const void *wq, const void *wsf, const void *bias,
+                                  void *y, int64_t M, int64_t N, int64_t K, int64_t ldy, cudaStream_t stream,
+                                  const DeviceInfo *dev) {
+    return launch_pair256(kOutBf16, true, xq, xsf, nullptr, wq, wsf, nullptr, bias, y, ldy, nullptr, nullptr, nullptr,
+                          M, N, K, stream, dev);
 }
 
 sol_status_t launch_pair256_nvfp4_quant_out(const void *xq, const void *xsf, const float *xts, const void *wq,
@@ -621,7 +652,7 @@ sol_status_t launch_pair256_nvfp4_quant_out(const void *xq, const void *xsf, con
                                             const float *ts_out, void *hq, void *hsf, uint32_t *amax_out,
                                             int64_t M, int64_t N, int64_t K, cudaStream_t stream,
                                             const DeviceInfo *dev) {
-    return launch_pair256(act == 1 ? kOutQuantGelu : kOutQuant, xq, xsf, xts, wq, wsf, wts, bias, hq, 0, ts_out, hsf,
+    return launch_pair256(act == 1 ? kOutQuantGelu : kOutQuant, false, xq, xsf, xts, wq, wsf, wts, bias, hq, 0, ts_out, hsf,
                           amax_out, M, N, K, stream, dev);
 }
 

@@ -149,6 +149,81 @@ quantize_group_kernel(const __grid_constant__ QuantGroup g, int64_t rows, int64_
     quantize_tile<kSwizzled>(g.x[z], rows, K, K, nullptr, g.scale_words[z] + 1, g.scale_words[z], g.q[z], g.sf[z]);
 }
 
+// MXFP4 quantizer (the OCP format Section 2 sets beside NVFP4): 32 elements share one E8M0 scale
+// 2^(floor(log2 amax) - 2); x / scale is an exact power-of-two scaling, so there is no division and no
+// tensor-level scale.  One block = 128 rows x 512 elements (= four scale chunks of 128 x 4); a thread
+// owns whole 32-element blocks: four 16-byte loads, one 16-byte store, one scale byte.
+constexpr int kMxTileK = 512;
+constexpr int kMxBlocksPerThread = kTileRows * (kMxTileK / 32) / kQuantThreads;  // 8
+
+template <bool kSwizzled>
+__global__ void __launch_bounds__(kQuantThreads)
+mxfp4_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld, uint8_t *__restrict__ q,
+                      uint8_t *__restrict__ sf) {
+    __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kMxTileK / 32)];  // 2 KB = 4 chunks
+    const int b = threadIdx.x & 15;   // 32-element block inside the tile
+    const int r0 = threadIdx.x >> 4;
+    const int64_t row0 = static_cast<int64_t>(blockIdx.y) * kTileRows;
+    const int64_t k = static_cast<int64_t>(blockIdx.x) * kMxTileK + b * 32;
+    const bool k_ok = k < K;
+    if (kSwizzled) {
+        reinterpret_cast<uint64_t *>(sf_tile)[threadIdx.x] = 0;
+        __syncthreads();
+    }
+    grid_dependency_wait();
+    grid_launch_dependents();
+    const int64_t nb = K >> 5;
+#pragma unroll 1
+    for (int batch = 0; batch < kMxBlocksPerThread / 2; ++batch) {
+        uint4 v[2][4];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int64_t r = row0 + r0 + 16 * (batch * 2 + i);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[i][u] = make_uint4(0, 0, 0, 0);
+            if (k_ok && r < rows) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(x + r * ld + k);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) v[i][u] = __ldcs(src + u);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int rl = r0 + 16 * (batch * 2 + i);
+            const int64_t r = row0 + rl;
+            const uint32_t m = max(abs_max_bits(v[i][0], v[i][1]), abs_max_bits(v[i][2], v[i][3]));
+            const uint32_t e8 = m >> 7;                      // biased exponent of the block maximum
+            const uint32_t sb = e8 > 2u ? e8 - 2u : 0u;      // shared exponent floor(log2 amax) - 2, clamped at -127
+            const float inv = __uint_as_float((254u - sb) << 23);  // 2^(127 - sb), exact
+            uint4 packed;
+            packed.x = quantize8(v[i][0], inv);
+            packed.y = quantize8(v[i][1], inv);
+            packed.z = quantize8(v[i][2], inv);
+            packed.w = quantize8(v[i][3], inv);
+            if (k_ok && r < rows) {
+                __stcs(reinterpret_cast<uint4 *>(q + r * (K >> 1) + (k >> 1)), packed);
+                if (kSwizzled) {
+                    sf_tile[(b >> 2) * 512 + (rl & 31) * 16 + (rl >> 5) * 4 + (b & 3)] = static_cast<uint8_t>(sb);
+                } else {
+                    sf[r * nb + (k >> 5)] = static_cast<uint8_t>(sb);
+                }
+            }
+        }
+    }
+    if (kSwizzled) {
+        __syncthreads();
+        const int64_t chunks_k = (nb + 3) >> 2;
+        if (threadIdx.x < 128) {
+            const int cidx = threadIdx.x >> 5;
+            const int64_t kc = static_cast<int64_t>(blockIdx.x) * 4 + cidx;
+            if (kc < chunks_k) {
+                uint8_t *dst = sf + (static_cast<int64_t>(blockIdx.y) * chunks_k + kc) * 512 + (threadIdx.x & 31) * 16;
+                *reinterpret_cast<uint4 *>(dst) = reinterpret_cast<const uint4 *>(sf_tile)[threadIdx.x];
+            }
+        }
+    }
+}
+
 // max |x| over the tensor as the bit pattern of the FP32 value (BF16 magnitude << 16).
 __global__ void __launch_bounds__(256)
 amax_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t vecs_per_row, int64_t ld,
@@ -247,6 +322,26 @@ sol_status_t launch_amax(const void *x, int64_t rows, int64_t K, int64_t ld, flo
 sol_status_t launch_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale,
                              void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream) {
     return launch_quantize_ex(x, rows, K, ld, tscale, nullptr, nullptr, q, sf, layout, stream);
+}
+
+sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
+                                   sol_sf_layout_t layout, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ceil_div(K, kMxTileK)), static_cast<unsigned>(ceil_div(rows, kTileRows)));
+    cfg.blockDim = dim3(kQuantThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    auto kern = layout == SOL_SF_SWIZZLED_128x4 ? mxfp4_quantize_kernel<true> : mxfp4_quantize_kernel<false>;
+    if (cudaLaunchKernelEx(&cfg, kern, static_cast<const uint16_t *>(x), rows, K, ld, static_cast<uint8_t *>(q),
+                           static_cast<uint8_t *>(sf)) != cudaSuccess) {
+        cudaGetLastError();
+        return SOL_ERR_CUDA;
+    }
+    return launch_status();
 }
 
 sol_status_t launch_quantize_from_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,

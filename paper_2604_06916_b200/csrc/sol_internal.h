@@ -67,6 +67,8 @@ sol_status_t launch_lora_merge(const MergeGroup &g, int count, int64_t ldw, int6
 sol_status_t launch_quantize_group(const QuantGroup &g, int count, int64_t rows, int64_t K, sol_sf_layout_t layout,
                                    cudaStream_t stream);
 int lora_max_rank();
+sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
+                                   sol_sf_layout_t layout, cudaStream_t stream);
 // Stage-1 selection and rank-consistency metrics (one block per prompt).
 sol_status_t launch_select_contrastive(const float *rewards, const uint64_t *seeds, int64_t P, int64_t N, int64_t K,
                                        int32_t *idx_out, uint64_t *seeds_out, float *adv_out, cudaStream_t stream);
@@ -88,8 +90,8 @@ bool make_tmap_2d(CUtensorMap *out, CUtensorMapDataType dtype, uint32_t elem_byt
                   uint32_t box_outer, CUtensorMapSwizzle swizzle);
 
 // Scale-factor buffer in the chunked layout as a 3-D tensor [row chunk][k chunk][128 x u32]; the box
-// covers 4 k-chunks of `box_row_chunks` row chunks (out-of-range chunks read as zero).
+// covers `box_k_chunks` k-chunks of `box_row_chunks` row chunks (out-of-range chunks read as zero).
 bool make_tmap_sf(CUtensorMap *out, const void *base, uint64_t chunks_k, uint64_t row_chunks,
-                  uint32_t box_row_chunks);
+                  uint32_t box_row_chunks, uint32_t box_k_chunks = 4);
 
 }  // namespace sol

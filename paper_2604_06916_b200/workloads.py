@@ -52,6 +52,11 @@ CONFIG_FLUX = _mk("flux1_12b_g8", 3, "student_t", None, (4096 + 512) * 8,
                   [("d_qkv", 3072, 9216), ("d_proj", 3072, 3072), ("d_mlp_in", 3072, 12288),
                    ("d_mlp_out", 12288, 3072), ("s_fused", 3072, 21504), ("s_out", 15360, 3072)])
 
+# the geometry the paper trained FLUX.1 at (512 x 512 images: 1024 image + 512 text tokens), same layers
+CONFIG_FLUX_512 = _mk("flux1_12b_512px_g8", 5, "student_t", None, (1024 + 512) * 8,
+                      [("d_qkv", 3072, 9216), ("d_proj", 3072, 3072), ("d_mlp_in", 3072, 12288),
+                       ("d_mlp_out", 12288, 3072), ("s_fused", 3072, 21504), ("s_out", 15360, 3072)])
+
 SWEEP_GROUPS = (4, 8, 16, 32, 64)
 SWEEP_TOKENS = 4608
 SWEEP_STEPS = 28
@@ -63,7 +68,7 @@ def config_sweep(group: int) -> Config:
                [("s_fused", 3072, 21504), ("s_out", 15360, 3072)])
 
 
-CONFIGS = {c.name: c for c in (CONFIG_SINGLE, CONFIG_SANA, CONFIG_SD35, CONFIG_FLUX)}
+CONFIGS = {c.name: c for c in (CONFIG_SINGLE, CONFIG_SANA, CONFIG_SD35, CONFIG_FLUX, CONFIG_FLUX_512)}
 
 
 def _normal(shape, gen, device, chunk_rows=4096):

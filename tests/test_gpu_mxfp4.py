@@ -1,0 +1,130 @@
+"""GPU parity: MXFP4 quantizer (bit-exact) and linear (tolerance / integer-exact) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_06916_b200 import workloads
+from tests.helpers import bits_of, check_linear, from_bits, sample_rows
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2604_06916_b200 import binding
+    binding.lib()
+    return binding
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def mx_offsets(rows, K):
+    nb = K // 32
+    chunks_k = (nb + 3) // 4
+    r = np.asarray(rows, dtype=np.int64)[:, None]
+    b = np.arange(nb, dtype=np.int64)[None, :]
+    rr = r % 128
+    return ((r // 128) * chunks_k + b // 4) * 512 + (rr % 32) * 16 + (rr // 32) * 4 + b % 4
+
+
+def test_offset_helper_matches_oracle_rule():
+    K = 416
+    offs = mx_offsets(np.array([0, 31, 32, 127, 128, 300]), K)
+    for i, r in enumerate([0, 31, 32, 127, 128, 300]):
+        for b in range(K // 32):
+            assert offs[i, b] == oracle.mx_sf_swizzled_offset(r, b, K)
+
+
+@pytest.mark.parametrize("M,K,pad", [(256, 512, 0), (1, 32, 0), (130, 160, 0), (257, 2240, 8), (40, 5600, 64), (300, 96, 32)])
+def test_quantizer_bit_exact_both_layouts(B, M, K, pad):
+    g = torch.Generator(device="cuda").manual_seed(M + K)
+    big = workloads.make_activation("outlier", M, K + pad, g, "cuda") * 3.0
+    x = big[:, :K]
+    xb = bits_of(x.contiguous())
+    want_q, want_sf = oracle.mxfp4_quantize(xb)
+    q, sf = B.mxfp4_quantize(x, B.SF_ROW_MAJOR)
+    assert np.array_equal(q.cpu().numpy(), want_q)
+    assert np.array_equal(sf.cpu().numpy().reshape(M, K // 32), want_sf)
+    q2, sf2 = B.mxfp4_quantize(x, B.SF_SWIZZLED_128x4)
+    assert np.array_equal(q2.cpu().numpy(), want_q)
+    assert np.array_equal(sf2.cpu().numpy(), oracle.mx_sf_swizzle(want_sf, K))      # padding bytes are 0
+
+
+def test_quantizer_special_values(B):
+    vals = np.zeros((2, 64))
+    vals[0, :9] = [12, 6, 3, -1.5, 0.5, 5, -12, 0.1015625, 2.5]
+    vals[1, :6] = [7.5, -5.0, 0.25, 2.0 ** -20, -2.0 ** -30, 1e-38]
+    xb = bits_of(torch.tensor(vals, dtype=torch.float64).to(torch.bfloat16))
+    xb[1, 40] = 0x8000     # -0
+    xb[1, 41] = 0x0001     # smallest subnormal
+    xb[0, 63] = 0x7F7F     # largest finite
+    x = from_bits(xb, "cuda")
+    q, sf = B.mxfp4_quantize(x, B.SF_ROW_MAJOR)
+    want_q, want_sf = oracle.mxfp4_quantize(xb)
+    assert np.array_equal(q.cpu().numpy(), want_q) and np.array_equal(sf.cpu().numpy().reshape(2, 2), want_sf)
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 256, 64), (128, 192, 256), (256, 384, 512), (130, 200, 96), (64, 8, 32),
+                                   (300, 456, 448), (200, 264, 1312)])
+def test_linear_integer_exact(B, M, N, K):
+    rng = np.random.default_rng(M + N + K)
+    qx = rng.integers(0, 256, size=(M, K // 2), dtype=np.uint8)
+    qw = rng.integers(0, 256, size=(N, K // 2), dtype=np.uint8)
+    sfx = (rng.integers(-2, 3, size=(M, K // 32)) + 127).astype(np.uint8)
+    sfw = (rng.integers(-2, 3, size=(N, K // 32)) + 127).astype(np.uint8)
+    Y = oracle.mxfp4_linear(qx, sfx, qw, sfw)
+    if np.abs(Y).max() * 4 >= 2 ** 24:
+        pytest.skip("sum too large for an exact FP32 accumulator")
+    y = B.mxfp4_linear(dev(qx), dev(oracle.mx_sf_swizzle(sfx, K)), dev(qw), dev(oracle.mx_sf_swizzle(sfw, K)))
+    B.sol_last_device_status()
+    got, want = bits_of(y), oracle.round_bf16(Y)
+    bad = got != want
+    assert not bad.any(), (f"{int(bad.sum())} of {bad.size} differ; rows {np.unique(np.argwhere(bad)[:, 0])[:10]} "
+                           f"cols {np.unique(np.argwhere(bad)[:, 1])[:10]}")
+
+
+def test_scale_placement_probe(B):
+    # one non-zero row of X whose 32-element blocks carry distinct scales, against one-hot rows of W:
+    # every output isolates one (row, block) scale and one nibble position
+    M, N, K = 256, 256, 512
+    for row in (0, 77, 128, 255):
+        qx = np.zeros((M, K // 2), np.uint8)
+        sfx = np.full((M, K // 32), 127, np.uint8)
+        qx[row, :] = 0x22                                   # every element 1.0
+        sfx[row, :] = (np.arange(K // 32) % 7 + 124).astype(np.uint8)
+        qw = np.zeros((N, K // 2), np.uint8)
+        sfw = np.full((N, K // 32), 127, np.uint8)
+        ks = (np.arange(N) * 37 + 5) % K
+        for n, k in enumerate(ks):
+            qw[n, k // 2] = 0x2 << (4 * (k & 1))
+            sfw[n, k // 32] = (n % 5) + 125
+        Y = oracle.mxfp4_linear(qx, sfx, qw, sfw)
+        y = B.mxfp4_linear(dev(qx), dev(oracle.mx_sf_swizzle(sfx, K)), dev(qw), dev(oracle.mx_sf_swizzle(sfw, K)))
+        assert np.array_equal(bits_of(y), oracle.round_bf16(Y)), f"row {row}"
+        assert np.count_nonzero(Y) == N
+
+
+@pytest.mark.parametrize("index", [1, 5])   # FLUX d_proj and s_out at full size, sampled rows
+def test_flux_layers_sampled_rows(B, index):
+    cfg = workloads.CONFIG_FLUX
+    layer = cfg.layers[index]
+    X, W, bias = workloads.make_layer(cfg, index, "cuda")
+    M, K, N = layer.M, layer.K, layer.N
+    xq, xsf = B.mxfp4_quantize(X)
+    wq, wsf = B.mxfp4_quantize(W)
+    y = B.mxfp4_linear(xq, xsf, wq, wsf, bias)
+    B.sol_last_device_status()
+    rows = sample_rows(M, seed=index)
+    rows_t = torch.from_numpy(rows).cuda()
+    # quantizer outputs of the sampled rows and of W, bit for bit
+    want_qx, want_sfx = oracle.mxfp4_quantize(bits_of(X[rows_t]))
+    want_qw, want_sfw = oracle.mxfp4_quantize(bits_of(W))
+    assert np.array_equal(xq[rows_t].cpu().numpy(), want_qx)
+    assert np.array_equal(xsf.cpu().numpy()[mx_offsets(rows, K)], want_sfx)
+    assert np.array_equal(wq.cpu().numpy(), want_qw)
+    assert np.array_equal(wsf.cpu().numpy(), oracle.mx_sf_swizzle(want_sfw, K))
+    Y = oracle.mxfp4_linear(want_qx, want_sfx, want_qw, want_sfw, bits_of(bias))
+    check_linear(bits_of(y[rows_t]), Y, f"{cfg.name}/{layer.name} mxfp4")
