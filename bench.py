@@ -545,6 +545,30 @@ def run_only(args):
         B.sol_last_device_status()
         print(json.dumps({"only": "weight_refresh", "matrices": 8, "us_per_matrix": 1e3 * sum(times) / len(times) / 8}))
         return
+    if args.only.startswith("mxfp4:"):
+        # one layer through the MXFP4 quantizer and GEMM
+        cfg = workloads.CONFIGS[args.workload]
+        index = [l.name for l in cfg.layers].index(args.only.split(":", 1)[1])
+        l = cfg.layers[index]
+        M = args.rows if args.rows > 0 else l.M
+        X, W, bias = workloads.make_layer(cfg, index, "cuda", M=M)
+        wq, wsf = B.mxfp4_quantize(W)
+        Y = torch.empty((M, l.N), dtype=torch.bfloat16, device="cuda")
+        times = []
+        for it in range(args.warmup + args.steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            xq, xsf = B.mxfp4_quantize(X)
+            B.mxfp4_linear(xq, xsf, wq, wsf, bias, out=Y)
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                times.append(e0.elapsed_time(e1))
+        B.sol_last_device_status()
+        t = sum(times) / len(times)
+        print(json.dumps({"only": args.only, "M": M, "K": l.K, "N": l.N, "mxfp4_stack_ms": t,
+                          "mxfp4_stack_tflops": 2.0 * M * l.N * l.K / t / 1e9}))
+        return
     if args.only == "mlp_pair":
         # FLUX feed-forward pair with the intermediate kept in NVFP4 (GELU in the first GEMM's epilogue)
         cfg = workloads.CONFIGS[args.workload]
@@ -603,7 +627,7 @@ def run_only(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair'")
+    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair' / 'mxfp4:<layer>'")
     ap.add_argument("--rows", type=int, default=0, help="profile mode: override M")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)

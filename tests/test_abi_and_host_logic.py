@@ -112,6 +112,16 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.solrl_rank_consistency(p, p, 2, 1, 1, p, None, None) == SHAPE
     assert L.solrl_rank_consistency(p, p, 2, 8, 9, p, None, None) == SHAPE
     assert L.solrl_rank_consistency(p, p, 2, 8, 4, p + 4, None, None) == ALIGN
+    # MXFP4
+    assert L.sol_mxfp4_scale_bytes(256, 512, 0) == 256 * 16 and L.sol_mxfp4_scale_bytes(256, 512, 1) == 2 * 4 * 512
+    assert L.sol_mxfp4_scale_bytes(130, 160, 1) == 2 * 2 * 512 and L.sol_mxfp4_scale_bytes(4, 48, 1) == 0
+    assert L.mxfp4_quantize(None, 4, 64, 64, p, p, 1, None) == NULLP
+    assert L.mxfp4_quantize(p, 4, 48, 48, p, p, 1, None) == SHAPE
+    assert L.mxfp4_quantize(p, 4, 64, 64, p, p, 3, None) == LAYOUT
+    assert L.mxfp4_quantize(p, 4, 64, 68, p, p, 1, None) == ALIGN
+    assert L.mxfp4_linear(p, p, p, p, None, None, 4, 8, 64, 8, None) == NULLP
+    assert L.mxfp4_linear(p, p, p, p, None, p, 4, 12, 64, 16, None) == SHAPE
+    assert L.mxfp4_linear(p, p + 8, p, p, None, p, 4, 8, 64, 8, None) == ALIGN
     # linear with quantized output
     assert L.nvfp4_linear_quantized_out(p, p, p, p, p, p, None, 0, None, p, p, None, 4, 64, 64, None) == NULLP
     assert L.nvfp4_linear_quantized_out(p, p, p, p, p, p, None, 0, p, p, p, None, 4, 96, 64, None) == SHAPE   # N % 64
