@@ -61,6 +61,9 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
                                               const float *tscale, const float *amax, float *tscale_out,
                                               uint8_t *__restrict__ q, uint8_t *__restrict__ sf) {
     __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kTileK / 16)];  // 2 KB = 4 chunks
+    // 1 / (float(sb) * T) for every scale byte: d takes at most 127 values per tensor, so the decode,
+    // the multiplication and the IEEE reciprocal run once per thread block instead of once per scale block
+    __shared__ float rcp_tab[128];
 
     const int b = threadIdx.x & 15;   // scale block inside the tile
     const int r0 = threadIdx.x >> 4;  // first row inside the tile
@@ -79,6 +82,11 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
     if (tscale_out != nullptr && threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0) *tscale_out = T;
     const float c = __fmul_rn(6.0f, T);
     const int64_t nb = K >> 4;
+    if (threadIdx.x < 128) {
+        const uint32_t code = threadIdx.x;
+        rcp_tab[code] = code ? __frcp_rn(__fmul_rn(e4m3_to_f32(code), T)) : 0.0f;
+    }
+    __syncthreads();
 
 #pragma unroll 1
     for (int batch = 0; batch < kBlocksPerThread / kBatch; ++batch) {
@@ -100,8 +108,7 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
             const float a = __uint_as_float(abs_max_bits(lo[i], hi[i]) << 16);
             const float sv = __fdiv_rn(a, c);
             const uint32_t sb = f32_to_e4m3_sat(sv);
-            const float d = __fmul_rn(e4m3_to_f32(sb), T);
-            const float rcp = sb ? __frcp_rn(d) : 0.0f;
+            const float rcp = rcp_tab[sb];
             uint2 packed;
             packed.x = quantize8(lo[i], rcp);
             packed.y = quantize8(hi[i], rcp);
