@@ -188,6 +188,34 @@ sol_status_t nvfp4_linear_quantized_out(const void *xq, const void *xsf, const f
                                         void *stream);
 
 /*
+ * The same for a linear whose outputs feed two consumers, as the first linear of a single-stream
+ * DiT block does (3072 -> 9216 + 12288 in the FLUX-shaped config): columns [0, n_split) leave as BF16
+ * (q, k, v for attention); columns [n_split, N) pass through the activation and leave quantized
+ * into columns [dest_col0, dest_col0 + N - n_split) of a WIDER quantized tensor [M, dest_K] -- the
+ * concatenated input of the next linear, whose other columns nvfp4_quantize_into fills.
+ *   y_bf16      [M, n_split] BF16, pitch ldy
+ *   hq_dest     packed nibbles [M, dest_K/2];  hsf_dest  chunked scales of an [M, dest_K] tensor
+ *   out_tscale  the tensor scale of the whole destination tensor (one T for all its parts)
+ *   n_split % 256 == 0, (N - n_split) % 64 == 0, dest_K % 64 == 0, dest_col0 % 64 == 0.
+ * Everything else as nvfp4_linear_quantized_out.
+ */
+sol_status_t nvfp4_linear_split_out(const void *xq, const void *xsf, const float *x_tscale, const void *wq,
+                                    const void *wsf, const float *w_tscale, const void *bias_bf16, void *y_bf16,
+                                    int64_t ldy, int64_t n_split, sol_activation_t activation,
+                                    const float *out_tscale, void *hq_dest, void *hsf_dest, int64_t dest_K,
+                                    int64_t dest_col0, float *amax_out, int64_t M, int64_t N, int64_t K,
+                                    void *stream);
+
+/*
+ * nvfp4_quantize writing into columns [dest_col0, dest_col0 + K) of a wider quantized tensor
+ * [M, dest_K] (chunked scale layout): the part of a concatenated activation that arrives in BF16.
+ * K, dest_K and dest_col0 are multiples of 64; bytes outside the column range are not touched, so
+ * the rows past M of the destination's last 128-row scale chunk must have been zeroed once.
+ */
+sol_status_t nvfp4_quantize_into(const void *x_bf16, int64_t M, int64_t K, int64_t ldx, const float *tensor_scale,
+                                 void *q_dest, void *sf_dest, int64_t dest_K, int64_t dest_col0, void *stream);
+
+/*
  * BF16 linear, the full-precision stage-2 reference (Section 3.4):
  *     Y[m,n] = bf16_rne( sum_k x[m,k] * w[n,k] + bias[n] ),  FP32 accumulate.
  */

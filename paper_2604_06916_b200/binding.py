@@ -24,7 +24,7 @@ EXPORTS = [
     "sol_nvfp4_static_scratch_bytes", "nvfp4_quantize_linear_static", "nvfp4_quantize_linear_host",
     "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch", "nvfp4_linear_quantized_out",
     "solrl_select_contrastive", "solrl_rank_consistency", "sol_mxfp4_scale_bytes", "mxfp4_quantize",
-    "mxfp4_linear",
+    "mxfp4_linear", "nvfp4_linear_split_out", "nvfp4_quantize_into",
 ]
 
 _lib = None
@@ -82,6 +82,11 @@ def lib() -> ctypes.CDLL:
     L.sol_mxfp4_scale_bytes.restype, L.sol_mxfp4_scale_bytes.argtypes = sz, [i64, i64, i32]
     L.mxfp4_quantize.restype, L.mxfp4_quantize.argtypes = i32, [vp, i64, i64, i64, vp, vp, i32, vp]
     L.mxfp4_linear.restype, L.mxfp4_linear.argtypes = i32, [vp, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp]
+    L.nvfp4_linear_split_out.restype = i32
+    L.nvfp4_linear_split_out.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i64, i64, i32, vp, vp, vp, i64, i64, vp, i64,
+                                         i64, i64, vp]
+    L.nvfp4_quantize_into.restype = i32
+    L.nvfp4_quantize_into.argtypes = [vp, i64, i64, i64, vp, vp, vp, i64, i64, vp]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -244,6 +249,32 @@ def nvfp4_linear(xq, xsf, x_tscale, wq, wsf, w_tscale, bias=None, out: torch.Ten
 
 
 ACT_NONE, ACT_GELU_TANH = 0, 1
+
+
+def nvfp4_linear_split_out(xq, xsf, x_tscale, wq, wsf, w_tscale, bias, n_split: int, activation: int, out_tscale,
+                           dest, dest_col0: int, y_out: torch.Tensor | None = None,
+                           amax_out: torch.Tensor | None = None):
+    """Columns below n_split -> BF16 `y_out`; the rest -> activation -> quantized into dest = (q [M, dest_K/2], sf)."""
+    M, K = xq.shape[0], xq.shape[1] * 2
+    N = wq.shape[0]
+    hq, hsf = dest
+    dest_K = hq.shape[1] * 2
+    if y_out is None:
+        y_out = torch.empty((M, n_split), dtype=torch.bfloat16, device=xq.device)
+    _check(lib().nvfp4_linear_split_out(_ptr(xq), _ptr(xsf), _ptr(x_tscale), _ptr(wq), _ptr(wsf), _ptr(w_tscale),
+                                        _ptr(bias), _ptr(y_out), y_out.stride(0), n_split, activation, _ptr(out_tscale),
+                                        _ptr(hq), _ptr(hsf), dest_K, dest_col0, _ptr(amax_out), M, N, K, _stream()),
+           "nvfp4_linear_split_out")
+    return y_out
+
+
+def nvfp4_quantize_into(x: torch.Tensor, tensor_scale: torch.Tensor, dest, dest_col0: int):
+    """Quantize BF16 x [M, K] into columns [dest_col0, dest_col0 + K) of dest = (q [M, dest_K/2], sf)."""
+    _need_2d_bf16(x, "x")
+    M, K = x.shape
+    hq, hsf = dest
+    _check(lib().nvfp4_quantize_into(_ptr(x), M, K, x.stride(0), _ptr(tensor_scale), _ptr(hq), _ptr(hsf),
+                                     hq.shape[1] * 2, dest_col0, _stream()), "nvfp4_quantize_into")
 
 
 def mxfp4_scale_bytes(rows: int, K: int, layout: int = SF_SWIZZLED_128x4) -> int:

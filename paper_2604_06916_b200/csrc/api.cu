@@ -400,6 +400,50 @@ sol_status_t solrl_rank_consistency(const float *rewards_ref, const float *rewar
                                    static_cast<cudaStream_t>(stream));
 }
 
+sol_status_t nvfp4_linear_split_out(const void *xq, const void *xsf, const float *x_tscale, const void *wq,
+                                    const void *wsf, const float *w_tscale, const void *bias_bf16, void *y_bf16,
+                                    int64_t ldy, int64_t n_split, sol_activation_t activation, const float *out_tscale,
+                                    void *hq_dest, void *hsf_dest, int64_t dest_K, int64_t dest_col0, float *amax_out,
+                                    int64_t M, int64_t N, int64_t K, void *stream) {
+    if (xq == nullptr || xsf == nullptr || x_tscale == nullptr || wq == nullptr || wsf == nullptr ||
+        w_tscale == nullptr || y_bf16 == nullptr || out_tscale == nullptr || hq_dest == nullptr || hsf_dest == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(M, K) || N <= 0 || N > (1LL << 24) || n_split <= 0 || n_split >= N || n_split % 256 != 0 ||
+        (N - n_split) % 64 != 0 || ldy < n_split || dest_K <= 0 || dest_K % 64 != 0 || dest_col0 < 0 ||
+        dest_col0 % 64 != 0 || dest_col0 + (N - n_split) > dest_K)
+        return SOL_ERR_BAD_SHAPE;
+    if (activation != SOL_ACT_NONE && activation != SOL_ACT_GELU_TANH) return SOL_ERR_BAD_LAYOUT;
+    if (!aligned16(xq) || !aligned16(xsf) || !aligned16(wq) || !aligned16(wsf) || !aligned16(y_bf16) ||
+        !aligned16(hq_dest) || !aligned16(hsf_dest) || ldy % 8 != 0 || (bias_bf16 != nullptr && !aligned16(bias_bf16)) ||
+        (reinterpret_cast<uintptr_t>(x_tscale) & 3u) || (reinterpret_cast<uintptr_t>(w_tscale) & 3u) ||
+        (reinterpret_cast<uintptr_t>(out_tscale) & 3u) || (reinterpret_cast<uintptr_t>(amax_out) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return gemm::launch_pair256_nvfp4_split_out(xq, xsf, x_tscale, wq, wsf, w_tscale, bias_bf16, y_bf16, ldy, n_split,
+                                                activation == SOL_ACT_GELU_TANH ? 1 : 0, out_tscale, hq_dest, hsf_dest,
+                                                dest_K, dest_col0, reinterpret_cast<uint32_t *>(amax_out), M, N, K,
+                                                static_cast<cudaStream_t>(stream), dev);
+}
+
+sol_status_t nvfp4_quantize_into(const void *x_bf16, int64_t M, int64_t K, int64_t ldx, const float *tensor_scale,
+                                 void *q_dest, void *sf_dest, int64_t dest_K, int64_t dest_col0, void *stream) {
+    if (x_bf16 == nullptr || tensor_scale == nullptr || q_dest == nullptr || sf_dest == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(M, K) || ldx < K || K % 64 != 0 || dest_K <= 0 || dest_K % 64 != 0 || dest_col0 < 0 ||
+        dest_col0 % 64 != 0 || dest_col0 + K > dest_K)
+        return SOL_ERR_BAD_SHAPE;
+    if (!aligned16(x_bf16) || !aligned16(q_dest) || !aligned16(sf_dest) || ldx % 8 != 0 ||
+        (reinterpret_cast<uintptr_t>(tensor_scale) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_quantize_into(x_bf16, M, K, ldx, tensor_scale, q_dest, sf_dest, dest_K, dest_col0,
+                                static_cast<cudaStream_t>(stream));
+}
+
 sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,
                                    const float *w_tscale, const void *bias_bf16, void *y_bf16, int64_t M,
                                    int64_t N, int64_t K, int64_t ldy, void *workspace, size_t workspace_bytes,

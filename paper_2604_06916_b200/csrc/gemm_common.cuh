@@ -51,6 +51,10 @@ struct Params {
     uint8_t *sf_out;        // scales of the output, chunked layout for an [M, N] tensor
     const float *ts_out;    // tensor scale T of the output (caller supplied)
     uint32_t *amax_out;     // running max |h| as FP32 bits (atomicMax), or null
+    int act;                // 0 = identity, 1 = GELU (tanh form) before the output quantizer
+    int n_split;            // split mode: columns below it leave as BF16, the rest quantized
+    int dest_col0;          // first column of the quantized part inside the destination tensor
+    int dest_chunks_k;      // scale chunks per 128-row tile of the destination tensor
 };
 
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
@@ -155,6 +159,12 @@ sol_status_t launch_pair_nvfp4(const void *xq, const void *xsf, const float *xts
 sol_status_t launch_pair256_nvfp4_quant_out(const void *xq, const void *xsf, const float *xts, const void *wq,
                                             const void *wsf, const float *wts, const void *bias, int act,
                                             const float *ts_out, void *hq, void *hsf, uint32_t *amax_out,
+                                            int64_t M, int64_t N, int64_t K, cudaStream_t stream,
+                                            const DeviceInfo *dev);
+sol_status_t launch_pair256_nvfp4_split_out(const void *xq, const void *xsf, const float *xts, const void *wq,
+                                            const void *wsf, const float *wts, const void *bias, void *y_bf16,
+                                            int64_t ldy, int64_t n_split, int act, const float *ts_out, void *hq,
+                                            void *hsf, int64_t dest_K, int64_t dest_col0, uint32_t *amax_out,
                                             int64_t M, int64_t N, int64_t K, cudaStream_t stream,
                                             const DeviceInfo *dev);
 sol_status_t launch_pair256_mxfp4(const void *xq, const void *xsf, const void *wq, const void *wsf, const void *bias,

@@ -87,7 +87,9 @@ __device__ __forceinline__ void epilogue_store(const CUtensorMap *tm_y, const Pa
 
 // Output modes of the kernel: BF16 Y, or Y passed through an activation and quantized for the next
 // linear (packed E2M1 + E4M3 block scales along N, with a caller-supplied tensor scale).
-enum : int { kOutBf16 = 0, kOutQuant = 1, kOutQuantGelu = 2 };
+// kOutSplit: tiles left of column n_split leave as BF16, tiles right of it quantized into a column
+// range of a wider destination tensor (the concatenated input of the next linear).
+enum : int { kOutBf16 = 0, kOutQuant = 1, kOutSplit = 2 };
 
 // tanh-form GELU, 0.5 y (1 + tanh(u)), u = sqrt(2/pi) y (1 + 0.044715 y^2), with the hardware tanh
 // (one special-function op per element; the epilogue is bound by that unit, and the exact form
@@ -106,11 +108,11 @@ __device__ __forceinline__ float gelu_tanh(float y) {
 // quantizer's FP32 sequence.  A row's 64 columns are 32 bytes of nibbles (staged, one TMA store
 // of 32 rows x 32 bytes per chunk) and the four scale bytes of one (row, k-chunk) slot of the
 // chunked scale layout (one 4-byte store).  `amax2` collects max|h| per BF16 half.
-template <int kOut>
 __device__ __forceinline__ void epilogue_quant_store(const CUtensorMap *tm_q, const Params &p, const uint32_t (&lo)[32],
                                                      const uint32_t (&hi)[32], int m0, int quad_in_tile, int row_tile,
-                                                     int nc, float alpha, float Tq, float c6T, uint32_t sbuf,
+                                                     int nc, int nc_dst, float alpha, float Tq, float c6T, uint32_t sbuf,
                                                      uint32_t sbias, int lane, uint32_t &amax2) {
+    const bool gelu = p.act != 0;
     if (lane == 0) ptx::tma_store_wait_read<0>();
     __syncwarp();
     uint32_t sfw = 0;
@@ -131,7 +133,7 @@ __device__ __forceinline__ void epilogue_quant_store(const CUtensorMap *tm_q, co
                 const uint32_t a1 = g < 4 ? lo[g * 8 + 2 * e + 1] : hi[(g - 4) * 8 + 2 * e + 1];
                 float y0 = fmaf(__uint_as_float(a0), alpha, __uint_as_float(bw[e] << 16));
                 float y1 = fmaf(__uint_as_float(a1), alpha, __uint_as_float(bw[e] & 0xFFFF0000u));
-                if (kOut == kOutQuantGelu) {
+                if (gelu) {
                     y0 = gelu_tanh(y0);
                     y1 = gelu_tanh(y1);
                 }
@@ -155,13 +157,13 @@ __device__ __forceinline__ void epilogue_quant_store(const CUtensorMap *tm_q, co
     if (unit_ok && row_tile * 128 < p.M) {
         // rows past M inside the last 128-row chunk are padding and read as 0
         if (m0 + lane >= p.M) sfw = 0;
-        const int64_t chunk = static_cast<int64_t>(row_tile) * (p.N >> 6) + (nc >> 6);
+        const int64_t chunk = static_cast<int64_t>(row_tile) * p.dest_chunks_k + (nc_dst >> 6);
         *reinterpret_cast<uint32_t *>(p.sf_out + chunk * 512 + lane * 16 + quad_in_tile * 4) = sfw;
     }
     ptx::fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) {
-        if (unit_ok && m0 < p.M) ptx::tma_store_2d(tm_q, nc >> 1, m0, sbuf);
+        if (unit_ok && m0 < p.M) ptx::tma_store_2d(tm_q, nc_dst >> 1, m0, sbuf);
         ptx::tma_store_commit();
     }
 }
@@ -171,8 +173,9 @@ __device__ __forceinline__ void epilogue_quant_store(const CUtensorMap *tm_q, co
 template <int kOut, bool kMx>
 __global__ void __launch_bounds__(kThreadsFp4, 1)
 gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                     const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_sfa,
-                     const __grid_constant__ CUtensorMap tm_sfb, const Params p) {
+                     const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ CUtensorMap tm_q,
+                     const __grid_constant__ CUtensorMap tm_sfa, const __grid_constant__ CUtensorMap tm_sfb,
+                     const Params p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
@@ -218,6 +221,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         ptx::prefetch_tmap(&tm_a);
         ptx::prefetch_tmap(&tm_b);
         ptx::prefetch_tmap(&tm_y);
+        ptx::prefetch_tmap(&tm_q);
         ptx::prefetch_tmap(&tm_sfa);
         ptx::prefetch_tmap(&tm_sfb);
     }
@@ -509,29 +513,32 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(ovl_bar);
             if (kTuning && (p.dbg & kDbgTrace) && warp == 2) SOL_TRACE(10, it);
-            if (kOut == kOutBf16)
+            // split mode decides per tile; the quantized part lands at a column offset of the destination
+            const bool as_bf16 = kOut == kOutBf16 || (kOut == kOutSplit && n0 < p.n_split);
+            const int dst_shift = kOut == kOutSplit ? p.dest_col0 - p.n_split : 0;
+            if (as_bf16)
                 epilogue_store(&tm_y, p, a_lo, a_hi, m0, n0 + first * 64, alpha, sbuf, sbias, lane);
             else
-                epilogue_quant_store<kOut>(&tm_y, p, a_lo, a_hi, m0, quad, row_tile, n0 + first * 64, alpha, Tq, c6T,
-                                           sbuf, sbias, lane, amax2);
+                epilogue_quant_store(&tm_q, p, a_lo, a_hi, m0, quad, row_tile, n0 + first * 64,
+                                     n0 + first * 64 + dst_shift, alpha, Tq, c6T, sbuf, sbias, lane, amax2);
             if (early) ptx::tmem_ld_32x32(t2 + shared_half, b_sh);
             ptx::tmem_ld_32x32(t2 + (shared_half ^ 32u), b_ot);
             ptx::tmem_ld_wait();
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(done_bar);
-            if (kOut == kOutBf16) {
+            if (as_bf16) {
                 if (x == 0)  // b_sh is the upper half
                     epilogue_store(&tm_y, p, b_ot, b_sh, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
                 else
                     epilogue_store(&tm_y, p, b_sh, b_ot, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
             } else {
                 if (x == 0)
-                    epilogue_quant_store<kOut>(&tm_y, p, b_ot, b_sh, m0, quad, row_tile, n0 + second * 64, alpha, Tq,
-                                               c6T, sbuf, sbias + 128, lane, amax2);
+                    epilogue_quant_store(&tm_q, p, b_ot, b_sh, m0, quad, row_tile, n0 + second * 64,
+                                         n0 + second * 64 + dst_shift, alpha, Tq, c6T, sbuf, sbias + 128, lane, amax2);
                 else
-                    epilogue_quant_store<kOut>(&tm_y, p, b_sh, b_ot, m0, quad, row_tile, n0 + second * 64, alpha, Tq,
-                                               c6T, sbuf, sbias + 128, lane, amax2);
+                    epilogue_quant_store(&tm_q, p, b_sh, b_ot, m0, quad, row_tile, n0 + second * 64,
+                                         n0 + second * 64 + dst_shift, alpha, Tq, c6T, sbuf, sbias + 128, lane, amax2);
             }
         }
         if (lane == 0) ptx::tma_store_wait_all<0>();
@@ -558,26 +565,39 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
 
 namespace {
 
+struct QuantOut {          // where a quantized output goes (kOutQuant, kOutSplit)
+    int act = 0;
+    const float *ts_out = nullptr;
+    void *hq = nullptr;
+    void *hsf = nullptr;
+    uint32_t *amax_out = nullptr;
+    int64_t n_split = 0;   // kOutSplit: columns [0, n_split) leave as BF16 through y / ldy
+    int64_t dest_K = 0;    // width of the destination tensor (its own N when not split)
+    int64_t dest_col0 = 0;
+};
+
 sol_status_t launch_pair256(int out_mode, bool mx, const void *xq, const void *xsf, const float *xts, const void *wq,
                             const void *wsf, const float *wts, const void *bias, void *y, int64_t ldy,
-                            const float *ts_out, void *hsf, uint32_t *amax_out, int64_t M, int64_t N, int64_t K,
-                            cudaStream_t stream, const DeviceInfo *dev) {
+                            const QuantOut &qo, int64_t M, int64_t N, int64_t K, cudaStream_t stream,
+                            const DeviceInfo *dev) {
     const uint64_t chunks_k = static_cast<uint64_t>(ceil_div(K, mx ? 128 : 64));
     const uint32_t box_k = mx ? 2 : 4;
-    CUtensorMap tm_a, tm_b, tm_y, tm_sfa, tm_sfb;
+    CUtensorMap tm_a, tm_b, tm_y, tm_q, tm_sfa, tm_sfb;
     bool ok = make_tmap_2d(&tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, xq, K / 2, M, K / 2, 128, kBM,
                            CU_TENSOR_MAP_SWIZZLE_128B) &&
               make_tmap_2d(&tm_b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, wq, K / 2, N, K / 2, 128, kBN / 2,
                            CU_TENSOR_MAP_SWIZZLE_128B) &&
               make_tmap_sf(&tm_sfa, xsf, chunks_k, static_cast<uint64_t>(ceil_div(M, 128)), 1, box_k) &&
               make_tmap_sf(&tm_sfb, wsf, chunks_k, static_cast<uint64_t>(ceil_div(N, 128)), 2, box_k);
-    if (out_mode == kOutBf16)
-        ok = ok && make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, N, M, ldy * 2, 64, 32,
-                                CU_TENSOR_MAP_SWIZZLE_128B);
-    else  // packed nibbles [M, N/2]: boxes of 32 rows x 32 bytes (64 columns)
-        ok = ok && make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, y, N / 2, M, N / 2, 32, 32,
+    if (out_mode != kOutQuant)  // BF16 output: all N columns, or the first n_split of them
+        ok = ok && make_tmap_2d(&tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, y, out_mode == kOutSplit ? qo.n_split : N, M,
+                                ldy * 2, 64, 32, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (out_mode != kOutBf16)   // packed nibbles [M, dest_K/2]: boxes of 32 rows x 32 bytes (64 columns)
+        ok = ok && make_tmap_2d(&tm_q, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, qo.hq, qo.dest_K / 2, M, qo.dest_K / 2, 32, 32,
                                 CU_TENSOR_MAP_SWIZZLE_NONE);
     if (!ok) return SOL_ERR_CUDA;
+    if (out_mode == kOutQuant) tm_y = tm_q;  // unused, but a valid descriptor for the prefetch
+    if (out_mode == kOutBf16) tm_q = tm_y;
     Params p{};
     p.sfa = static_cast<const uint8_t *>(xsf);
     p.sfb = static_cast<const uint8_t *>(wsf);
@@ -588,16 +608,20 @@ sol_status_t launch_pair256(int out_mode, bool mx, const void *xq, const void *x
     p.M = static_cast<int>(M);
     p.N = static_cast<int>(N);
     p.K = static_cast<int>(K);
-    p.sf_out = static_cast<uint8_t *>(hsf);
-    p.ts_out = ts_out;
-    p.amax_out = amax_out;
+    p.sf_out = static_cast<uint8_t *>(qo.hsf);
+    p.ts_out = qo.ts_out;
+    p.amax_out = qo.amax_out;
+    p.act = qo.act;
+    p.n_split = static_cast<int>(qo.n_split);
+    p.dest_col0 = static_cast<int>(qo.dest_col0);
+    p.dest_chunks_k = static_cast<int>(qo.dest_K >> 6);
 #ifdef SOL_TUNING
     if (const char *e = getenv("SOL_DBG")) p.dbg = static_cast<uint32_t>(atoi(e));
 #endif
     auto kern = mx ? gemm_pair_fp4_kernel<kOutBf16, true>
                 : out_mode == kOutBf16 ? gemm_pair_fp4_kernel<kOutBf16, false>
                 : out_mode == kOutQuant ? gemm_pair_fp4_kernel<kOutQuant, false>
-                                        : gemm_pair_fp4_kernel<kOutQuantGelu, false>;
+                                        : gemm_pair_fp4_kernel<kOutSplit, false>;
     static bool configured[4][64] = {};
     const int slot = mx ? 3 : out_mode;
     if (dev->device < 64 && !configured[slot][dev->device]) {
@@ -624,7 +648,7 @@ sol_status_t launch_pair256(int out_mode, bool mx, const void *xq, const void *x
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_y, tm_sfa, tm_sfb, p) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_b, tm_y, tm_q, tm_sfa, tm_sfb, p) != cudaSuccess) {
         cudaGetLastError();
         return SOL_ERR_CUDA;
     }
@@ -636,15 +660,14 @@ sol_status_t launch_pair256(int out_mode, bool mx, const void *xq, const void *x
 sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
                                   const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
                                   int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev) {
-    return launch_pair256(kOutBf16, false, xq, xsf, xts, wq, wsf, wts, bias, y, ldy, nullptr, nullptr, nullptr, M, N,
-                          K, stream, dev);
+    return launch_pair256(kOutBf16, false, xq, xsf, xts, wq, wsf, wts, bias, y, ldy, QuantOut{}, M, N, K, stream, dev);
 }
 
 sol_status_t launch_pair256_mxfp4(const void *xq, const void *xsf, const void *wq, const void *wsf, const void *bias,
                                   void *y, int64_t M, int64_t N, int64_t K, int64_t ldy, cudaStream_t stream,
                                   const DeviceInfo *dev) {
-    return launch_pair256(kOutBf16, true, xq, xsf, nullptr, wq, wsf, nullptr, bias, y, ldy, nullptr, nullptr, nullptr,
-                          M, N, K, stream, dev);
+    return launch_pair256(kOutBf16, true, xq, xsf, nullptr, wq, wsf, nullptr, bias, y, ldy, QuantOut{}, M, N, K, stream,
+                          dev);
 }
 
 sol_status_t launch_pair256_nvfp4_quant_out(const void *xq, const void *xsf, const float *xts, const void *wq,
@@ -652,8 +675,32 @@ sol_status_t launch_pair256_nvfp4_quant_out(const void *xq, const void *xsf, con
                                             const float *ts_out, void *hq, void *hsf, uint32_t *amax_out,
                                             int64_t M, int64_t N, int64_t K, cudaStream_t stream,
                                             const DeviceInfo *dev) {
-    return launch_pair256(act == 1 ? kOutQuantGelu : kOutQuant, false, xq, xsf, xts, wq, wsf, wts, bias, hq, 0, ts_out, hsf,
-                          amax_out, M, N, K, stream, dev);
+    QuantOut qo;
+    qo.act = act;
+    qo.ts_out = ts_out;
+    qo.hq = hq;
+    qo.hsf = hsf;
+    qo.amax_out = amax_out;
+    qo.dest_K = N;
+    return launch_pair256(kOutQuant, false, xq, xsf, xts, wq, wsf, wts, bias, nullptr, 0, qo, M, N, K, stream, dev);
+}
+
+sol_status_t launch_pair256_nvfp4_split_out(const void *xq, const void *xsf, const float *xts, const void *wq,
+                                            const void *wsf, const float *wts, const void *bias, void *y_bf16,
+                                            int64_t ldy, int64_t n_split, int act, const float *ts_out, void *hq,
+                                            void *hsf, int64_t dest_K, int64_t dest_col0, uint32_t *amax_out,
+                                            int64_t M, int64_t N, int64_t K, cudaStream_t stream,
+                                            const DeviceInfo *dev) {
+    QuantOut qo;
+    qo.act = act;
+    qo.ts_out = ts_out;
+    qo.hq = hq;
+    qo.hsf = hsf;
+    qo.amax_out = amax_out;
+    qo.n_split = n_split;
+    qo.dest_K = dest_K;
+    qo.dest_col0 = dest_col0;
+    return launch_pair256(kOutSplit, false, xq, xsf, xts, wq, wsf, wts, bias, y_bf16, ldy, qo, M, N, K, stream, dev);
 }
 
 }  // namespace gemm

@@ -49,6 +49,16 @@ __device__ __forceinline__ uint32_t quantize8(const uint4 &v, float rcp) {
     return qmath::quantize8(v.x, v.y, v.z, v.w, rcp);
 }
 
+// Where the quantized tensor lands: normally a dense [rows, K/2] nibble matrix and its own scale
+// buffer; for a slice of a wider tensor (one part of a concatenated activation) the row pitch, the
+// byte column and the scale chunk column of the destination.
+struct QuantDest {
+    int64_t q_pitch;       // bytes between rows of the nibble matrix
+    int64_t q_col0;        // first byte column
+    int64_t sf_chunks_k;   // scale chunks per 128-row tile in the destination (chunked layout)
+    int64_t sf_chunk0;     // first chunk column
+};
+
 // One block quantizes a 128-row x 256-element tile.  A thread owns whole scale blocks (16
 // elements = two 16-byte loads, one 8-byte store, one scale byte), so the scale arithmetic runs
 // once per 16 elements: the kernel has to stay under ~8 instructions per element to be bound
@@ -59,7 +69,7 @@ __device__ __forceinline__ uint32_t quantize8(const uint4 &v, float rcp) {
 template <bool kSwizzled>
 __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
                                               const float *tscale, const float *amax, float *tscale_out,
-                                              uint8_t *__restrict__ q, uint8_t *__restrict__ sf) {
+                                              uint8_t *__restrict__ q, uint8_t *__restrict__ sf, const QuantDest dst) {
     __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kTileK / 16)];  // 2 KB = 4 chunks
     // 1 / (float(sb) * T) for every scale byte: d takes at most 127 values per tensor, so the decode,
     // the multiplication and the IEEE reciprocal run once per thread block instead of once per scale block
@@ -113,7 +123,7 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
             packed.x = quantize8(lo[i], rcp);
             packed.y = quantize8(hi[i], rcp);
             if (k_ok && r < rows) {
-                __stcs(reinterpret_cast<uint2 *>(q + r * (K >> 1) + (k >> 1)), packed);
+                __stcs(reinterpret_cast<uint2 *>(q + r * dst.q_pitch + dst.q_col0 + (k >> 1)), packed);
                 if (kSwizzled) {
                     sf_tile[(b >> 2) * 512 + (rl & 31) * 16 + (rl >> 5) * 4 + (b & 3)] = static_cast<uint8_t>(sb);
                 } else {
@@ -131,9 +141,9 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
             const int cidx = threadIdx.x >> 5;
             const int64_t kc = static_cast<int64_t>(blockIdx.x) * 4 + cidx;
             if (kc < chunks_k) {
-                uint8_t *dst = sf + (static_cast<int64_t>(blockIdx.y) * chunks_k + kc) * 512 +
+                uint8_t *out = sf + (static_cast<int64_t>(blockIdx.y) * dst.sf_chunks_k + dst.sf_chunk0 + kc) * 512 +
                                (threadIdx.x & 31) * 16;
-                *reinterpret_cast<uint4 *>(dst) = reinterpret_cast<const uint4 *>(sf_tile)[threadIdx.x];
+                *reinterpret_cast<uint4 *>(out) = reinterpret_cast<const uint4 *>(sf_tile)[threadIdx.x];
             }
         }
     }
@@ -143,8 +153,8 @@ template <bool kSwizzled>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
                 const float *tscale, const float *amax, float *tscale_out, uint8_t *__restrict__ q,
-                uint8_t *__restrict__ sf) {
-    quantize_tile<kSwizzled>(x, rows, K, ld, tscale, amax, tscale_out, q, sf);
+                uint8_t *__restrict__ sf, const QuantDest dst) {
+    quantize_tile<kSwizzled>(x, rows, K, ld, tscale, amax, tscale_out, q, sf, dst);
 }
 
 // The same over a group of equally shaped dense tensors, one per blockIdx.z, each with its own
@@ -153,7 +163,8 @@ template <bool kSwizzled>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_group_kernel(const __grid_constant__ QuantGroup g, int64_t rows, int64_t K) {
     const int z = blockIdx.z;
-    quantize_tile<kSwizzled>(g.x[z], rows, K, K, nullptr, g.scale_words[z] + 1, g.scale_words[z], g.q[z], g.sf[z]);
+    const QuantDest dst = {K >> 1, 0, ((K >> 4) + 3) >> 2, 0};
+    quantize_tile<kSwizzled>(g.x[z], rows, K, K, nullptr, g.scale_words[z] + 1, g.scale_words[z], g.q[z], g.sf[z], dst);
 }
 
 // MXFP4 quantizer (the OCP format Section 2 sets beside NVFP4): 32 elements share one E8M0 scale
@@ -296,7 +307,8 @@ sol_status_t launch_amax_bits(const void *x, int64_t rows, int64_t K, int64_t ld
 // their first global access.
 sol_status_t launch_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale,
                                 const float *amax, float *tscale_out, void *q, void *sf,
-                                sol_sf_layout_t layout, cudaStream_t stream) {
+                                sol_sf_layout_t layout, cudaStream_t stream, const QuantDest *dest = nullptr) {
+    const QuantDest dst = dest != nullptr ? *dest : QuantDest{K >> 1, 0, ((K >> 4) + 3) >> 2, 0};
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(ceil_div(K, kTileK)), static_cast<unsigned>(ceil_div(rows, kTileRows)));
     cfg.blockDim = dim3(kQuantThreads);
@@ -309,7 +321,7 @@ sol_status_t launch_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t 
     cfg.numAttrs = 1;
     auto kern = layout == SOL_SF_SWIZZLED_128x4 ? quantize_kernel<true> : quantize_kernel<false>;
     if (cudaLaunchKernelEx(&cfg, kern, static_cast<const uint16_t *>(x), rows, K, ld, tscale, amax, tscale_out,
-                           static_cast<uint8_t *>(q), static_cast<uint8_t *>(sf)) != cudaSuccess) {
+                           static_cast<uint8_t *>(q), static_cast<uint8_t *>(sf), dst) != cudaSuccess) {
         cudaGetLastError();
         return SOL_ERR_CUDA;
     }
@@ -317,6 +329,12 @@ sol_status_t launch_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t 
 }
 
 }  // namespace
+
+sol_status_t launch_quantize_into(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale, void *q,
+                                  void *sf, int64_t dest_K, int64_t dest_col0, cudaStream_t stream) {
+    const QuantDest dst = {dest_K >> 1, dest_col0 >> 1, dest_K >> 6, dest_col0 >> 6};
+    return launch_quantize_ex(x, rows, K, ld, tscale, nullptr, nullptr, q, sf, SOL_SF_SWIZZLED_128x4, stream, &dst);
+}
 
 sol_status_t launch_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *tscale_out,
                          cudaStream_t stream, const DeviceInfo *dev) {

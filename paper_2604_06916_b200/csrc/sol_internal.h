@@ -67,6 +67,10 @@ sol_status_t launch_lora_merge(const MergeGroup &g, int count, int64_t ldw, int6
 sol_status_t launch_quantize_group(const QuantGroup &g, int count, int64_t rows, int64_t K, sol_sf_layout_t layout,
                                    cudaStream_t stream);
 int lora_max_rank();
+// Quantizes x [rows, K] into columns [dest_col0, dest_col0 + K) of a wider quantized tensor [rows, dest_K]
+// (chunked scale layout; K, dest_K and dest_col0 multiples of 64).
+sol_status_t launch_quantize_into(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale, void *q,
+                                  void *sf, int64_t dest_K, int64_t dest_col0, cudaStream_t stream);
 sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
                                    sol_sf_layout_t layout, cudaStream_t stream);
 // Stage-1 selection and rank-consistency metrics (one block per prompt).

@@ -112,6 +112,16 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.solrl_rank_consistency(p, p, 2, 1, 1, p, None, None) == SHAPE
     assert L.solrl_rank_consistency(p, p, 2, 8, 9, p, None, None) == SHAPE
     assert L.solrl_rank_consistency(p, p, 2, 8, 4, p + 4, None, None) == ALIGN
+    # split output and quantize-into-slice
+    assert L.nvfp4_linear_split_out(p, p, p, p, p, p, None, None, 256, 256, 0, p, p, p, 256, 0, None, 4, 512, 64, None) == NULLP
+    assert L.nvfp4_linear_split_out(p, p, p, p, p, p, None, p, 256, 128, 0, p, p, p, 256, 0, None, 4, 512, 64, None) == SHAPE   # n_split % 256
+    assert L.nvfp4_linear_split_out(p, p, p, p, p, p, None, p, 256, 256, 0, p, p, p, 256, 64, None, 4, 512, 64, None) == SHAPE  # part does not fit
+    assert L.nvfp4_linear_split_out(p, p, p, p, p, p, None, p, 256, 256, 0, p, p, p, 320, 32, None, 4, 512, 64, None) == SHAPE  # dest_col0 % 64
+    assert L.nvfp4_linear_split_out(p, p, p, p, p, p, None, p, 256, 256, 0, p, p + 8, p, 256, 0, None, 4, 512, 64, None) == ALIGN
+    assert L.nvfp4_quantize_into(p, 4, 64, 64, p, None, p, 128, 0, None) == NULLP
+    assert L.nvfp4_quantize_into(p, 4, 96, 96, p, p, p, 192, 0, None) == SHAPE     # K % 64
+    assert L.nvfp4_quantize_into(p, 4, 64, 64, p, p, p, 128, 128, None) == SHAPE   # past the end
+    assert L.nvfp4_quantize_into(p, 4, 64, 64, p, p + 4, p, 128, 0, None) == ALIGN
     # MXFP4
     assert L.sol_mxfp4_scale_bytes(256, 512, 0) == 256 * 16 and L.sol_mxfp4_scale_bytes(256, 512, 1) == 2 * 4 * 512
     assert L.sol_mxfp4_scale_bytes(130, 160, 1) == 2 * 2 * 512 and L.sol_mxfp4_scale_bytes(4, 48, 1) == 0

@@ -162,3 +162,104 @@ def test_rejects_bad_arguments(B):
         B._check(B.lib().nvfp4_linear_quantized_out(z.data_ptr(), z.data_ptr(), t.data_ptr(), z.data_ptr(), z.data_ptr(),
                                                     t.data_ptr(), None, 0, t.data_ptr(), z.data_ptr(), z.data_ptr(), None,
                                                     64, 96, 64, None), "nvfp4_linear_quantized_out")
+
+
+def test_quantize_into_slice_bit_exact(B):
+    # two BF16 parts quantized into one wider tensor equal the oracle's quantizer on their concatenation
+    g = torch.Generator(device="cuda").manual_seed(21)
+    M, K1, K2 = 300, 192, 448
+    X1 = workloads.make_activation("student_t", M, K1, g, "cuda")
+    X2 = workloads.make_activation("outlier", M, K2, g, "cuda")
+    cat_bits = np.concatenate([bits_of(X1), bits_of(X2)], axis=1)
+    T = oracle.tensor_scale(cat_bits)
+    want_q, want_sf = oracle.quantize(cat_bits, T)
+    K = K1 + K2
+    hq = torch.full((M, K // 2), 0xEE, dtype=torch.uint8, device="cuda")
+    hsf = torch.zeros(B.scale_bytes(M, K), dtype=torch.uint8, device="cuda")
+    ts = torch.tensor([T], dtype=torch.float32, device="cuda")
+    B.nvfp4_quantize_into(X2, ts, (hq, hsf), K1)
+    assert torch.all(hq[:, : K1 // 2] == 0xEE)                 # the other column range is untouched
+    B.nvfp4_quantize_into(X1, ts, (hq, hsf), 0)
+    assert np.array_equal(hq.cpu().numpy(), want_q)
+    assert np.array_equal(hsf.cpu().numpy(), oracle.sf_swizzle(want_sf, K))
+
+
+@pytest.mark.parametrize("M,N,n_split,K,col0,dest_K", [(256, 512, 256, 64, 0, 256), (300, 832, 256, 256, 128, 768),
+                                                       (520, 1024, 512, 512, 64, 640)])
+def test_split_output_integer_exact_bit_for_bit(B, M, N, n_split, K, col0, dest_K):
+    rng = np.random.default_rng(M + N + K)
+    qx = rng.integers(0, 256, size=(M, K // 2), dtype=np.uint8)
+    qw = rng.integers(0, 256, size=(N, K // 2), dtype=np.uint8)
+    sfx = ((rng.integers(-2, 3, size=(M, K // 16)) + 7) << 3).astype(np.uint8)
+    sfw = ((rng.integers(-2, 3, size=(N, K // 16)) + 7) << 3).astype(np.uint8)
+    Y = oracle.nvfp4_linear(qx, sfx, 1.0, qw, sfw, 1.0)
+    h = oracle.round_bf16(Y[:, n_split:])
+    T_out = float(oracle.tensor_scale(h))
+    q_star, sf_star = oracle.quantize(h, T_out)
+    part = N - n_split
+    hq = torch.full((M, dest_K // 2), 0xEE, dtype=torch.uint8, device="cuda")
+    hsf = torch.full((B.scale_bytes(M, dest_K),), 0xDD, dtype=torch.uint8, device="cuda")
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    y = B.nvfp4_linear_split_out(*upload(qx, sfx, K, 1.0), *upload(qw, sfw, K, 1.0), None, n_split, B.ACT_NONE,
+                                 torch.tensor([T_out], dtype=torch.float32, device="cuda"), (hq, hsf), col0,
+                                 amax_out=amax)
+    B.sol_last_device_status()
+    assert np.array_equal(bits_of(y), oracle.round_bf16(Y[:, :n_split]))
+    got_q = hq.cpu().numpy()
+    assert np.array_equal(got_q[:, col0 // 2:(col0 + part) // 2], q_star)
+    untouched = np.ones(dest_K // 2, bool)
+    untouched[col0 // 2:(col0 + part) // 2] = False
+    assert np.all(got_q[:, untouched] == 0xEE)
+    sf_all = unswizzle_rows(hsf.cpu().numpy(), np.arange(M), dest_K)
+    assert np.array_equal(sf_all[:, col0 // 16:(col0 + part) // 16], sf_star)
+    mask = np.ones(dest_K // 16, bool)
+    mask[col0 // 16:(col0 + part) // 16] = False
+    assert np.all(sf_all[:, mask] == 0xDD)
+    assert amax.item() == np.abs(oracle.bits_to_f64(h)).max()
+
+
+def test_single_stream_block_chain_against_oracle(B):
+    # first linear: q/k/v part in BF16 + GELU(MLP part) quantized into the concat buffer at column 256;
+    # a BF16 "attention output" quantized into columns [0, 256); second linear on the concat buffer
+    g = torch.Generator(device="cuda").manual_seed(33)
+    M, K, n_split, n_mlp, attn_w, N2 = 384, 512, 768, 1024, 256, 256
+    N = n_split + n_mlp
+    X = workloads.make_activation("student_t", M, K, g, "cuda")
+    W1 = (torch.randn(N, K, generator=g, device="cuda") * K ** -0.5).to(torch.bfloat16)
+    b1 = (torch.randn(N, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    attn = (torch.randn(M, attn_w, generator=g, device="cuda") * 0.5).to(torch.bfloat16)
+    W2 = (torch.randn(N2, attn_w + n_mlp, generator=g, device="cuda") * (attn_w + n_mlp) ** -0.5).to(torch.bfloat16)
+    xb, w1b = bits_of(X), bits_of(W1)
+    Tx, Tw1 = oracle.tensor_scale(xb), oracle.tensor_scale(w1b)
+    qx, sfx = oracle.quantize(xb, Tx)
+    qw1, sfw1 = oracle.quantize(w1b, Tw1)
+    Y1 = oracle.nvfp4_linear(qx, sfx, Tx, qw1, sfw1, Tw1, bits_of(b1))
+    H = oracle.gelu_tanh(Y1[:, n_split:])
+    cat = np.concatenate([bits_of(attn), oracle.round_bf16(H)], axis=1)
+    T_cat = float(oracle.tensor_scale(cat))
+    q_cat, sf_cat = oracle.quantize(cat, T_cat)
+    dest_K = attn_w + n_mlp
+    hq = torch.zeros((M, dest_K // 2), dtype=torch.uint8, device="cuda")
+    hsf = torch.zeros(B.scale_bytes(M, dest_K), dtype=torch.uint8, device="cuda")
+    ts = torch.tensor([T_cat], dtype=torch.float32, device="cuda")
+    y_qkv = B.nvfp4_linear_split_out(*upload(qx, sfx, K, Tx), *upload(qw1, sfw1, K, Tw1), b1, n_split, B.ACT_GELU_TANH, ts,
+                                     (hq, hsf), attn_w)
+    B.nvfp4_quantize_into(attn, ts, (hq, hsf), 0)
+    B.sol_last_device_status()
+    from tests.helpers import check_linear
+    check_linear(bits_of(y_qkv), Y1[:, :n_split], "qkv part")
+    got_q = hq.cpu().numpy()
+    sf_rm = unswizzle_rows(hsf.cpu().numpy(), np.arange(M), dest_K)
+    assert np.array_equal(got_q[:, : attn_w // 2], q_cat[:, : attn_w // 2])               # BF16 part: bit-exact
+    assert np.array_equal(sf_rm[:, : attn_w // 16], sf_cat[:, : attn_w // 16])
+    check_valid(got_q[:, attn_w // 2:], sf_rm[:, attn_w // 16:], Y1[:, n_split:], H, q_cat[:, attn_w // 2:],
+                sf_cat[:, attn_w // 16:], T_cat, 0.99, 1)
+    # second linear on the concat buffer against the oracle's chain
+    w2q, w2sf, w2ts = B.nvfp4_quantize_weight(W2)
+    y2 = B.nvfp4_linear(hq, hsf, ts, w2q, w2sf, w2ts)
+    Tw2 = oracle.tensor_scale(bits_of(W2))
+    qw2, sfw2 = oracle.quantize(bits_of(W2), Tw2)
+    Y2 = oracle.nvfp4_linear(q_cat, sf_cat, T_cat, qw2, sfw2, Tw2)
+    err = np.abs(oracle.bits_to_f64(bits_of(y2)) - Y2)
+    rms = np.sqrt(np.mean(Y2 * Y2, axis=1, keepdims=True))
+    assert np.all(err <= 2.0 ** -4 * np.abs(Y2) + 0.1 * rms) and np.mean(err / rms) < 0.01
