@@ -30,7 +30,7 @@ NOMINAL_BF16_TFLOPS = 2250.0    # vendor dense BF16 peak
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (None until a capture of the current kernel exists)
-# ncu (profiles/gemm_pair_and_quantizer_flux_d_proj.md), d_proj launch: GEMM 69.1 MB read + 172.7 MB
+# ncu capture of one d_proj launch (summaries under profiles/): GEMM 69.1 MB read + 171.6 MB
 # written for 295.5 MB algorithmic (Y partly still dirty in L2 at kernel end); quantizer 226.5 + 26.5 MB
 # for 290.2 MB algorithmic.  Scaled to all six layers by the algorithmic bytes (traffic is proportional).
 NCU_TRAFFIC_RATIO = {"gemm": (69.06 + 171.63) / 295.5, "quantize": (226.53 + 26.43) / 290.2}
