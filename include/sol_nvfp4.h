@@ -236,6 +236,23 @@ sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *
                                    size_t workspace_bytes, void *stream);
 
 /*
+ * The fused entry without the amax pass ("delayed" tensor scale): X is quantized with the T the
+ * caller carries over from an earlier call on the same activation stream, and the amax of THIS X
+ * is collected by the quantizer as a by-product (it computes every block maximum anyway), so the
+ * second HBM read of X disappears.  A T that has become too small only saturates more block scales.
+ *   scale_state  two floats (device, 8-byte aligned): [0] = T used by this call (> 0; read only),
+ *                [1] = running max|x| as an FP32 value, raised by this call with an atomic max
+ *   sol_roll_tensor_scale(state): [0] <- max|x| / 2688 (1 if it is 0), [1] <- 0 -- one tiny kernel,
+ *                called between denoising steps (or whenever the caller wants T refreshed)
+ * Given the same T the result is bit-identical to nvfp4_quantize + nvfp4_linear.
+ */
+sol_status_t nvfp4_quantize_linear_delayed(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,
+                                           const float *w_tscale, const void *bias_bf16, void *y_bf16, int64_t M,
+                                           int64_t N, int64_t K, int64_t ldy, float *scale_state, void *workspace,
+                                           size_t workspace_bytes, void *stream);
+sol_status_t sol_roll_tensor_scale(float *scale_state, void *stream);
+
+/*
  * The fused entry for HOST activations and outputs (the end-to-end path a caller with data in host
  * memory takes): copies X host -> x_dev, runs nvfp4_quantize_linear, copies y_dev -> Y host, all
  * queued on `stream` (truly asynchronous only if the host buffers are pinned).

@@ -25,6 +25,7 @@ EXPORTS = [
     "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch", "nvfp4_linear_quantized_out",
     "solrl_select_contrastive", "solrl_rank_consistency", "sol_mxfp4_scale_bytes", "mxfp4_quantize",
     "mxfp4_linear", "nvfp4_linear_split_out", "nvfp4_quantize_into",
+    "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale",
 ]
 
 _lib = None
@@ -87,6 +88,9 @@ def lib() -> ctypes.CDLL:
                                          i64, i64, vp]
     L.nvfp4_quantize_into.restype = i32
     L.nvfp4_quantize_into.argtypes = [vp, i64, i64, i64, vp, vp, vp, i64, i64, vp]
+    L.nvfp4_quantize_linear_delayed.restype = i32
+    L.nvfp4_quantize_linear_delayed.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, sz, vp]
+    L.sol_roll_tensor_scale.restype, L.sol_roll_tensor_scale.argtypes = i32, [vp, vp]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -275,6 +279,26 @@ def nvfp4_quantize_into(x: torch.Tensor, tensor_scale: torch.Tensor, dest, dest_
     hq, hsf = dest
     _check(lib().nvfp4_quantize_into(_ptr(x), M, K, x.stride(0), _ptr(tensor_scale), _ptr(hq), _ptr(hsf),
                                      hq.shape[1] * 2, dest_col0, _stream()), "nvfp4_quantize_into")
+
+
+def nvfp4_quantize_linear_delayed(x, wq, wsf, w_tscale, bias, scale_state: torch.Tensor,
+                                  workspace: torch.Tensor | None = None, out: torch.Tensor | None = None):
+    """Fused quantize + NVFP4 linear with T = scale_state[0]; max|x| is accumulated into scale_state[1]."""
+    _need_2d_bf16(x, "x")
+    M, K = x.shape
+    N = wq.shape[0]
+    if workspace is None:
+        workspace = torch.empty(linear_workspace_bytes(M, N, K), dtype=torch.uint8, device=x.device)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    _check(lib().nvfp4_quantize_linear_delayed(_ptr(x), x.stride(0), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
+                                               _ptr(out), M, N, K, out.stride(0), _ptr(scale_state), _ptr(workspace),
+                                               workspace.numel(), _stream()), "nvfp4_quantize_linear_delayed")
+    return out
+
+
+def sol_roll_tensor_scale(scale_state: torch.Tensor):
+    _check(lib().sol_roll_tensor_scale(_ptr(scale_state), _stream()), "sol_roll_tensor_scale")
 
 
 def mxfp4_scale_bytes(rows: int, K: int, layout: int = SF_SWIZZLED_128x4) -> int:

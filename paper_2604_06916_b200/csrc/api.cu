@@ -471,6 +471,43 @@ sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *
     return launch_gemm_nvfp4(xq, xsf, xts, wq, wsf, w_tscale, bias_bf16, y_bf16, M, N, K, ldy, s, dev);
 }
 
+sol_status_t nvfp4_quantize_linear_delayed(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,
+                                           const float *w_tscale, const void *bias_bf16, void *y_bf16, int64_t M,
+                                           int64_t N, int64_t K, int64_t ldy, float *scale_state, void *workspace,
+                                           size_t workspace_bytes, void *stream) {
+    if (x_bf16 == nullptr || wq == nullptr || wsf == nullptr || w_tscale == nullptr || y_bf16 == nullptr ||
+        workspace == nullptr || scale_state == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    sol_status_t st = check_linear_common(bias_bf16, y_bf16, M, N, K, ldy);
+    if (st != SOL_OK) return st;
+    if (ldx < K) return SOL_ERR_BAD_SHAPE;
+    if (!aligned16(x_bf16) || ldx % 8 != 0 || !aligned16(wq) || !aligned16(wsf) ||
+        (reinterpret_cast<uintptr_t>(w_tscale) & 3u) || (reinterpret_cast<uintptr_t>(workspace) & 255u) ||
+        (reinterpret_cast<uintptr_t>(scale_state) & 7u))
+        return SOL_ERR_ALIGNMENT;
+    if (workspace_bytes < sol_nvfp4_linear_workspace_bytes(M, N, K)) return SOL_ERR_WORKSPACE_TOO_SMALL;
+    const DeviceInfo *dev = nullptr;
+    st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    uint8_t *xq = ws;
+    uint8_t *xsf = xq + align256(sol_nvfp4_data_bytes(M, K));
+    st = launch_quantize_tracking(x_bf16, M, K, ldx, scale_state, xq, xsf, reinterpret_cast<uint32_t *>(scale_state + 1),
+                                  s);
+    if (st != SOL_OK) return st;
+    return launch_gemm_nvfp4(xq, xsf, scale_state, wq, wsf, w_tscale, bias_bf16, y_bf16, M, N, K, ldy, s, dev);
+}
+
+sol_status_t sol_roll_tensor_scale(float *scale_state, void *stream) {
+    if (scale_state == nullptr) return SOL_ERR_NULL_POINTER;
+    if (reinterpret_cast<uintptr_t>(scale_state) & 7u) return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_roll_scale(scale_state, static_cast<cudaStream_t>(stream));
+}
+
 sol_status_t nvfp4_quantize_linear_host(const void *x_host, int64_t ldx, const void *wq, const void *wsf,
                                         const float *w_tscale, const void *bias_bf16, void *y_host, int64_t M,
                                         int64_t N, int64_t K, int64_t ldy, void *x_dev, void *y_dev,

@@ -57,6 +57,7 @@ struct QuantDest {
     int64_t q_col0;        // first byte column
     int64_t sf_chunks_k;   // scale chunks per 128-row tile in the destination (chunked layout)
     int64_t sf_chunk0;     // first chunk column
+    uint32_t *amax_track;  // nullable: running max|x| of the quantized tensor as FP32 bits (atomicMax)
 };
 
 // One block quantizes a 128-row x 256-element tile.  A thread owns whole scale blocks (16
@@ -98,6 +99,7 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
     }
     __syncthreads();
 
+    uint32_t seen_max = 0;  // BF16 magnitude bits of the largest element this thread has quantized
 #pragma unroll 1
     for (int batch = 0; batch < kBlocksPerThread / kBatch; ++batch) {
         uint4 lo[kBatch], hi[kBatch];
@@ -115,7 +117,9 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
         for (int i = 0; i < kBatch; ++i) {
             const int rl = r0 + 16 * (batch * kBatch + i);  // row inside the tile
             const int64_t r = row0 + rl;
-            const float a = __uint_as_float(abs_max_bits(lo[i], hi[i]) << 16);
+            const uint32_t abits = abs_max_bits(lo[i], hi[i]);
+            seen_max = max(seen_max, abits);
+            const float a = __uint_as_float(abits << 16);
             const float sv = __fdiv_rn(a, c);
             const uint32_t sb = f32_to_e4m3_sat(sv);
             const float rcp = rcp_tab[sb];
@@ -147,6 +151,17 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
             }
         }
     }
+    if (dst.amax_track != nullptr) {  // the tensor's amax as a by-product, for the next call's tensor scale
+        __shared__ uint32_t warp_seen[kQuantThreads / 32];
+        seen_max = __reduce_max_sync(0xFFFFFFFFu, seen_max);
+        if ((threadIdx.x & 31) == 0) warp_seen[threadIdx.x >> 5] = seen_max;
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            uint32_t m = threadIdx.x < kQuantThreads / 32 ? warp_seen[threadIdx.x] : 0;
+            m = __reduce_max_sync(0xFFFFFFFFu, m);
+            if (threadIdx.x == 0 && m) atomicMax(dst.amax_track, m << 16);
+        }
+    }
 }
 
 template <bool kSwizzled>
@@ -163,7 +178,7 @@ template <bool kSwizzled>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_group_kernel(const __grid_constant__ QuantGroup g, int64_t rows, int64_t K) {
     const int z = blockIdx.z;
-    const QuantDest dst = {K >> 1, 0, ((K >> 4) + 3) >> 2, 0};
+    const QuantDest dst = {K >> 1, 0, ((K >> 4) + 3) >> 2, 0, nullptr};
     quantize_tile<kSwizzled>(g.x[z], rows, K, K, nullptr, g.scale_words[z] + 1, g.scale_words[z], g.q[z], g.sf[z], dst);
 }
 
@@ -308,7 +323,7 @@ sol_status_t launch_amax_bits(const void *x, int64_t rows, int64_t K, int64_t ld
 sol_status_t launch_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale,
                                 const float *amax, float *tscale_out, void *q, void *sf,
                                 sol_sf_layout_t layout, cudaStream_t stream, const QuantDest *dest = nullptr) {
-    const QuantDest dst = dest != nullptr ? *dest : QuantDest{K >> 1, 0, ((K >> 4) + 3) >> 2, 0};
+    const QuantDest dst = dest != nullptr ? *dest : QuantDest{K >> 1, 0, ((K >> 4) + 3) >> 2, 0, nullptr};
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(ceil_div(K, kTileK)), static_cast<unsigned>(ceil_div(rows, kTileRows)));
     cfg.blockDim = dim3(kQuantThreads);
@@ -332,8 +347,27 @@ sol_status_t launch_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t 
 
 sol_status_t launch_quantize_into(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale, void *q,
                                   void *sf, int64_t dest_K, int64_t dest_col0, cudaStream_t stream) {
-    const QuantDest dst = {dest_K >> 1, dest_col0 >> 1, dest_K >> 6, dest_col0 >> 6};
+    const QuantDest dst = {dest_K >> 1, dest_col0 >> 1, dest_K >> 6, dest_col0 >> 6, nullptr};
     return launch_quantize_ex(x, rows, K, ld, tscale, nullptr, nullptr, q, sf, SOL_SF_SWIZZLED_128x4, stream, &dst);
+}
+
+sol_status_t launch_quantize_tracking(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale, void *q,
+                                      void *sf, uint32_t *amax_track, cudaStream_t stream) {
+    const QuantDest dst = {K >> 1, 0, ((K >> 4) + 3) >> 2, 0, amax_track};
+    return launch_quantize_ex(x, rows, K, ld, tscale, nullptr, nullptr, q, sf, SOL_SF_SWIZZLED_128x4, stream, &dst);
+}
+
+namespace {
+// state[0] = T derived from the amax collected in state[1]; state[1] = 0 for the next window
+__global__ void roll_scale_kernel(float *state) {
+    state[0] = tensor_scale_from_amax(state[1]);
+    state[1] = 0.0f;
+}
+}  // namespace
+
+sol_status_t launch_roll_scale(float *state, cudaStream_t stream) {
+    roll_scale_kernel<<<1, 1, 0, stream>>>(state);
+    return launch_status();
 }
 
 sol_status_t launch_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *tscale_out,

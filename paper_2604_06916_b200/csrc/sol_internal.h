@@ -71,6 +71,11 @@ int lora_max_rank();
 // (chunked scale layout; K, dest_K and dest_col0 multiples of 64).
 sol_status_t launch_quantize_into(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale, void *q,
                                   void *sf, int64_t dest_K, int64_t dest_col0, cudaStream_t stream);
+// Quantizer with a caller-supplied T that also collects max|x| into *amax_track (atomicMax on FP32 bits).
+sol_status_t launch_quantize_tracking(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale, void *q,
+                                      void *sf, uint32_t *amax_track, cudaStream_t stream);
+// state[0] <- T(state[1]); state[1] <- 0.
+sol_status_t launch_roll_scale(float *state, cudaStream_t stream);
 sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
                                    sol_sf_layout_t layout, cudaStream_t stream);
 // Stage-1 selection and rank-consistency metrics (one block per prompt).

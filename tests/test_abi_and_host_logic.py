@@ -122,6 +122,11 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.nvfp4_quantize_into(p, 4, 96, 96, p, p, p, 192, 0, None) == SHAPE     # K % 64
     assert L.nvfp4_quantize_into(p, 4, 64, 64, p, p, p, 128, 128, None) == SHAPE   # past the end
     assert L.nvfp4_quantize_into(p, 4, 64, 64, p, p + 4, p, 128, 0, None) == ALIGN
+    # delayed tensor scale
+    assert L.nvfp4_quantize_linear_delayed(p, 64, p, p, p, None, p, 4, 8, 64, 8, None, p, 1 << 20, None) == NULLP
+    assert L.nvfp4_quantize_linear_delayed(p, 64, p, p, p, None, p, 4, 8, 64, 8, p + 4, p, 1 << 20, None) == ALIGN
+    assert L.nvfp4_quantize_linear_delayed(p, 64, p, p, p, None, p, 4, 8, 64, 8, p, p, 16, None) == WS
+    assert L.sol_roll_tensor_scale(None, None) == NULLP
     # MXFP4
     assert L.sol_mxfp4_scale_bytes(256, 512, 0) == 256 * 16 and L.sol_mxfp4_scale_bytes(256, 512, 1) == 2 * 4 * 512
     assert L.sol_mxfp4_scale_bytes(130, 160, 1) == 2 * 2 * 512 and L.sol_mxfp4_scale_bytes(4, 48, 1) == 0

@@ -216,3 +216,24 @@ def test_flux_layers_every_output_against_library_matmul_screen(B, index):
         assert bool((err <= tol).all()), f"rows {r0}..: {(err > tol).sum().item()} outputs off"
         worst = max(worst, float((err / tol.clamp_min(1e-30)).max()))
     assert worst <= 1.0
+
+
+def test_delayed_scale_entry(B):
+    # with the same T the delayed entry equals quantize + linear bit for bit, its by-product is the
+    # exact amax of X, and rolling the state gives the tensor scale the dynamic path would compute
+    X, W, bias = workloads.make_layer(workloads.CONFIG_SANA, 1, "cuda", M=1000)
+    wq, wsf, wts = B.nvfp4_quantize_weight(W)
+    state = torch.tensor([0.05, 0.0], dtype=torch.float32, device="cuda")
+    y = B.nvfp4_quantize_linear_delayed(X, wq, wsf, wts, bias, state)
+    ts = state[:1].clone()
+    xq, xsf = B.nvfp4_quantize(X, ts)
+    assert torch.equal(y, B.nvfp4_linear(xq, xsf, ts, wq, wsf, wts, bias))
+    assert state[0].item() == np.float32(0.05)
+    amax = np.abs(oracle.bits_to_f64(bits_of(X))).max()
+    assert state[1].item() == amax
+    B.sol_roll_tensor_scale(state)
+    assert state[0].item() == oracle.tensor_scale(bits_of(X)) and state[1].item() == 0.0
+    # second step with the rolled scale = the dynamic entry on the same X
+    y2 = B.nvfp4_quantize_linear_delayed(X, wq, wsf, wts, bias, state)
+    assert torch.equal(y2, B.nvfp4_quantize_linear(X, wq, wsf, wts, bias))
+    B.sol_last_device_status()
