@@ -71,6 +71,8 @@ def _load():
     L.oracle_mxfp4_linear.argtypes = [u8p, u8p, u8p, u8p, u16p, i64, i64, i64p, i64, f64p]
     L.oracle_gelu_tanh.restype, L.oracle_gelu_tanh.argtypes = ctypes.c_double, [ctypes.c_double]
     L.oracle_gelu_tanh_array.restype, L.oracle_gelu_tanh_array.argtypes = None, [f64p, i64, f64p]
+    L.oracle_layernorm_modulate.restype = None
+    L.oracle_layernorm_modulate.argtypes = [u16p, i64, i64, i64, u16p, u16p, i64, ctypes.c_double, f64p]
     L.oracle_lora_merge.restype = None
     L.oracle_lora_merge.argtypes = [u16p, i64, u16p, i64, u16p, i64, i64, i64, i64, f32, u16p]
     _lib = L
@@ -292,6 +294,30 @@ def nvfp4_linear_quantized(qx, sfx, Tx, qw, sfw, Tw, bias_bits, act: int, T_out,
     h = round_bf16(H)
     q, sf = quantize(h, T_out)
     return H, h, q, sf
+
+
+LN_EPS = 1e-6
+
+
+def layernorm_modulate(x_bits, scale_bits, shift_bits, rows_per_sample: int, eps: float = LN_EPS) -> np.ndarray:
+    """FP64 y = LN(x) * (1 + scale[sample]) + shift[sample]; x [rows, K], scale/shift [samples, K] BF16 bits."""
+    x, sc, sh = _c(x_bits, np.uint16), _c(scale_bits, np.uint16), _c(shift_bits, np.uint16)
+    rows, K = x.shape
+    samples = (rows + rows_per_sample - 1) // rows_per_sample
+    if sc.shape != (samples, K) or sh.shape != (samples, K):
+        raise ValueError("scale/shift must be [samples, K]")
+    out = np.empty((rows, K), np.float64)
+    _load().oracle_layernorm_modulate(_p(x, ctypes.c_uint16), rows, K, K, _p(sc, ctypes.c_uint16),
+                                      _p(sh, ctypes.c_uint16), rows_per_sample, float(eps), _p(out, ctypes.c_double))
+    return out
+
+
+def layernorm_modulate_quantized(x_bits, scale_bits, shift_bits, rows_per_sample: int, T, eps: float = LN_EPS):
+    """(Y FP64, h = bf16(Y) bits, nibbles, row-major scales): the normalised input of a linear, quantized."""
+    Y = layernorm_modulate(x_bits, scale_bits, shift_bits, rows_per_sample, eps)
+    h = round_bf16(Y)
+    q, sf = quantize(h, T)
+    return Y, h, q, sf
 
 
 # ----------------------------------------------------------------- weight refresh

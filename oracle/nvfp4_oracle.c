@@ -391,6 +391,35 @@ void oracle_gelu_tanh_array(const double *x, int64_t n, double *out) {
     for (int64_t i = 0; i < n; ++i) out[i] = oracle_gelu_tanh(x[i]);
 }
 
+/* Adaptive layer norm in front of a DiT linear (the producer of most quantized activations; the
+ * paper does not restate it): per row, with no learned affine,
+ *     mu = mean(x),  var = mean((x - mu)^2),  xhat = (x - mu) / sqrt(var + eps),
+ *     y[k] = xhat[k] * (1 + scale[s][k]) + shift[s][k],      s = row / rows_per_sample,
+ * evaluated in FP64 on the BF16 inputs.  x [rows, K] pitch ld; scale, shift [samples, K] dense. */
+void oracle_layernorm_modulate(const uint16_t *x, int64_t rows, int64_t K, int64_t ld, const uint16_t *scale,
+                               const uint16_t *shift, int64_t rows_per_sample, double eps, double *out) {
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        const uint16_t *xr = x + r * ld;
+        const int64_t s = r / rows_per_sample;
+        double mu = 0.0;
+        for (int64_t k = 0; k < K; ++k) mu += (double)oracle_bf16_to_f32(xr[k]);
+        mu /= (double)K;
+        double var = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+            double d = (double)oracle_bf16_to_f32(xr[k]) - mu;
+            var += d * d;
+        }
+        var /= (double)K;
+        const double inv = 1.0 / sqrt(var + eps);
+        for (int64_t k = 0; k < K; ++k) {
+            double xh = ((double)oracle_bf16_to_f32(xr[k]) - mu) * inv;
+            out[r * K + k] = xh * (1.0 + (double)oracle_bf16_to_f32(scale[s * K + k])) +
+                             (double)oracle_bf16_to_f32(shift[s * K + k]);
+        }
+    }
+}
+
 /* ------------------------------------------------------------------ weight refresh (LoRA merge) */
 
 /* The policy is trained through rank-r adapters (Section 4.1: r = 32, alpha = 64) and its

@@ -47,3 +47,37 @@ def test_quantized_output_is_the_composition_of_pinned_parts():
         assert np.array_equal(h, oracle.round_bf16(H))
         q2, sf2 = oracle.quantize(h, 0.01)
         assert np.array_equal(q, q2) and np.array_equal(sf, sf2)
+
+
+def _bits(t):
+    return t.to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+
+def test_layernorm_modulate_against_library_routine_and_invariants():
+    rng = np.random.default_rng(7)
+    rows, K, rps = 12, 96, 4
+    x = torch.from_numpy(rng.standard_normal((rows, K)) * 3 + 1.5).to(torch.bfloat16)
+    sc = torch.from_numpy(rng.standard_normal((3, K)) * 0.2).to(torch.bfloat16)
+    sh = torch.from_numpy(rng.standard_normal((3, K)) * 0.1).to(torch.bfloat16)
+    Y = oracle.layernorm_modulate(_bits(x), _bits(sc), _bits(sh), rps)
+    xd, scd, shd = x.double(), sc.double(), sh.double()
+    ln = torch.nn.functional.layer_norm(xd, (K,), eps=oracle.LN_EPS)                    # library routine, FP64
+    want = ln * (1 + scd.repeat_interleave(rps, dim=0)) + shd.repeat_interleave(rps, dim=0)
+    assert np.max(np.abs(Y - want.numpy())) < 1e-12
+    # zero modulation: rows have mean 0 and variance var / (var + eps)
+    z = torch.zeros((3, K), dtype=torch.bfloat16)
+    Y0 = oracle.layernorm_modulate(_bits(x), _bits(z), _bits(z), rps)
+    var = xd.var(dim=1, unbiased=False).numpy()
+    assert np.allclose(Y0.mean(axis=1), 0, atol=1e-13) and np.allclose((Y0 ** 2).mean(axis=1), var / (var + oracle.LN_EPS))
+    # invariant under a*x + b of the input (a > 0, up to eps) -- powers of two keep the inputs exact in BF16
+    Y4 = oracle.layernorm_modulate(_bits(x * 4), _bits(z), _bits(z), rps)
+    assert np.max(np.abs(Y4 - Y0)) < 1e-6
+    # the sample index really selects the modulation row: rows 4..7 use scale[1]
+    sc2 = torch.zeros((3, K), dtype=torch.bfloat16)
+    sc2[1] = 1.0
+    Y2 = oracle.layernorm_modulate(_bits(x), _bits(sc2), _bits(z), rps)
+    assert np.allclose(Y2[4:8], 2 * Y0[4:8]) and np.allclose(Y2[:4], Y0[:4]) and np.allclose(Y2[8:], Y0[8:])
+    # constant row: xhat = 0, output = shift
+    xc = torch.full((4, K), 2.5, dtype=torch.bfloat16)
+    Yc = oracle.layernorm_modulate(_bits(xc), _bits(sc[:1]), _bits(sh[:1]), 4)
+    assert np.allclose(Yc, sh[:1].double().numpy().repeat(4, axis=0))
