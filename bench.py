@@ -461,6 +461,42 @@ def run_ours(args):
                                    "nvfp4_linear with a calibrated T"}
             del xq, xsf, cat, y_qkv
 
+    # ---- adaptive layer norm fused with the quantizer (the producer of the q/k/v, MLP-in and single-stream
+    # inputs): one pass against torch's layer norm + modulation followed by our amax + quantizer
+    ln_quant = None
+    if world == 1 and not args.lean:
+        l0 = layers[0]
+        rps = workloads.SWEEP_TOKENS if l0.M % workloads.SWEEP_TOKENS == 0 else l0.M
+        n_s = l0.M // rps
+        gen = torch.Generator(device=dev).manual_seed(55)
+        sc = (torch.randn(n_s, l0.K, generator=gen, device=dev) * 0.3).to(torch.bfloat16)
+        sh = (torch.randn(n_s, l0.K, generator=gen, device=dev) * 0.2).to(torch.bfloat16)
+        Xl = data[0]["X"]
+        state = torch.ones(1, dtype=torch.float32, device=dev)
+        amax = torch.zeros(1, dtype=torch.float32, device=dev)
+        lq = (torch.empty((l0.M, l0.K // 2), dtype=torch.uint8, device=dev),
+              torch.empty(B.scale_bytes(l0.M, l0.K), dtype=torch.uint8, device=dev))
+        B.nvfp4_layernorm_quantize(Xl, sc, sh, rps, state, amax_out=amax, out=lq)
+        state.copy_(amax / 2688.0)
+        t_fused = loop_ms(lambda: B.nvfp4_layernorm_quantize(Xl, sc, sh, rps, state, amax_out=amax, out=lq))
+        xts_l = torch.empty(1, dtype=torch.float32, device=dev)
+
+        def ln_unfused():
+            h = torch.nn.functional.layer_norm(Xl, (l0.K,), eps=1e-6)
+            h = (h.view(n_s, rps, l0.K) * (1 + sc[:, None, :]) + sh[:, None, :]).view(l0.M, l0.K)
+            B.sol_amax_bf16(h, out=xts_l)
+            B.nvfp4_quantize(h, xts_l, out=lq)
+
+        t_unf = loop_ms(ln_unfused)
+        elems = l0.M * l0.K
+        ln_quant = {"shape": [l0.M, l0.K], "fused_us": t_fused * 1e3, "torch_norm_then_amax_quantize_us": t_unf * 1e3,
+                    "speedup": t_unf / t_fused, "fused_algorithmic_gbs": elems * 2.5625 / (t_fused * 1e-3) / 1e9,
+                    "roofline": {"bound": "hbm", "kernel": "layernorm_quantize_kernel",
+                                 "achieved": elems * 2.5625 / (t_fused * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                                 "unit": "GB/s", "frac": elems * 2.5625 / (t_fused * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                 "traffic": None, "peak_source": peak_src}}
+        del lq, sc, sh
+
     # ---- stage-1 selection and rank metrics at the paper's sizes (48 prompts per epoch, N = 96, K = 24):
     # two launches of one block per prompt, a few microseconds each (launch latency, not throughput)
     selection = None
@@ -563,7 +599,7 @@ def run_ours(args):
                                "peak_source": peak_src},
         "stack_tflops_delayed_scale": world * flops / (ms_static / args.steps * 1e-3) / 1e12,
         "mxfp4_stack_tflops": world * flops / (ms_mx / args.steps * 1e-3) / 1e12,
-        "weight_refresh": refresh, "mlp_pair_nvfp4_intermediate": mlp_pair, "single_stream_pair_nvfp4_intermediate": single_pair, "stage1_selection": selection,
+        "weight_refresh": refresh, "mlp_pair_nvfp4_intermediate": mlp_pair, "single_stream_pair_nvfp4_intermediate": single_pair, "layernorm_quantize": ln_quant, "stage1_selection": selection,
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": kernels_per_layer * len(layers) * args.steps,
         "bf16_vs_torch_matmul_note": "MEASURED_PEAKS bf16 (torch.matmul 8192^3): %.0f burst / %.0f sustained TF" % (
@@ -626,6 +662,27 @@ def run_only(args):
         print(json.dumps({"only": args.only, "M": M, "K": l.K, "N": l.N, "mxfp4_stack_ms": t,
                           "mxfp4_stack_tflops": 2.0 * M * l.N * l.K / t / 1e9}))
         return
+    if args.only == "layernorm_quantize":
+        cfg = workloads.CONFIGS[args.workload]
+        l0 = cfg.layers[0]
+        M = args.rows if args.rows > 0 else l0.M
+        X, _, _ = workloads.make_layer(cfg, 0, "cuda", M=M)
+        rps = workloads.SWEEP_TOKENS if M % workloads.SWEEP_TOKENS == 0 else M
+        gen = torch.Generator(device="cuda").manual_seed(55)
+        sc = (torch.randn(M // rps, l0.K, generator=gen, device="cuda") * 0.3).to(torch.bfloat16)
+        sh = (torch.randn(M // rps, l0.K, generator=gen, device="cuda") * 0.2).to(torch.bfloat16)
+        ts = torch.full((1,), 0.004, dtype=torch.float32, device="cuda")
+        times = []
+        for it in range(args.warmup + args.steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.nvfp4_layernorm_quantize(X, sc, sh, rps, ts)
+            e1.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                times.append(e0.elapsed_time(e1))
+        print(json.dumps({"only": "layernorm_quantize", "M": M, "K": l0.K, "us": 1e3 * sum(times) / len(times)}))
+        return
     if args.only == "mlp_pair":
         # FLUX feed-forward pair with the intermediate kept in NVFP4 (GELU in the first GEMM's epilogue)
         cfg = workloads.CONFIGS[args.workload]
@@ -684,7 +741,7 @@ def run_only(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair' / 'mxfp4:<layer>'")
+    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair' / 'mxfp4:<layer>' / 'layernorm_quantize'")
     ap.add_argument("--rows", type=int, default=0, help="profile mode: override M")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)

@@ -216,6 +216,23 @@ sol_status_t nvfp4_quantize_into(const void *x_bf16, int64_t M, int64_t K, int64
                                  void *q_dest, void *sf_dest, int64_t dest_K, int64_t dest_col0, void *stream);
 
 /*
+ * The quantizer fused into the other producer of a DiT linear's input: an adaptive layer norm.
+ *     mu, var = mean and population variance of row m;  xhat = (x - mu) / sqrt(var + eps)   (FP32)
+ *     h[m,k]  = bf16_rne( xhat[k] * (1 + scale[s,k]) + shift[s,k] ),   s = m / rows_per_sample
+ *     (q, sf) = nvfp4_quantize's mapping applied to h with T = *tensor_scale (caller supplied)
+ * One pass over x: 2 B read and 0.56 B written per element instead of a norm pass, an amax pass
+ * and a quantizer pass.
+ *   x_bf16       [M, K] BF16, pitch ldx;  K % 64 == 0, K <= 4096
+ *   scale, shift [ceil(M / rows_per_sample), K] BF16, dense (the per-sample modulation)
+ *   q_out        [M, K/2];  sf_out  SOL_SF_SWIZZLED_128x4 scales of an [M, K] tensor, every byte written
+ *   amax_out     nullable running max|h| (atomic max on the FP32 value), as in nvfp4_linear_quantized_out
+ */
+sol_status_t nvfp4_layernorm_quantize(const void *x_bf16, int64_t M, int64_t K, int64_t ldx, const void *scale_bf16,
+                                      const void *shift_bf16, int64_t rows_per_sample, float eps,
+                                      const float *tensor_scale, void *q_out, void *sf_out, float *amax_out,
+                                      void *stream);
+
+/*
  * BF16 linear, the full-precision stage-2 reference (Section 3.4):
  *     Y[m,n] = bf16_rne( sum_k x[m,k] * w[n,k] + bias[n] ),  FP32 accumulate.
  */

@@ -25,7 +25,7 @@ EXPORTS = [
     "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch", "nvfp4_linear_quantized_out",
     "solrl_select_contrastive", "solrl_rank_consistency", "sol_mxfp4_scale_bytes", "mxfp4_quantize",
     "mxfp4_linear", "nvfp4_linear_split_out", "nvfp4_quantize_into",
-    "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale",
+    "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale", "nvfp4_layernorm_quantize",
 ]
 
 _lib = None
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_quantize_linear_delayed.restype = i32
     L.nvfp4_quantize_linear_delayed.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, sz, vp]
     L.sol_roll_tensor_scale.restype, L.sol_roll_tensor_scale.argtypes = i32, [vp, vp]
+    L.nvfp4_layernorm_quantize.restype = i32
+    L.nvfp4_layernorm_quantize.argtypes = [vp, i64, i64, i64, vp, vp, i64, ctypes.c_float, vp, vp, vp, vp, vp]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -299,6 +301,22 @@ def nvfp4_quantize_linear_delayed(x, wq, wsf, w_tscale, bias, scale_state: torch
 
 def sol_roll_tensor_scale(scale_state: torch.Tensor):
     _check(lib().sol_roll_tensor_scale(_ptr(scale_state), _stream()), "sol_roll_tensor_scale")
+
+
+def nvfp4_layernorm_quantize(x, scale, shift, rows_per_sample: int, tensor_scale, eps: float = 1e-6,
+                             amax_out: torch.Tensor | None = None, out=None):
+    """LN(x) * (1 + scale[sample]) + shift[sample], quantized for the next linear: (nibbles, swizzled scales)."""
+    _need_2d_bf16(x, "x")
+    _need_2d_bf16(scale, "scale")
+    _need_2d_bf16(shift, "shift")
+    M, K = x.shape
+    if out is None:
+        out = _alloc_q(M, K, SF_SWIZZLED_128x4, x.device)
+    q, sf = out
+    _check(lib().nvfp4_layernorm_quantize(_ptr(x), M, K, x.stride(0), _ptr(scale), _ptr(shift), rows_per_sample,
+                                          float(eps), _ptr(tensor_scale), _ptr(q), _ptr(sf), _ptr(amax_out), _stream()),
+           "nvfp4_layernorm_quantize")
+    return q, sf
 
 
 def mxfp4_scale_bytes(rows: int, K: int, layout: int = SF_SWIZZLED_128x4) -> int:

@@ -444,6 +444,27 @@ sol_status_t nvfp4_quantize_into(const void *x_bf16, int64_t M, int64_t K, int64
                                 static_cast<cudaStream_t>(stream));
 }
 
+sol_status_t nvfp4_layernorm_quantize(const void *x_bf16, int64_t M, int64_t K, int64_t ldx, const void *scale_bf16,
+                                      const void *shift_bf16, int64_t rows_per_sample, float eps,
+                                      const float *tensor_scale, void *q_out, void *sf_out, float *amax_out,
+                                      void *stream) {
+    if (x_bf16 == nullptr || scale_bf16 == nullptr || shift_bf16 == nullptr || tensor_scale == nullptr ||
+        q_out == nullptr || sf_out == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(M, K) || K % 64 != 0 || K > layernorm_max_k() || ldx < K || rows_per_sample <= 0 || !(eps >= 0.0f))
+        return SOL_ERR_BAD_SHAPE;
+    if (!aligned16(x_bf16) || !aligned16(scale_bf16) || !aligned16(shift_bf16) || !aligned16(q_out) ||
+        !aligned16(sf_out) || ldx % 8 != 0 || (reinterpret_cast<uintptr_t>(tensor_scale) & 3u) ||
+        (reinterpret_cast<uintptr_t>(amax_out) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_layernorm_quantize(x_bf16, M, K, ldx, scale_bf16, shift_bf16, rows_per_sample, eps, tensor_scale,
+                                     q_out, sf_out, reinterpret_cast<uint32_t *>(amax_out),
+                                     static_cast<cudaStream_t>(stream));
+}
+
 sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,
                                    const float *w_tscale, const void *bias_bf16, void *y_bf16, int64_t M,
                                    int64_t N, int64_t K, int64_t ldy, void *workspace, size_t workspace_bytes,

@@ -1,0 +1,206 @@
+// Adaptive layer norm fused with the NVFP4 activation quantizer, for sm_100a.
+//
+// Most quantized activations of a DiT block are produced by a layer norm (no learned affine)
+// followed by a per-sample modulation, y = LN(x) (1 + scale[s]) + shift[s]; the linear that follows
+// wants Q(y) (paper Section 2's Q with a caller-supplied tensor scale, Section 3.4's NVFP4 rollout).
+// Unfused that is a norm pass (2 B read + 2 B written per element), an amax pass (2 B) and the
+// quantizer (2.56 B); this kernel reads x once and writes 0.56 B per element.
+//
+// One warp owns one row at a time: its K values stay in registers (packed BF16) between the mean, the
+// centred variance and the normalise / modulate / quantize sweep, so the row loop has no
+// shared-memory traffic for x and no block-level synchronisation.  A lane owns whole 16-element
+// scale blocks (blocks lane, lane + 32, ...), so K <= 4096.  A thread block works on rows of ONE
+// sample and keeps that sample's modulation in shared memory as FP32 pairs (1 + scale, shift).  The
+// block scale and the sixteen codes follow the quantizer's FP32 sequence on h = bf16(y); max|h| is
+// collected for the next call's tensor scale.
+#include "quant_math.cuh"
+#include "sol_internal.h"
+
+namespace sol {
+namespace {
+
+constexpr int kLnThreads = 128;
+constexpr int kLnWarps = kLnThreads / 32;
+constexpr int kLnMaxBlocksPerLane = 8;   // 8 x 32 lanes x 16 elements = 4096
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// two FP32 -> packed BF16 (first argument in the low half), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+// grid = (blocks per sample, samples); block (j, s) takes rows s*rows_per_sample + j*kLnWarps + warp,
+// striding by gridDim.x * kLnWarps inside the sample.
+template <int kBlocksPerLane>
+__global__ void __launch_bounds__(kLnThreads)
+layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, int64_t ld,
+                          const uint16_t *__restrict__ scale, const uint16_t *__restrict__ shift,
+                          int64_t rows_per_sample, float eps, const float *__restrict__ tscale,
+                          uint8_t *__restrict__ q, uint8_t *__restrict__ sf, uint32_t *amax_track) {
+    // (1 + scale, shift) of this block's sample for element pairs, laid out [pair within block][block] so
+    // that the 32 lanes of a warp (consecutive blocks) read consecutive 16-byte words
+    extern __shared__ __align__(16) float4 mod[];
+    __shared__ float rcp_tab[128];
+    __shared__ uint32_t warp_seen[kLnWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t sample = blockIdx.y;
+    const float T = *tscale;
+    const float c6T = __fmul_rn(6.0f, T);
+    for (uint32_t code = threadIdx.x; code < 128; code += kLnThreads)
+        rcp_tab[code] = code ? __frcp_rn(__fmul_rn(qmath::e4m3_to_f32(code), T)) : 0.0f;
+    const int nblocks = K >> 4;                 // scale blocks per row
+    for (int k2 = threadIdx.x; k2 < (K >> 1); k2 += kLnThreads) {
+        const uint32_t sc = __ldg(reinterpret_cast<const uint32_t *>(scale + sample * K) + k2);
+        const uint32_t sh = __ldg(reinterpret_cast<const uint32_t *>(shift + sample * K) + k2);
+        mod[(k2 & 7) * nblocks + (k2 >> 3)] =
+            make_float4(1.0f + qmath::bf16_lo(sc), qmath::bf16_lo(sh), 1.0f + qmath::bf16_hi(sc), qmath::bf16_hi(sh));
+    }
+    __syncthreads();
+
+    const int64_t chunks_k = nblocks >> 2;      // K is a multiple of 64: whole chunks only
+    const int64_t first = sample * rows_per_sample;
+    const int64_t last = min(rows, first + rows_per_sample);
+    const float inv_k = 1.0f / static_cast<float>(K);
+    uint32_t seen = 0;
+    for (int64_t r = first + static_cast<int64_t>(blockIdx.x) * kLnWarps + warp; r < last;
+         r += static_cast<int64_t>(gridDim.x) * kLnWarps) {
+        // ---- the row into registers, packed as loaded (two BF16 per register: half the registers of an
+        // FP32 copy, which buys the occupancy a latency-bound row loop needs); block i of this lane =
+        // elements [(lane + 32 i) * 16, +16)
+        uint32_t w[kBlocksPerLane][8];
+        float s1 = 0.0f;
+#pragma unroll
+        for (int i = 0; i < kBlocksPerLane; ++i) {
+            const int b = lane + 32 * i;
+            uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
+            if (b < nblocks) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(x + r * ld + b * 16);
+                v0 = __ldcs(src);
+                v1 = __ldcs(src + 1);
+            }
+            w[i][0] = v0.x; w[i][1] = v0.y; w[i][2] = v0.z; w[i][3] = v0.w;
+            w[i][4] = v1.x; w[i][5] = v1.y; w[i][6] = v1.z; w[i][7] = v1.w;
+        }
+#pragma unroll
+        for (int i = 0; i < kBlocksPerLane; ++i)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s1 += qmath::bf16_lo(w[i][e]) + qmath::bf16_hi(w[i][e]);
+        const float mu = warp_sum(s1) * inv_k;
+        float s2 = 0.0f;
+#pragma unroll
+        for (int i = 0; i < kBlocksPerLane; ++i) {
+            if (lane + 32 * i < nblocks) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float d0 = qmath::bf16_lo(w[i][e]) - mu, d1 = qmath::bf16_hi(w[i][e]) - mu;
+                    s2 = fmaf(d0, d0, s2);
+                    s2 = fmaf(d1, d1, s2);
+                }
+            }
+        }
+        const float rstd = 1.0f / sqrtf(warp_sum(s2) * inv_k + eps);
+        const float nmr = -mu * rstd;   // xhat = fma(x, rstd, -mu * rstd)
+        const int64_t row_tile = r >> 7;
+        const int rr = static_cast<int>(r & 127);
+        uint8_t *sf_row = sf + row_tile * chunks_k * 512 + (rr & 31) * 16 + (rr >> 5) * 4;
+        // ---- normalise, modulate, round to BF16, quantize
+#pragma unroll
+        for (int i = 0; i < kBlocksPerLane; ++i) {
+            const int b = lane + 32 * i;
+            uint32_t sb = 0;
+            if (b < nblocks) {
+                const float4 *mp = mod + b;
+                uint32_t hw[8];
+                uint32_t bm = 0;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float4 m = mp[e * nblocks];   // (1 + scale, shift) of two neighbouring elements
+                    const float y0 = fmaf(fmaf(qmath::bf16_lo(w[i][e]), rstd, nmr), m.x, m.y);
+                    const float y1 = fmaf(fmaf(qmath::bf16_hi(w[i][e]), rstd, nmr), m.z, m.w);
+                    hw[e] = pack_bf16x2(y0, y1);
+                    bm = qmath::absmax2(bm, hw[e]);
+                }
+                bm &= 0x7FFF7FFFu;
+                const uint32_t abits = max(bm & 0xFFFFu, bm >> 16);
+                seen = max(seen, abits);
+                const float a = __uint_as_float(abits << 16);
+                sb = qmath::f32_to_e4m3_sat(__fdiv_rn(a, c6T));
+                const float rcp = rcp_tab[sb];
+                uint2 packed;
+                packed.x = qmath::quantize8(hw[0], hw[1], hw[2], hw[3], rcp);
+                packed.y = qmath::quantize8(hw[4], hw[5], hw[6], hw[7], rcp);
+                __stcs(reinterpret_cast<uint2 *>(q + r * (K >> 1) + b * 8), packed);
+            }
+            // four neighbouring lanes hold the four scale bytes of one (row, chunk) slot: one 4-byte store
+            uint32_t word = sb;
+            word |= __shfl_down_sync(0xFFFFFFFFu, sb, 1) << 8;
+            word |= __shfl_down_sync(0xFFFFFFFFu, sb, 2) << 16;
+            word |= __shfl_down_sync(0xFFFFFFFFu, sb, 3) << 24;
+            if ((lane & 3) == 0 && b < nblocks) *reinterpret_cast<uint32_t *>(sf_row + (b >> 2) * 512) = word;
+        }
+    }
+    // rows past M inside the last 128-row scale chunk are padding and read as 0 (first block only)
+    if (blockIdx.x == 0 && blockIdx.y == 0) {
+        const int64_t padded_rows = (rows + 127) / 128 * 128;
+        for (int64_t r = rows + warp; r < padded_rows; r += kLnWarps) {
+            const int rr = static_cast<int>(r & 127);
+            uint8_t *sf_row = sf + (r >> 7) * chunks_k * 512 + (rr & 31) * 16 + (rr >> 5) * 4;
+            for (int64_t c = lane; c < chunks_k; c += 32) *reinterpret_cast<uint32_t *>(sf_row + c * 512) = 0u;
+        }
+    }
+    if (amax_track != nullptr) {
+        seen = __reduce_max_sync(0xFFFFFFFFu, seen);
+        if (lane == 0) warp_seen[warp] = seen;
+        __syncthreads();
+        if (threadIdx.x < 32) {
+            uint32_t m = threadIdx.x < kLnWarps ? warp_seen[threadIdx.x] : 0;
+            m = __reduce_max_sync(0xFFFFFFFFu, m);
+            if (threadIdx.x == 0 && m) atomicMax(amax_track, m << 16);
+        }
+    }
+}
+
+}  // namespace
+
+int layernorm_max_k() { return kLnMaxBlocksPerLane * 32 * 16; }
+
+sol_status_t launch_layernorm_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, const void *scale,
+                                       const void *shift, int64_t rows_per_sample, float eps, const float *tscale,
+                                       void *q, void *sf, uint32_t *amax_track, cudaStream_t stream) {
+    const int64_t samples = ceil_div(rows, rows_per_sample);
+    if (samples > 65535) return SOL_ERR_BAD_SHAPE;
+    const DeviceInfo *dev = current_device_info();
+    const int sms = dev != nullptr && dev->ok ? dev->sm_count : 148;
+    const size_t smem = static_cast<size_t>(K) * sizeof(float2);
+    const int per_lane = static_cast<int>(ceil_div(K / 16, 32));
+    auto launch = [&](auto kern) {
+        // one wave of resident blocks, split evenly over the samples, never more blocks per sample
+        // than it has groups of rows
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kLnThreads, smem) != cudaSuccess || per_sm < 1)
+            per_sm = 1;
+        int64_t per_sample = (static_cast<int64_t>(sms) * per_sm) / samples;
+        const int64_t row_groups = ceil_div(rows_per_sample < rows ? rows_per_sample : rows, kLnWarps);
+        if (per_sample > row_groups) per_sample = row_groups;
+        if (per_sample < 1) per_sample = 1;
+        const dim3 grid(static_cast<unsigned>(per_sample), static_cast<unsigned>(samples));
+        kern<<<grid, kLnThreads, smem, stream>>>(static_cast<const uint16_t *>(x), rows, static_cast<int>(K), ld,
+                                                 static_cast<const uint16_t *>(scale), static_cast<const uint16_t *>(shift),
+                                                 rows_per_sample, eps, tscale, static_cast<uint8_t *>(q),
+                                                 static_cast<uint8_t *>(sf), amax_track);
+    };
+    if (per_lane <= 2) launch(layernorm_quantize_kernel<2>);
+    else if (per_lane <= 4) launch(layernorm_quantize_kernel<4>);
+    else if (per_lane <= 6) launch(layernorm_quantize_kernel<6>);
+    else launch(layernorm_quantize_kernel<8>);
+    return launch_status();
+}
+
+}  // namespace sol

@@ -76,6 +76,11 @@ sol_status_t launch_quantize_tracking(const void *x, int64_t rows, int64_t K, in
                                       void *sf, uint32_t *amax_track, cudaStream_t stream);
 // state[0] <- T(state[1]); state[1] <- 0.
 sol_status_t launch_roll_scale(float *state, cudaStream_t stream);
+// Layer norm + per-sample modulation + NVFP4 quantizer in one pass (K a multiple of 64, K <= layernorm_max_k()).
+sol_status_t launch_layernorm_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, const void *scale,
+                                       const void *shift, int64_t rows_per_sample, float eps, const float *tscale,
+                                       void *q, void *sf, uint32_t *amax_track, cudaStream_t stream);
+int layernorm_max_k();
 sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
                                    sol_sf_layout_t layout, cudaStream_t stream);
 // Stage-1 selection and rank-consistency metrics (one block per prompt).

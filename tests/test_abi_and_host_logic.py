@@ -127,6 +127,12 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.nvfp4_quantize_linear_delayed(p, 64, p, p, p, None, p, 4, 8, 64, 8, p + 4, p, 1 << 20, None) == ALIGN
     assert L.nvfp4_quantize_linear_delayed(p, 64, p, p, p, None, p, 4, 8, 64, 8, p, p, 16, None) == WS
     assert L.sol_roll_tensor_scale(None, None) == NULLP
+    # layer norm fused with the quantizer
+    assert L.nvfp4_layernorm_quantize(p, 4, 64, 64, p, None, 4, 1e-6, p, p, p, None, None) == NULLP
+    assert L.nvfp4_layernorm_quantize(p, 4, 96, 96, p, p, 4, 1e-6, p, p, p, None, None) == SHAPE      # K % 64
+    assert L.nvfp4_layernorm_quantize(p, 4, 8192, 8192, p, p, 4, 1e-6, p, p, p, None, None) == SHAPE  # K > 4096
+    assert L.nvfp4_layernorm_quantize(p, 4, 64, 64, p, p, 0, 1e-6, p, p, p, None, None) == SHAPE
+    assert L.nvfp4_layernorm_quantize(p, 4, 64, 64, p + 8, p, 4, 1e-6, p, p, p, None, None) == ALIGN
     # MXFP4
     assert L.sol_mxfp4_scale_bytes(256, 512, 0) == 256 * 16 and L.sol_mxfp4_scale_bytes(256, 512, 1) == 2 * 4 * 512
     assert L.sol_mxfp4_scale_bytes(130, 160, 1) == 2 * 2 * 512 and L.sol_mxfp4_scale_bytes(4, 48, 1) == 0
