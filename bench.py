@@ -662,6 +662,94 @@ def run_only(args):
         print(json.dumps({"only": args.only, "M": M, "K": l.K, "N": l.N, "mxfp4_stack_ms": t,
                           "mxfp4_stack_tflops": 2.0 * M * l.N * l.K / t / 1e9}))
         return
+    if args.only == "single_block":
+        # One FLUX-shaped single-stream block forward, NVFP4 against BF16.  The linears, the norm + quantizer
+        # and the split / concat epilogues are this library's kernels; attention is torch's scaled-dot-product
+        # attention (a library kernel, not part of the path under test) and the gate / residual, BF16 GELU and
+        # concat of the BF16 path are plain torch ops.
+        import torch.nn.functional as F
+        cfg = workloads.CONFIGS[args.workload]
+        names = [l.name for l in cfg.layers]
+        i1, i2 = names.index("s_fused"), names.index("s_out")
+        l1, l2 = cfg.layers[i1], cfg.layers[i2]
+        M, H = l1.M, l1.K
+        rps = workloads.SWEEP_TOKENS if M % workloads.SWEEP_TOKENS == 0 else M
+        n_s, heads, hd = M // rps, H // 128, 128
+        n_qkv, n_mlp = 3 * H, l1.N - 3 * H
+        X, W1, b1 = workloads.make_layer(cfg, i1, "cuda")
+        _, W2, b2 = workloads.make_layer(cfg, i2, "cuda", M=128)
+        gen = torch.Generator(device="cuda").manual_seed(77)
+        sc, sh, gate = [(torch.randn(n_s, H, generator=gen, device="cuda") * 0.2).to(torch.bfloat16) for _ in range(3)]
+        w1q, w2q = B.nvfp4_quantize_weight(W1), B.nvfp4_quantize_weight(W2)
+        state = torch.ones(1, dtype=torch.float32, device="cuda")
+        amax_in = torch.zeros(1, dtype=torch.float32, device="cuda")
+        amax_cat = torch.zeros(1, dtype=torch.float32, device="cuda")
+        t_cat = torch.ones(1, dtype=torch.float32, device="cuda")
+        xq = (torch.empty((M, H // 2), dtype=torch.uint8, device="cuda"),
+              torch.empty(B.scale_bytes(M, H), dtype=torch.uint8, device="cuda"))
+        cat = (torch.zeros((M, l2.K // 2), dtype=torch.uint8, device="cuda"),
+               torch.zeros(B.scale_bytes(M, l2.K), dtype=torch.uint8, device="cuda"))
+        y_qkv = torch.empty((M, n_qkv), dtype=torch.bfloat16, device="cuda")
+        y1 = torch.empty((M, l1.N), dtype=torch.bfloat16, device="cuda")
+        y2 = torch.empty((M, H), dtype=torch.bfloat16, device="cuda")
+
+        def attention(qkv):
+            q, k, v = qkv.view(n_s, rps, 3, heads, hd).permute(2, 0, 3, 1, 4)
+            o = F.scaled_dot_product_attention(q, k, v)
+            return o.transpose(1, 2).reshape(M, H)
+
+        def finish(lin2):
+            return X + (gate[:, None, :] * lin2.view(n_s, rps, H)).view(M, H)
+
+        def block_fp4():
+            B.nvfp4_layernorm_quantize(X, sc, sh, rps, state, amax_out=amax_in, out=xq)
+            B.nvfp4_linear_split_out(xq[0], xq[1], state, *w1q, b1, n_qkv, B.ACT_GELU_TANH, t_cat, cat, H,
+                                     y_out=y_qkv, amax_out=amax_cat)
+            attn = attention(y_qkv)
+            B.nvfp4_quantize_into(attn, t_cat, cat, 0)
+            B.nvfp4_linear(cat[0], cat[1], t_cat, *w2q, b2, out=y2)
+            return finish(y2)
+
+        def block_bf16():
+            h = F.layer_norm(X, (H,), eps=1e-6)
+            h = (h.view(n_s, rps, H) * (1 + sc[:, None, :]) + sh[:, None, :]).view(M, H)
+            B.bf16_linear(h, W1, b1, out=y1)
+            attn = attention(y1[:, :n_qkv])
+            c = torch.cat((attn, F.gelu(y1[:, n_qkv:], approximate="tanh")), dim=1)
+            B.bf16_linear(c, W2, b2, out=y2)
+            return finish(y2)
+
+        out4 = block_fp4()                       # calibrate the delayed scales from the first pass
+        state.copy_(amax_in / 2688.0)
+        t_cat.copy_(torch.maximum(amax_cat, B.sol_amax_bf16(attention(y_qkv)) * 2688.0) / 2688.0)
+        res = {}
+        for name, fn in (("nvfp4", block_fp4), ("bf16", block_bf16)):
+            for _ in range(max(1, args.warmup)):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                out = fn()
+            e1.record()
+            torch.cuda.synchronize()
+            res[name] = e0.elapsed_time(e1) / args.steps
+            res[name + "_out"] = out
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            attention(y_qkv)
+        e1.record()
+        torch.cuda.synchronize()
+        t_attn = e0.elapsed_time(e1) / args.steps
+        B.sol_last_device_status()
+        diff = (res["nvfp4_out"].float() - res["bf16_out"].float())
+        rel = float(diff.pow(2).mean().sqrt() / res["bf16_out"].float().pow(2).mean().sqrt())
+        print(json.dumps({"only": "single_block", "M": M, "hidden": H, "nvfp4_ms": res["nvfp4"], "bf16_ms": res["bf16"],
+                          "speedup": res["bf16"] / res["nvfp4"], "attention_ms_in_both": t_attn,
+                          "speedup_without_attention": (res["bf16"] - t_attn) / (res["nvfp4"] - t_attn),
+                          "rel_rms_difference_of_outputs": rel}))
+        return
     if args.only == "layernorm_quantize":
         cfg = workloads.CONFIGS[args.workload]
         l0 = cfg.layers[0]
@@ -741,7 +829,7 @@ def run_only(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair' / 'mxfp4:<layer>' / 'layernorm_quantize'")
+    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair' / 'mxfp4:<layer>' / 'layernorm_quantize' / 'single_block'")
     ap.add_argument("--rows", type=int, default=0, help="profile mode: override M")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
