@@ -6,13 +6,16 @@
 // Unfused that is a norm pass (2 B read + 2 B written per element), an amax pass (2 B) and the
 // quantizer (2.56 B); this kernel reads x once and writes 0.56 B per element.
 //
-// One warp owns one row at a time: its K values stay in registers (packed BF16) between the mean, the
-// centred variance and the normalise / modulate / quantize sweep, so the row loop has no
-// shared-memory traffic for x and no block-level synchronisation.  A lane owns whole 16-element
+// One warp owns one row at a time: its K values stay in registers between the mean, the centred
+// variance and the normalise / modulate / quantize sweep, and there is no block-level
+// synchronisation in the row loop.  Rows reach the warp through a two-slot ring in shared memory
+// filled by bulk asynchronous copies (cp.async.bulk + mbarrier) that the warp issues two rows ahead,
+// so the HBM latency is not paid by a warp that holds 160 registers per thread.  A lane owns whole 16-element
 // scale blocks (blocks lane, lane + 32, ...), so K <= 4096.  A thread block works on rows of ONE
 // sample and keeps that sample's modulation in shared memory as FP32 pairs (1 + scale, shift).  The
 // block scale and the sixteen codes follow the quantizer's FP32 sequence on h = bf16(y); max|h| is
 // collected for the next call's tensor scale.
+#include "ptx.cuh"
 #include "quant_math.cuh"
 #include "sol_internal.h"
 
@@ -29,6 +32,15 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
+// One row (bytes, a multiple of 16, 16-byte aligned on both sides) global -> shared, completing on `bar`.
+__device__ __forceinline__ void bulk_load_row(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+constexpr long long kLnWaitLimitCycles = 2000000000LL;
+
 // two FP32 -> packed BF16 (first argument in the low half), round to nearest even
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t d;
@@ -43,10 +55,13 @@ __global__ void __launch_bounds__(kLnThreads)
 layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, int64_t ld,
                           const uint16_t *__restrict__ scale, const uint16_t *__restrict__ shift,
                           int64_t rows_per_sample, float eps, const float *__restrict__ tscale,
-                          uint8_t *__restrict__ q, uint8_t *__restrict__ sf, uint32_t *amax_track) {
+                          uint8_t *__restrict__ q, uint8_t *__restrict__ sf, uint32_t *amax_track,
+                          uint32_t *status) {
     // (1 + scale, shift) of this block's sample for element pairs, laid out [pair within block][block] so
-    // that the 32 lanes of a warp (consecutive blocks) read consecutive 16-byte words
+    // that the 32 lanes of a warp (consecutive blocks) read consecutive 16-byte words; behind it the row
+    // ring (two slots of K BF16 per warp)
     extern __shared__ __align__(16) float4 mod[];
+    __shared__ __align__(8) uint64_t ring_bar[kLnWarps][2];
     __shared__ float rcp_tab[128];
     __shared__ uint32_t warp_seen[kLnWarps];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -69,11 +84,42 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
     const int64_t last = min(rows, first + rows_per_sample);
     const float inv_k = 1.0f / static_cast<float>(K);
     uint32_t seen = 0;
-    for (int64_t r = first + static_cast<int64_t>(blockIdx.x) * kLnWarps + warp; r < last;
-         r += static_cast<int64_t>(gridDim.x) * kLnWarps) {
-        // ---- the row into registers, packed as loaded (two BF16 per register: half the registers of an
-        // FP32 copy, which buys the occupancy a latency-bound row loop needs); block i of this lane =
-        // elements [(lane + 32 i) * 16, +16)
+    const uint32_t row_bytes = static_cast<uint32_t>(K) * 2u;
+    const uint32_t ring = ptx::smem_u32(mod) + static_cast<uint32_t>(K) * 8u + warp * 2u * row_bytes;
+    const uint32_t bar0 = ptx::smem_u32(&ring_bar[warp][0]);
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * kLnWarps;
+    const int64_t r_first = first + static_cast<int64_t>(blockIdx.x) * kLnWarps + warp;
+    if (lane == 0) {
+        ptx::mbar_init(bar0, 1);
+        ptx::mbar_init(bar0 + 8, 1);
+        ptx::fence_mbar_init();
+    }
+    __syncwarp();
+    if (lane == 0) {   // rows 0 and 1 of this warp
+        for (int j = 0; j < 2; ++j)
+            if (r_first + j * stride < last) {
+                ptx::mbar_arrive_expect_tx(bar0 + 8u * j, row_bytes);
+                bulk_load_row(ring + j * row_bytes, x + (r_first + j * stride) * ld, row_bytes, bar0 + 8u * j);
+            }
+    }
+    int64_t j = 0;
+    for (int64_t r = r_first; r < last; r += stride, ++j) {
+        const uint32_t slot = static_cast<uint32_t>(j) & 1u, parity = static_cast<uint32_t>(j >> 1) & 1u;
+        if (!ptx::mbar_try_wait(bar0 + 8u * slot, parity)) {   // bounded: a copy that never lands ends the loop
+            const long long t0 = clock64();
+            bool ok = true;
+            while (!ptx::mbar_try_wait(bar0 + 8u * slot, parity)) {
+                if (clock64() - t0 > kLnWaitLimitCycles) {
+                    ok = false;
+                    break;
+                }
+            }
+            if (!__all_sync(0xFFFFFFFFu, ok)) {   // warp-uniform exit
+                if (lane == 0 && status != nullptr) atomicExch(status, 0xA00u);
+                break;
+            }
+        }
+        // ---- the row from the ring into registers; block i of this lane = elements [(lane + 32 i) * 16, +16)
         uint32_t w[kBlocksPerLane][8];
         float s1 = 0.0f;
 #pragma unroll
@@ -81,12 +127,18 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
             const int b = lane + 32 * i;
             uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
             if (b < nblocks) {
-                const uint4 *src = reinterpret_cast<const uint4 *>(x + r * ld + b * 16);
-                v0 = __ldcs(src);
-                v1 = __ldcs(src + 1);
+                const uint32_t src = ring + slot * row_bytes + b * 32;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v0.x), "=r"(v0.y), "=r"(v0.z), "=r"(v0.w) : "r"(src));
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v1.x), "=r"(v1.y), "=r"(v1.z), "=r"(v1.w) : "r"(src + 16));
             }
             w[i][0] = v0.x; w[i][1] = v0.y; w[i][2] = v0.z; w[i][3] = v0.w;
             w[i][4] = v1.x; w[i][5] = v1.y; w[i][6] = v1.z; w[i][7] = v1.w;
+        }
+        __syncwarp();
+        if (lane == 0 && r + 2 * stride < last) {   // the slot is free again: fetch the row after next
+            ptx::fence_proxy_async_smem();
+            ptx::mbar_arrive_expect_tx(bar0 + 8u * slot, row_bytes);
+            bulk_load_row(ring + slot * row_bytes, x + (r + 2 * stride) * ld, row_bytes, bar0 + 8u * slot);
         }
 #pragma unroll
         for (int i = 0; i < kBlocksPerLane; ++i)
@@ -178,11 +230,13 @@ sol_status_t launch_layernorm_quantize(const void *x, int64_t rows, int64_t K, i
     if (samples > 65535) return SOL_ERR_BAD_SHAPE;
     const DeviceInfo *dev = current_device_info();
     const int sms = dev != nullptr && dev->ok ? dev->sm_count : 148;
-    const size_t smem = static_cast<size_t>(K) * sizeof(float2);
+    // modulation table (8 bytes per element) + per warp two row slots of 2 bytes per element
+    const size_t smem = static_cast<size_t>(K) * 8 + static_cast<size_t>(kLnWarps) * 2 * K * 2;
     const int per_lane = static_cast<int>(ceil_div(K / 16, 32));
     auto launch = [&](auto kern) {
         // one wave of resident blocks, split evenly over the samples, never more blocks per sample
         // than it has groups of rows
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
         int per_sm = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kLnThreads, smem) != cudaSuccess || per_sm < 1)
             per_sm = 1;
@@ -194,7 +248,7 @@ sol_status_t launch_layernorm_quantize(const void *x, int64_t rows, int64_t K, i
         kern<<<grid, kLnThreads, smem, stream>>>(static_cast<const uint16_t *>(x), rows, static_cast<int>(K), ld,
                                                  static_cast<const uint16_t *>(scale), static_cast<const uint16_t *>(shift),
                                                  rows_per_sample, eps, tscale, static_cast<uint8_t *>(q),
-                                                 static_cast<uint8_t *>(sf), amax_track);
+                                                 static_cast<uint8_t *>(sf), amax_track, device_status_word());
     };
     if (per_lane <= 2) launch(layernorm_quantize_kernel<2>);
     else if (per_lane <= 4) launch(layernorm_quantize_kernel<4>);
