@@ -22,8 +22,7 @@
 namespace sol {
 namespace {
 
-constexpr int kLnThreads = 128;
-constexpr int kLnWarps = kLnThreads / 32;
+constexpr int kLnMaxWarps = 16;          // upper bound of warps per block (the launcher uses 4)
 constexpr int kLnMaxBlocksPerLane = 8;   // 8 x 32 lanes x 16 elements = 4096
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -51,7 +50,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // grid = (blocks per sample, samples); block (j, s) takes rows s*rows_per_sample + j*kLnWarps + warp,
 // striding by gridDim.x * kLnWarps inside the sample.
 template <int kBlocksPerLane>
-__global__ void __launch_bounds__(kLnThreads)
+__global__ void __launch_bounds__(kLnMaxWarps * 32)
 layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, int64_t ld,
                           const uint16_t *__restrict__ scale, const uint16_t *__restrict__ shift,
                           int64_t rows_per_sample, float eps, const float *__restrict__ tscale,
@@ -61,10 +60,11 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
     // that the 32 lanes of a warp (consecutive blocks) read consecutive 16-byte words; behind it the row
     // ring (two slots of K BF16 per warp)
     extern __shared__ __align__(16) float4 mod[];
-    __shared__ __align__(8) uint64_t ring_bar[kLnWarps][2];
+    __shared__ __align__(8) uint64_t ring_bar[kLnMaxWarps][2];
     __shared__ float rcp_tab[128];
-    __shared__ uint32_t warp_seen[kLnWarps];
+    __shared__ uint32_t warp_seen[kLnMaxWarps];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int kLnWarps = blockDim.x >> 5, kLnThreads = blockDim.x;
     const int64_t sample = blockIdx.y;
     const float T = *tscale;
     const float c6T = __fmul_rn(6.0f, T);
@@ -140,24 +140,32 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
             ptx::mbar_arrive_expect_tx(bar0 + 8u * slot, row_bytes);
             bulk_load_row(ring + slot * row_bytes, x + (r + 2 * stride) * ld, row_bytes, bar0 + 8u * slot);
         }
-#pragma unroll
-        for (int i = 0; i < kBlocksPerLane; ++i)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) s1 += qmath::bf16_lo(w[i][e]) + qmath::bf16_hi(w[i][e]);
-        const float mu = warp_sum(s1) * inv_k;
+        // mean and variance in one sweep over data shifted by a pivot taken from the row (its first element):
+        // sum (x - p) and sum (x - p)^2 lose no accuracy to cancellation as long as p lies within the data,
+        // and the two warp reductions run side by side instead of one after the other
+        const float pivot = __shfl_sync(0xFFFFFFFFu, qmath::bf16_lo(w[0][0]), 0);
         float s2 = 0.0f;
 #pragma unroll
         for (int i = 0; i < kBlocksPerLane; ++i) {
             if (lane + 32 * i < nblocks) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float d0 = qmath::bf16_lo(w[i][e]) - mu, d1 = qmath::bf16_hi(w[i][e]) - mu;
+                    const float d0 = qmath::bf16_lo(w[i][e]) - pivot, d1 = qmath::bf16_hi(w[i][e]) - pivot;
+                    s1 += d0 + d1;
                     s2 = fmaf(d0, d0, s2);
                     s2 = fmaf(d1, d1, s2);
                 }
             }
         }
-        const float rstd = 1.0f / sqrtf(warp_sum(s2) * inv_k + eps);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
+            s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+        }
+        const float dm = s1 * inv_k;                       // mean - pivot
+        const float mu = pivot + dm;
+        const float var = fmaxf(fmaf(-dm, dm, s2 * inv_k), 0.0f);
+        const float rstd = 1.0f / sqrtf(var + eps);
         const float nmr = -mu * rstd;   // xhat = fma(x, rstd, -mu * rstd)
         const int64_t row_tile = r >> 7;
         const int rr = static_cast<int>(r & 127);
@@ -230,13 +238,17 @@ sol_status_t launch_layernorm_quantize(const void *x, int64_t rows, int64_t K, i
     if (samples > 65535) return SOL_ERR_BAD_SHAPE;
     const DeviceInfo *dev = current_device_info();
     const int sms = dev != nullptr && dev->ok ? dev->sm_count : 148;
-    // modulation table (8 bytes per element) + per warp two row slots of 2 bytes per element
+    // modulation table (8 bytes per element) + per warp two row slots of 2 bytes per element.  Four warps
+    // per block, three blocks per SM at K = 3072; one block of 14-16 warps per SM measured no faster
+    // (the kernel is bound by instruction issue, not by rows in flight).
+    const int kLnWarps = 4;
+    const int kLnThreads = kLnWarps * 32;
     const size_t smem = static_cast<size_t>(K) * 8 + static_cast<size_t>(kLnWarps) * 2 * K * 2;
     const int per_lane = static_cast<int>(ceil_div(K / 16, 32));
     auto launch = [&](auto kern) {
         // one wave of resident blocks, split evenly over the samples, never more blocks per sample
         // than it has groups of rows
-        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024);
         int per_sm = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kLnThreads, smem) != cudaSuccess || per_sm < 1)
             per_sm = 1;
