@@ -190,9 +190,13 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     auto acc_empty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 2 + s); };
     auto ovl_free_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 4 + s); };
     auto sf_ready_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 6 + s); };
-    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * (2 * kStages + 6 + kSfBufs));
+    // The scale tiles of a stage complete on a barrier of their own: they are a sixth of the stage's bytes
+    // and land first, so their copy into TMEM (a ~500-cycle chain: copy warp wake-up, tcgen05.cp, commit)
+    // overlaps the arrival of A and B instead of following it.
+    auto sf_full_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 6 + kSfBufs + s); };
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * (3 * kStages + 6 + kSfBufs));
     volatile uint32_t *abort_flag =
-        reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * (2 * kStages + 6 + kSfBufs) + 4);
+        reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * (3 * kStages + 6 + kSfBufs) + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();
@@ -208,6 +212,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(sf_full_bar(s), 1);
             ptx::mbar_init(empty_bar(s), 1);
         }
         for (int s = 0; s < 2; ++s) {
@@ -240,8 +245,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         // ------------------------------------------------------------ TMA producer: A and B tiles (both CTAs)
         const bool elected = ptx::elect_one();
         const uint32_t full0 = ptx::map_to_cta(full_bar(0), 0);  // the even CTA's barriers
-        const bool sf_load = !(kTuning && (p.dbg & kDbgNoSfLoad));
-        const uint32_t tx = 2u * (kABytes + kBBytes + (sf_load ? kSfLoadBytes : 0));
+        const uint32_t tx = 2u * (kABytes + kBBytes);
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -273,7 +277,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         // ------------------------------------------------------------ TMA producer: scale-factor tiles (both CTAs)
         if (!(kTuning && (p.dbg & kDbgNoSfLoad))) {
             const bool elected = ptx::elect_one();
-            const uint32_t full0 = ptx::map_to_cta(full_bar(0), 0);
+            const uint32_t full0 = ptx::map_to_cta(sf_full_bar(0), 0);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -289,6 +293,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     }
                     const uint32_t ssfa = smem_base + stage * kStageBytes + kABytes + kBBytes;
                     if (elected) {
+                        if (leader) ptx::mbar_arrive_expect_tx(sf_full_bar(stage), 2u * kSfLoadBytes);
                         ptx::tma_load_3d_pair(ssfa, &tm_sfa, 0, kt * kSfChunksK, rca, full0 + 8u * stage);
                         ptx::tma_load_3d_pair(ssfa + kSfaBytes, &tm_sfb, 0, kt * kSfChunksK, rcb, full0 + 8u * stage);
                     }
@@ -337,17 +342,26 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 if (trace) SOL_TRACE(8, it);
                 const uint32_t d_tmem = tmem_base + x * kAccStride;
                 for (int kt = 0; kt < k_tiles; ++kt) {
-                    if (!no_sf_wait) {
-                        // the copy warps waited for this stage's loads, so their barrier covers A and B too;
-                        // `sf_seen`: the previous k-tile already saw this barrier complete (peek below)
-                        if (!sf_seen &&
+                    // two conditions per k-tile: the scales are in TMEM (`sf_ready`, signalled by the copy warps)
+                    // and A and B are in shared memory (`full`); `sf_seen`: the previous k-tile already saw
+                    // both complete (peek below)
+                    if (!sf_seen) {
+                        if (!no_sf_wait &&
                             !wait_bounded(sf_ready_bar(sf_buf), sf_phase, abort_flag, p.status, 0x500u | sf_buf)) {
                             ok = false;
                             break;
                         }
-                    } else if (!wait_bounded(full_bar(stage), phase, abort_flag, p.status, 0x300u | stage)) {
-                        ok = false;
-                        break;
+                        if (!wait_bounded(full_bar(stage), phase, abort_flag, p.status, 0x300u | stage)) {
+                            ok = false;
+                            break;
+                        }
+                        // diagnostic build without scale copies: nobody else waits for the scale tiles, and the
+                        // stage must not be released (and its barrier re-armed) before they have landed
+                        if (no_sf_wait && !(p.dbg & kDbgNoSfLoad) &&
+                            !wait_bounded(sf_full_bar(stage), phase, abort_flag, p.status, 0x310u | stage)) {
+                            ok = false;
+                            break;
+                        }
                     }
                     ptx::tc_fence_after_sync();
                     if (trace) SOL_TRACE(6, gi);
@@ -379,9 +393,12 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     const uint32_t nb = sf_buf + 1 == kSfBufs ? 0u : sf_buf + 1;
                     const uint32_t np = sf_buf + 1 == kSfBufs ? sf_phase ^ 1u : sf_phase;
                     // commit frees the stage in both CTAs; the peek tells whether the next buffer is ready
+                    const int ns = stage + 1 == kStages ? 0 : stage + 1;
+                    const uint32_t nph = stage + 1 == kStages ? phase ^ 1u : phase;
                     bool seen = false;
-                    if (elected) seen = ptx::tc_commit_pair_mcast_and_peek(empty_bar(stage), 3, sf_ready_bar(nb), np);
-                    sf_seen = __any_sync(0xFFFFFFFFu, seen) != 0;  // keeps the loop warp-uniform
+                    if (elected)
+                        seen = ptx::tc_commit_pair_mcast_and_peek2(empty_bar(stage), 3, sf_ready_bar(nb), np, full_bar(ns), nph);
+                    sf_seen = !no_sf_wait && __any_sync(0xFFFFFFFFu, seen) != 0;  // keeps the loop warp-uniform
                     if (trace) SOL_TRACE(3, gi);
                     ++gi;
                     sf_buf = nb;
@@ -412,7 +429,8 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             bool ok = true;
             for (int t = pair; ok && t < total_tiles; t += num_pairs) {
                 for (int kt = 0; kt < k_tiles; ++kt) {
-                    if (!wait_bounded(full_bar(stage), phase, abort_flag, p.status, 0x600u | stage)) {
+                    if (!(kTuning && (p.dbg & kDbgNoSfLoad)) &&
+                        !wait_bounded(sf_full_bar(stage), phase, abort_flag, p.status, 0x600u | stage)) {
                         ok = false;
                         break;
                     }

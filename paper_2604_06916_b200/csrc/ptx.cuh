@@ -312,6 +312,22 @@ __device__ __forceinline__ bool tc_commit_pair_mcast_and_peek(uint32_t bar, uint
         : "memory");
     return done != 0;
 }
+// The same with two barriers tested (both must have completed their phase for `true`).
+__device__ __forceinline__ bool tc_commit_pair_mcast_and_peek2(uint32_t bar, uint16_t mask, uint32_t peek_a,
+                                                               uint32_t parity_a, uint32_t peek_b, uint32_t parity_b) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%3], %4;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 q, [%5], %6;\n\t"
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%1], %2;\n\t"
+        "and.pred p, p, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "h"(mask), "r"(peek_a), "r"(parity_a), "r"(peek_b), "r"(parity_b)
+        : "memory");
+    return done != 0;
+}
 __device__ __forceinline__ void tc_copy_sf_pair(uint32_t taddr, uint64_t s_desc) {
     asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(s_desc) : "memory");
 }
