@@ -27,7 +27,7 @@ constexpr bool kTuning = true;
 #else
 constexpr bool kTuning = false;
 #endif
-enum : uint32_t { kDbgNoSfCopy = 1, kDbgNoMma = 2, kDbgNoEpilogue = 4, kDbgNoSfLoad = 8, kDbgNoStore = 16, kDbgTrace = 64 };
+enum : uint32_t { kDbgNoSfCopy = 1, kDbgNoMma = 2, kDbgNoEpilogue = 4, kDbgNoSfLoad = 8, kDbgNoStore = 16, kDbgTrace = 64, kDbgNoBLoad = 128 };
 
 #ifdef SOL_TUNING
 // timeline of the first pair: [event type][k-tile index] = clock64 of the even CTA's SM (rank 1: types 4,5)

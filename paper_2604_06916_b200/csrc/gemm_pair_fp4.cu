@@ -42,6 +42,11 @@ constexpr int kSfCol = kAccStride + kBN;       // 352
 constexpr int kEpiWarpsFp4 = 8;
 constexpr int kSfCopyWarps = 4;                // one per MMA of a k-tile: three tcgen05.cp each
 constexpr int kWarps = 2 + kEpiWarpsFp4 + kSfCopyWarps + 1;
+#ifdef SOL_SF_COPY
+constexpr bool kSfViaStore = false;
+#else
+constexpr bool kSfViaStore = true;   // scale tiles reach TMEM by tcgen05.st from the copy warps, not tcgen05.cp
+#endif
 constexpr int kThreadsFp4 = 32 * kWarps;       // 544
 constexpr int kEpiBytes = kEpiWarpsFp4 * kEpiBufBytes;
 constexpr int kBiasBytes = kEpiWarpsFp4 * 256;  // per epilogue warp: BF16 bias of its two 64-column chunks
@@ -220,7 +225,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             ptx::mbar_init(acc_empty_bar(s), 2 * kEpiWarpsFp4);
             ptx::mbar_init(ovl_free_bar(s), 2 * kEpiWarpsFp4);
         }
-        for (int s = 0; s < kSfBufs; ++s) ptx::mbar_init(sf_ready_bar(s), kSfCopyWarps);
+        for (int s = 0; s < kSfBufs; ++s) ptx::mbar_init(sf_ready_bar(s), kSfViaStore ? 2 * kSfCopyWarps : kSfCopyWarps);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tm_a);
@@ -245,7 +250,9 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         // ------------------------------------------------------------ TMA producer: A and B tiles (both CTAs)
         const bool elected = ptx::elect_one();
         const uint32_t full0 = ptx::map_to_cta(full_bar(0), 0);  // the even CTA's barriers
-        const uint32_t tx = 2u * (kABytes + kBBytes);
+        const bool no_b = kTuning && (p.dbg & kDbgNoBLoad);
+        const uint32_t tx = 2u * (kABytes + (no_b ? 0 : kBBytes));
+        [[maybe_unused]] int gi_trace = 0;
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -261,10 +268,11 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     break;
                 }
                 const uint32_t sa = smem_base + stage * kStageBytes;
+                if (kTuning && (p.dbg & kDbgTrace) && leader) { SOL_TRACE(0, gi_trace); ++gi_trace; }
                 if (elected) {
                     if (leader) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
                     ptx::tma_load_2d_pair(sa, &tm_a, kx, m0, full0 + 8u * stage);
-                    ptx::tma_load_2d_pair(sa + kABytes, &tm_b, kx, nb0, full0 + 8u * stage);
+                    if (!no_b) ptx::tma_load_2d_pair(sa + kABytes, &tm_b, kx, nb0, full0 + 8u * stage);
                 }
                 if (++stage == kStages) {
                     stage = 0;
@@ -277,7 +285,8 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         // ------------------------------------------------------------ TMA producer: scale-factor tiles (both CTAs)
         if (!(kTuning && (p.dbg & kDbgNoSfLoad))) {
             const bool elected = ptx::elect_one();
-            const uint32_t full0 = ptx::map_to_cta(sf_full_bar(0), 0);
+            // store path: each CTA's tiles complete on its own barrier, where its own copy warps wait
+            const uint32_t full0 = ptx::map_to_cta(sf_full_bar(0), kSfViaStore ? rank : 0u);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -293,7 +302,8 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     }
                     const uint32_t ssfa = smem_base + stage * kStageBytes + kABytes + kBBytes;
                     if (elected) {
-                        if (leader) ptx::mbar_arrive_expect_tx(sf_full_bar(stage), 2u * kSfLoadBytes);
+                        if (kSfViaStore) ptx::mbar_arrive_expect_tx(sf_full_bar(stage), kSfLoadBytes);
+                        else if (leader) ptx::mbar_arrive_expect_tx(sf_full_bar(stage), 2u * kSfLoadBytes);
                         ptx::tma_load_3d_pair(ssfa, &tm_sfa, 0, kt * kSfChunksK, rca, full0 + 8u * stage);
                         ptx::tma_load_3d_pair(ssfa + kSfaBytes, &tm_sfb, 0, kt * kSfChunksK, rcb, full0 + 8u * stage);
                     }
@@ -417,9 +427,10 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         // ------------------------------------------------------------ scale-factor copy warps (even CTA)
         // tcgen05.cp blocks its issuing warp for ~100 cycles, so the twelve copies of a k-tile are
         // spread over four warps and kept off the MMA thread; the third TMEM buffer hides their latency.
-        if (leader && !(kTuning && (p.dbg & kDbgNoSfCopy))) {
+        if ((leader || kSfViaStore) && !(kTuning && (p.dbg & kDbgNoSfCopy))) {
             const bool elected = ptx::elect_one();
             const int w = warp - (2 + kEpiWarpsFp4);
+            const uint32_t ready0 = ptx::map_to_cta(sf_ready_bar(0), 0);  // the even CTA's barriers
             int stage = 0;
             uint32_t phase = 0;
             uint32_t gi = 0;
@@ -440,9 +451,33 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                         break;
                     }
                     ptx::tc_fence_after_sync();
-                    if (kTuning && (p.dbg & kDbgTrace) && w == 0) SOL_TRACE(4, gi);
+                    if (kTuning && (p.dbg & kDbgTrace) && w == 0 && leader) SOL_TRACE(4, gi);
                     const int nmma = (kt + 1 < k_tiles) ? kMmasPerStage : tail_mmas;
-                    if (elected) {
+                    if (kSfViaStore) {
+                        // Every warp writes its own TMEM quadrant: lane t takes line t (16 bytes) of each
+                        // 512-byte chunk, the four warps together give the four-fold replication that the
+                        // scaled MMA reads.  Nothing of this passes through the tensor pipe.
+                        const uint32_t ssf = smem_base + stage * kStageBytes + kABytes + kBBytes + lane * 16;
+                        const uint32_t sf_t =
+                            tmem_base + kSfCol + sf_buf * kSfBufCols + (static_cast<uint32_t>(warp & 3) << 21);
+                        uint4 v[3 * kSfChunksK];
+#pragma unroll
+                        for (int c = 0; c < kSfChunksK; ++c) {
+                            v[c] = ptx::lds128(ssf + c * 512);
+                            v[kSfChunksK + c] = ptx::lds128(ssf + kSfaBytes + c * 512);
+                            v[2 * kSfChunksK + c] = ptx::lds128(ssf + kSfaBytes + kSfRowChunkBytes + c * 512);
+                        }
+#pragma unroll
+                        for (int c = 0; c < kSfChunksK; ++c) {
+                            ptx::tc_store_32x32b_x4(sf_t + 4 * c, v[c]);
+                            ptx::tc_store_32x32b_x4(sf_t + 16 + 8 * c, v[kSfChunksK + c]);
+                            ptx::tc_store_32x32b_x4(sf_t + 20 + 8 * c, v[2 * kSfChunksK + c]);
+                        }
+                        ptx::tc_wait_st();
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (elected) ptx::mbar_arrive_cluster(ready0 + 8u * sf_buf);
+                    } else if (elected) {
                         const uint32_t ssf = smem_base + stage * kStageBytes + kABytes + kBBytes;
                         const uint32_t sf_t = tmem_base + kSfCol + sf_buf * kSfBufCols;
                         // warp w: scale chunk w of the stage (NVFP4: the scales of MMA w; MXFP4: of MMAs 2w and
@@ -455,7 +490,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                         }
                         ptx::tc_commit_pair(sf_ready_bar(sf_buf));
                     }
-                    if (kTuning && (p.dbg & kDbgTrace) && w == 0) SOL_TRACE(5, gi);
+                    if (kTuning && (p.dbg & kDbgTrace) && w == 0 && leader) SOL_TRACE(5, gi);
                     ++gi;
                     if (++sf_buf == kSfBufs) sf_buf = 0;
                     if (++old_stage == kStages) {
@@ -650,7 +685,10 @@ sol_status_t launch_pair256(int out_mode, bool mx, const void *xq, const void *x
     p.m_tiles = static_cast<int>(ceil_div(p.M, 2 * kBM));
     p.n_tiles = static_cast<int>(ceil_div(p.N, kBN));
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
-    const int max_pairs = dev->sm_count / 2;
+    int max_pairs = dev->sm_count / 2;
+#ifdef SOL_TUNING
+    if (const char *e = getenv("SOL_PAIRS")) max_pairs = atoi(e);
+#endif
     const int pairs = static_cast<int>(tiles < max_pairs ? tiles : max_pairs);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs), 1, 1);

@@ -331,6 +331,20 @@ __device__ __forceinline__ bool tc_commit_pair_mcast_and_peek2(uint32_t bar, uin
 __device__ __forceinline__ void tc_copy_sf_pair(uint32_t taddr, uint64_t s_desc) {
     asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(s_desc) : "memory");
 }
+// Registers to tensor memory: lane t of the warp writes r0..r3 to columns c..c+3 of TMEM lane
+// (quadrant base + t); the quadrant (bits 16.. of taddr) must be the one the warp may access
+// (warp index mod 4).  Asynchronous: tc_wait_st() before the data is handed to another thread.
+__device__ __forceinline__ void tc_store_32x32b_x4(uint32_t taddr, uint4 v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(v.x), "r"(v.y),
+                 "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
+    return v;
+}
 
 }  // namespace ptx
 }  // namespace sol
