@@ -233,6 +233,25 @@ sol_status_t nvfp4_layernorm_quantize(const void *x_bf16, int64_t M, int64_t K, 
                                       void *stream);
 
 /*
+ * Scaled-dot-product attention of a DiT block in BF16 (the rollout models of Section 4.1 are
+ * diffusion transformers; the method quantizes their linear layers, Section 3, and leaves attention
+ * in BF16 in the FP4 and in the BF16 path alike):
+ *     out[b, s, h, :] = sum_t softmax_t( q[b,s,h,:] . k[b,t,h,:] / sqrt(128) ) v[b,t,h,:]
+ * No mask, no dropout, head dimension 128.  Scores and sums in FP32, probabilities rounded to BF16
+ * before the product with V, output rounded to BF16.
+ *   q, out   [batch, seq_q, heads, 128] BF16: element (b, s, h, d) at ((b * seq_q + s) * ld + h * 128 + d),
+ *            ld_q / ld_out elements between consecutive tokens (>= heads * 128, multiple of 8), so q, k
+ *            and v may be column slices of one fused projection output
+ *   k, v     [batch, seq_kv, heads, 128] BF16, the same way with ld_k / ld_v
+ * All pointers are device pointers, 16-byte aligned, owned by the caller; out must not alias an input.
+ * Errors: SOL_ERR_NULL_POINTER, SOL_ERR_BAD_SHAPE (a non-positive extent, ld < heads * 128, heads or batch
+ * above 65535), SOL_ERR_ALIGNMENT, SOL_ERR_UNSUPPORTED_ARCH, SOL_ERR_CUDA; nothing is launched on an error.
+ */
+sol_status_t sol_attention_bf16(const void *q, const void *k, const void *v, void *out, int64_t batch, int64_t seq_q,
+                                int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v, int64_t ld_out,
+                                void *stream);
+
+/*
  * BF16 linear, the full-precision stage-2 reference (Section 3.4):
  *     Y[m,n] = bf16_rne( sum_k x[m,k] * w[n,k] + bias[n] ),  FP32 accumulate.
  */

@@ -25,7 +25,7 @@ EXPORTS = [
     "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch", "nvfp4_linear_quantized_out",
     "solrl_select_contrastive", "solrl_rank_consistency", "sol_mxfp4_scale_bytes", "mxfp4_quantize",
     "mxfp4_linear", "nvfp4_linear_split_out", "nvfp4_quantize_into",
-    "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale", "nvfp4_layernorm_quantize",
+    "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale", "nvfp4_layernorm_quantize", "sol_attention_bf16",
 ]
 
 _lib = None
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_quantize_linear_delayed.restype = i32
     L.nvfp4_quantize_linear_delayed.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, sz, vp]
     L.sol_roll_tensor_scale.restype, L.sol_roll_tensor_scale.argtypes = i32, [vp, vp]
+    L.sol_attention_bf16.restype = i32
+    L.sol_attention_bf16.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, vp]
     L.nvfp4_layernorm_quantize.restype = i32
     L.nvfp4_layernorm_quantize.argtypes = [vp, i64, i64, i64, vp, vp, i64, ctypes.c_float, vp, vp, vp, vp, vp]
     L.sol_last_device_status.restype = i32
@@ -317,6 +319,35 @@ def nvfp4_layernorm_quantize(x, scale, shift, rows_per_sample: int, tensor_scale
                                           float(eps), _ptr(tensor_scale), _ptr(q), _ptr(sf), _ptr(amax_out), _stream()),
            "nvfp4_layernorm_quantize")
     return q, sf
+
+
+def sol_attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor | None = None):
+    """softmax(q k^T / sqrt(128)) v per batch element and head.
+
+    q [B, Sq, H, 128], k and v [B, Skv, H, 128], BF16; the last two dimensions contiguous, the batch
+    dimension densely on top of the token dimension (stride(0) == S * stride(1)) -- views into a fused
+    projection output qualify.  Returns [B, Sq, H, 128].
+    """
+    for name, t in (("q", q), ("k", k), ("v", v)):
+        if t.dtype != torch.bfloat16 or t.dim() != 4 or t.shape[3] != 128:
+            raise ValueError(f"{name} must be a [B, S, H, 128] BF16 tensor")
+        if t.stride(3) != 1 or (t.shape[2] > 1 and t.stride(2) != 128) or \
+                (t.shape[0] > 1 and t.shape[1] > 1 and t.stride(0) != t.shape[1] * t.stride(1)):
+            raise ValueError(f"{name}: heads and head dimension must be contiguous, batches stacked densely")
+    B, Sq, H, _ = q.shape
+
+    def pitch(t):  # elements between consecutive tokens (a dimension of extent 1 has no meaningful stride)
+        if t.shape[1] > 1:
+            return t.stride(1)
+        return t.stride(0) if t.shape[0] > 1 else t.shape[2] * 128
+
+    if k.shape != v.shape or k.shape[0] != B or k.shape[2] != H:
+        raise ValueError("k and v must share [B, Skv, H, 128] with q's batch and heads")
+    if out is None:
+        out = torch.empty((B, Sq, H, 128), dtype=torch.bfloat16, device=q.device)
+    _check(lib().sol_attention_bf16(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, Sq, k.shape[1], H, pitch(q), pitch(k),
+                                    pitch(v), pitch(out), _stream()), "sol_attention_bf16")
+    return out
 
 
 def mxfp4_scale_bytes(rows: int, K: int, layout: int = SF_SWIZZLED_128x4) -> int:

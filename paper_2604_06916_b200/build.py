@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "gemm_pair.cu", "gemm_pair_fp4.cu", "static_scratch.cu",
-           "lora_merge.cu", "selection.cu", "layernorm_quantize.cu"]
+           "lora_merge.cu", "selection.cu", "layernorm_quantize.cu", "attention.cu"]
 LIB = os.path.join(HERE, "libsol_nvfp4.so")
 
 

@@ -86,6 +86,19 @@ bool make_tmap_2d(CUtensorMap *out, CUtensorMapDataType dtype, uint32_t elem_byt
               swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch1_bytes,
+                       uint64_t pitch2_bytes, uint32_t box0, uint32_t box1) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[3] = {d0, d1, d2};
+    cuuint64_t strides[2] = {pitch1_bytes, pitch2_bytes};
+    cuuint32_t box[3] = {box0, box1, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_tmap_sf(CUtensorMap *out, const void *base, uint64_t chunks_k, uint64_t row_chunks,
                   uint32_t box_row_chunks, uint32_t box_k_chunks) {
     EncodeTiledFn fn = encode_fn();
@@ -463,6 +476,24 @@ sol_status_t nvfp4_layernorm_quantize(const void *x_bf16, int64_t M, int64_t K, 
     return launch_layernorm_quantize(x_bf16, M, K, ldx, scale_bf16, shift_bf16, rows_per_sample, eps, tensor_scale,
                                      q_out, sf_out, reinterpret_cast<uint32_t *>(amax_out),
                                      static_cast<cudaStream_t>(stream));
+}
+
+sol_status_t sol_attention_bf16(const void *q, const void *k, const void *v, void *out, int64_t batch, int64_t seq_q,
+                                int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v, int64_t ld_out,
+                                void *stream) {
+    if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return SOL_ERR_NULL_POINTER;
+    const int64_t cols = heads * 128;
+    if (batch <= 0 || seq_q <= 0 || seq_kv <= 0 || heads <= 0 || batch > 65535 || heads > 65535 ||
+        seq_q > (1LL << 24) || seq_kv > (1LL << 24) || ld_q < cols || ld_k < cols || ld_v < cols || ld_out < cols)
+        return SOL_ERR_BAD_SHAPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || ld_q % 8 != 0 || ld_k % 8 != 0 ||
+        ld_v % 8 != 0 || ld_out % 8 != 0)
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return attn::launch_attention(q, k, v, out, batch, seq_q, seq_kv, heads, ld_q, ld_k, ld_v, ld_out,
+                                  static_cast<cudaStream_t>(stream));
 }
 
 sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,

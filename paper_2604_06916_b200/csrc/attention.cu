@@ -1,0 +1,328 @@
+// Scaled-dot-product attention of a DiT block (BF16 in and out, head dimension 128, no mask):
+//     O = softmax(Q K^T / sqrt(128)) V   per batch element and head.
+// The linear layers around it run in NVFP4; attention itself stays in BF16 in both the FP4 and the
+// BF16 path of the method, so this kernel is what a whole-block forward needs besides the linears.
+//
+// One CTA per 128 query rows of one (batch, head); K and V stream through a two-stage ring of
+// 128-row tiles.  Per K/V tile j:
+//     S_j = Q K_j^T            tcgen05.mma kind::f16, 128 x 128 x 128, accumulator in TMEM (two S buffers)
+//     softmax                  one thread per query row (= TMEM lane): tcgen05.ld of the row, running
+//                              max m and sum l (online softmax), p = exp2(s c - m), P as BF16 into
+//                              shared memory in the K-major 128-byte-swizzled operand layout
+//     O  = alpha O + P V_j     O rescaled in TMEM by the row's alpha when its max moved (tcgen05.ld /
+//                              st), then tcgen05.mma with V as an MN-major operand (V is [kv][d])
+// S_{j+1} is issued before P_j V_j, so the tensor pipe works on the next scores while the softmax
+// warps work on this tile.  The epilogue divides by l and leaves through TMA stores.
+//
+// Warps: 0 = TMA producer, 1 = TMEM owner and MMA issuer, 2..5 = softmax / epilogue (one per TMEM
+// lane quadrant).  Every mbarrier wait is bounded.
+#include "gemm_common.cuh"
+#include "sol_internal.h"
+
+namespace sol {
+namespace attn {
+namespace {
+
+using gemm::wait_bounded;
+
+constexpr int kD = 128;                 // head dimension
+constexpr int kBQ = 128;                // query rows per CTA
+constexpr int kBKV = 128;               // keys per tile
+constexpr int kBox = 128 * 128;         // bytes of a [128 rows][64 BF16] box
+constexpr int kTile = 2 * kBox;         // a [128][128] BF16 tile: box of columns 0..63, box of 64..127
+constexpr int kKvStages = 2;
+constexpr int kThreads = 192;
+constexpr int kSmem = kTile * (2 + 2 * kKvStages) + 256;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256;
+static_assert(kSmem <= 232448, "shared memory budget");
+
+struct Params {
+    int seq_kv;
+    float scale_log2;      // log2(e) / sqrt(d)
+    uint32_t *status;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const Params p) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t smem_base = ptx::smem_u32(smem_raw);
+    if (smem_base & 1023u) {  // the swizzled operand layout needs 1024-byte alignment
+        if (threadIdx.x == 0) atomicExch(p.status, 0xB00u);
+        return;
+    }
+    const uint32_t sQ = smem_base;                        // Q, later the output staging buffer
+    const uint32_t sK = smem_base + kTile;                // kKvStages tiles
+    const uint32_t sV = sK + kKvStages * kTile;
+    const uint32_t sP = sV + kKvStages * kTile;
+    const uint32_t bar_base = sP + kTile;
+    uint8_t *bar_gen = smem_raw + (bar_base - smem_base);
+    auto bar = [&](int i) { return bar_base + 8u * i; };
+    constexpr int kQFull = 0, kKFull = 1, kKEmpty = 3, kVFull = 5, kVEmpty = 7, kSFull = 9, kSFree = 11, kPFull = 13,
+                  kPvDone = 14, kNumBars = 15;
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * kNumBars);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * kNumBars + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int q0 = blockIdx.x * kBQ, head = blockIdx.y, batch = blockIdx.z;
+    const int n_tiles = (p.seq_kv + kBKV - 1) / kBKV;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kNumBars; ++i) ptx::mbar_init(bar(i), (i == kSFree || i == kSFree + 1 || i == kPFull) ? 4 : 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tm_q);
+        ptx::prefetch_tmap(&tm_k);
+        ptx::prefetch_tmap(&tm_v);
+        ptx::prefetch_tmap(&tm_o);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(tmem_ptr_smem), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_ptr_smem;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (ptx::elect_one()) {
+            const int x0 = head * kD;
+            ptx::mbar_arrive_expect_tx(bar(kQFull), kTile);
+            ptx::tma_load_3d(sQ, &tm_q, x0, q0, batch, bar(kQFull));
+            ptx::tma_load_3d(sQ + kBox, &tm_q, x0 + 64, q0, batch, bar(kQFull));
+            for (int j = 0; j < n_tiles; ++j) {
+                const int st = j & 1;
+                const uint32_t par = static_cast<uint32_t>(j >> 1) & 1u;
+                if (!wait_bounded(bar(kKEmpty + st), par ^ 1u, abort_flag, p.status, 0xB10u | st)) break;
+                ptx::mbar_arrive_expect_tx(bar(kKFull + st), kTile);
+                ptx::tma_load_3d(sK + st * kTile, &tm_k, x0, j * kBKV, batch, bar(kKFull + st));
+                ptx::tma_load_3d(sK + st * kTile + kBox, &tm_k, x0 + 64, j * kBKV, batch, bar(kKFull + st));
+                if (!wait_bounded(bar(kVEmpty + st), par ^ 1u, abort_flag, p.status, 0xB20u | st)) break;
+                ptx::mbar_arrive_expect_tx(bar(kVFull + st), kTile);
+                ptx::tma_load_3d(sV + st * kTile, &tm_v, x0, j * kBKV, batch, bar(kVFull + st));
+                ptx::tma_load_3d(sV + st * kTile + kBox, &tm_v, x0 + 64, j * kBKV, batch, bar(kVFull + st));
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (ptx::elect_one()) {
+            // BF16 x BF16 -> FP32, M = 128, N = 128; bit 16: B is MN-major (V)
+            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(128 >> 3) << 17) |
+                                      (static_cast<uint32_t>(128 >> 4) << 24);
+            const uint32_t idesc_pv = idesc_qk | (1u << 16);
+            auto issue_qk = [&](int j) {
+                const int st = j & 1;
+                const uint32_t d_tmem = tmem_base + kColS + st * 128;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {  // 16 elements of d per instruction
+                    const uint64_t a = ptx::smem_desc_sw128(sQ + (i >> 2) * kBox) + 2u * (i & 3);
+                    const uint64_t b = ptx::smem_desc_sw128(sK + st * kTile + (i >> 2) * kBox) + 2u * (i & 3);
+                    ptx::mma_bf16(d_tmem, a, b, idesc_qk, i > 0);
+                }
+                ptx::tc_commit(bar(kSFull + st));
+                ptx::tc_commit(bar(kKEmpty + st));
+            };
+            bool ok = wait_bounded(bar(kQFull), 0, abort_flag, p.status, 0xB30u) &&
+                      wait_bounded(bar(kKFull), 0, abort_flag, p.status, 0xB31u);
+            if (ok) {
+                ptx::tc_fence_after_sync();
+                issue_qk(0);
+            }
+            for (int j = 0; ok && j < n_tiles; ++j) {
+                if (j + 1 < n_tiles) {  // the next tile's scores first: they overlap this tile's softmax
+                    const int st = (j + 1) & 1;
+                    const uint32_t u = static_cast<uint32_t>(j + 1) >> 1;
+                    if (!wait_bounded(bar(kKFull + st), u & 1u, abort_flag, p.status, 0xB40u | st)) break;
+                    if (u > 0 && !wait_bounded(bar(kSFree + st), (u - 1) & 1u, abort_flag, p.status, 0xB50u | st)) break;
+                    ptx::tc_fence_after_sync();
+                    issue_qk(j + 1);
+                }
+                const int st = j & 1;
+                if (!wait_bounded(bar(kPFull), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, 0xB60u)) break;
+                if (!wait_bounded(bar(kVFull + st), static_cast<uint32_t>(j >> 1) & 1u, abort_flag, p.status, 0xB70u | st))
+                    break;
+                ptx::tc_fence_after_sync();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {  // 16 keys per instruction
+                    const uint64_t a = ptx::smem_desc_sw128(sP + (i >> 2) * kBox) + 2u * (i & 3);
+                    const uint64_t b = ptx::smem_desc_sw128_mn(sV + st * kTile + i * 2048, kBox, 1024);
+                    ptx::mma_bf16(tmem_base + kColO, a, b, idesc_pv, (j | i) != 0);
+                }
+                ptx::tc_commit(bar(kPvDone));
+                ptx::tc_commit(bar(kVEmpty + st));
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ softmax and epilogue: thread = query row
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;                       // row of the tile = TMEM lane
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        const uint32_t p_row = sP + r * 128;
+        const uint32_t sw = static_cast<uint32_t>(r & 7);
+        float m = -INFINITY, l = 0.0f;
+        bool ok = true;
+        for (int j = 0; j < n_tiles; ++j) {
+            const int st = j & 1;
+            if (!wait_bounded(bar(kSFull + st), static_cast<uint32_t>(j >> 1) & 1u, abort_flag, p.status, 0xB80u | st)) {
+                ok = false;
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            uint32_t s[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(t_lane + kColS + st * 128 + 32 * c, s[c]);
+            ptx::tmem_ld_wait();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(kSFree + st));  // the scores are in registers
+            const int valid = p.seq_kv - j * kBKV;              // keys of this tile that exist (>= 1)
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    float v = __uint_as_float(s[c][e]);
+                    if (c * 32 + e >= valid) v = -INFINITY;
+                    s[c][e] = __float_as_uint(v);
+                    mx = fmaxf(mx, v);
+                }
+            const float m_new = fmaxf(m, mx * p.scale_log2);
+            const float alpha = ex2(m - m_new);   // 0 on the first tile (m = -inf)
+            float sum = 0.0f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    const float p0 = ex2(fmaf(__uint_as_float(s[c][e]), p.scale_log2, -m_new));
+                    const float p1 = ex2(fmaf(__uint_as_float(s[c][e + 1]), p.scale_log2, -m_new));
+                    sum += p0 + p1;
+                    s[c][e >> 1] = pack_bf16(p0, p1);  // 16 words per 32 keys, packed in place
+                }
+            l = fmaf(l, alpha, sum);
+            m = m_new;
+            if (j > 0) {
+                // the previous P.V has completed: P's buffer is free and O may be rescaled
+                if (!wait_bounded(bar(kPvDone), static_cast<uint32_t>(j - 1) & 1u, abort_flag, p.status, 0xB90u)) {
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                if (__any_sync(0xFFFFFFFFu, alpha != 1.0f)) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        ptx::tmem_ld_32x32(t_lane + kColO + 32 * c, o);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        ptx::tmem_st_32x32(t_lane + kColO + 32 * c, o);
+                    }
+                    ptx::tc_wait_st();
+                }
+            }
+            // P row: 128 BF16 = 16 chunks of 16 bytes; chunk ch lives in box ch / 8 at position (ch % 8) ^ (row % 8)
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int ch = c * 4 + q;
+                    const uint32_t addr = p_row + (ch >> 3) * kBox + ((static_cast<uint32_t>(ch & 7) ^ sw) << 4);
+                    sts128(addr, s[c][4 * q], s[c][4 * q + 1], s[c][4 * q + 2], s[c][4 * q + 3]);
+                }
+            ptx::fence_proxy_async_smem();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(bar(kPFull));
+        }
+        if (ok && wait_bounded(bar(kPvDone), static_cast<uint32_t>(n_tiles - 1) & 1u, abort_flag, p.status, 0xBA0u)) {
+            ptx::tc_fence_after_sync();
+            const float inv = 1.0f / l;
+            const uint32_t o_row = sQ + r * 128;  // Q is no longer read: every MMA has completed
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t o[32];
+                ptx::tmem_ld_32x32(t_lane + kColO + 32 * c, o);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        w[e] = pack_bf16(__uint_as_float(o[8 * q + 2 * e]) * inv, __uint_as_float(o[8 * q + 2 * e + 1]) * inv);
+                    const int ch = c * 4 + q;
+                    sts128(o_row + (ch >> 3) * kBox + ((static_cast<uint32_t>(ch & 7) ^ sw) << 4), w[0], w[1], w[2], w[3]);
+                }
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {  // this warp's 32 rows, two boxes of 64 columns (clipped at the end of the sequence)
+                ptx::tma_store_3d(&tm_o, head * kD, q0 + quad * 32, batch, sQ + quad * 32 * 128);
+                ptx::tma_store_3d(&tm_o, head * kD + 64, q0 + quad * 32, batch, sQ + kBox + quad * 32 * 128);
+                ptx::tma_store_commit();
+                ptx::tma_store_wait_all<0>();
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace
+
+sol_status_t launch_attention(const void *q, const void *k, const void *v, void *out, int64_t batch, int64_t seq_q,
+                              int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v, int64_t ld_out,
+                              cudaStream_t stream) {
+    CUtensorMap tm_q, tm_k, tm_v, tm_o;
+    const uint64_t cols = static_cast<uint64_t>(heads) * kD;
+    auto make = [&](CUtensorMap *tm, const void *base, int64_t seq, int64_t ld, uint32_t box_rows) {
+        return make_tmap_3d_bf16(tm, base, cols, static_cast<uint64_t>(seq), static_cast<uint64_t>(batch),
+                                 static_cast<uint64_t>(ld) * 2, static_cast<uint64_t>(seq) * ld * 2, 64, box_rows);
+    };
+    if (!make(&tm_q, q, seq_q, ld_q, kBQ) || !make(&tm_k, k, seq_kv, ld_k, kBKV) || !make(&tm_v, v, seq_kv, ld_v, kBKV) ||
+        !make(&tm_o, out, seq_q, ld_out, 32))
+        return SOL_ERR_CUDA;
+    Params p{};
+    p.seq_kv = static_cast<int>(seq_kv);
+    p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(kD));
+    p.status = device_status_word();
+    static bool configured[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SOL_ERR_CUDA;
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+            return SOL_ERR_CUDA;
+        configured[dev] = true;
+    }
+    const dim3 grid(static_cast<unsigned>((seq_q + kBQ - 1) / kBQ), static_cast<unsigned>(heads),
+                    static_cast<unsigned>(batch));
+    attention_kernel<<<grid, kThreads, kSmem, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
+    return launch_status();
+}
+
+}  // namespace attn
+}  // namespace sol

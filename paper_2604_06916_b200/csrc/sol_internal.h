@@ -103,6 +103,17 @@ bool make_tmap_2d(CUtensorMap *out, CUtensorMapDataType dtype, uint32_t elem_byt
                   uint64_t inner, uint64_t outer, uint64_t pitch_bytes, uint32_t box_inner,
                   uint32_t box_outer, CUtensorMapSwizzle swizzle);
 
+// [d2][d1][d0] BF16 tensor with byte pitches between rows (d1) and slabs (d2); 128-byte swizzle, boxes of
+// box0 x box1 x 1 elements.
+bool make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t pitch1_bytes,
+                       uint64_t pitch2_bytes, uint32_t box0, uint32_t box1);
+
+namespace attn {
+sol_status_t launch_attention(const void *q, const void *k, const void *v, void *out, int64_t batch, int64_t seq_q,
+                              int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v, int64_t ld_out,
+                              cudaStream_t stream);
+}
+
 // Scale-factor buffer in the chunked layout as a 3-D tensor [row chunk][k chunk][128 x u32]; the box
 // covers `box_k_chunks` k-chunks of `box_row_chunks` row chunks (out-of-range chunks read as zero).
 bool make_tmap_sf(CUtensorMap *out, const void *base, uint64_t chunks_k, uint64_t row_chunks,

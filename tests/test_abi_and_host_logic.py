@@ -133,6 +133,13 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.nvfp4_layernorm_quantize(p, 4, 8192, 8192, p, p, 4, 1e-6, p, p, p, None, None) == SHAPE  # K > 4096
     assert L.nvfp4_layernorm_quantize(p, 4, 64, 64, p, p, 0, 1e-6, p, p, p, None, None) == SHAPE
     assert L.nvfp4_layernorm_quantize(p, 4, 64, 64, p + 8, p, 4, 1e-6, p, p, p, None, None) == ALIGN
+    # attention
+    assert L.sol_attention_bf16(p, p, None, p, 1, 4, 4, 1, 128, 128, 128, 128, None) == NULLP
+    assert L.sol_attention_bf16(p, p, p, p, 1, 0, 4, 1, 128, 128, 128, 128, None) == SHAPE
+    assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 2, 128, 256, 256, 256, None) == SHAPE      # pitch < heads * 128
+    assert L.sol_attention_bf16(p, p, p, p, 70000, 4, 4, 1, 128, 128, 128, 128, None) == SHAPE
+    assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 1, 132, 128, 128, 128, None) == ALIGN      # pitch % 8
+    assert L.sol_attention_bf16(p, p + 8, p, p, 1, 4, 4, 1, 128, 128, 128, 128, None) == ALIGN
     # MXFP4
     assert L.sol_mxfp4_scale_bytes(256, 512, 0) == 256 * 16 and L.sol_mxfp4_scale_bytes(256, 512, 1) == 2 * 4 * 512
     assert L.sol_mxfp4_scale_bytes(130, 160, 1) == 2 * 2 * 512 and L.sol_mxfp4_scale_bytes(4, 48, 1) == 0

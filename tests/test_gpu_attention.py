@@ -1,0 +1,106 @@
+"""GPU parity: BF16 attention (head dimension 128) through the C ABI against the FP64 oracle.
+
+Tolerance (derived in oracle.attention.attention_tolerance): 2^-8 |O| + 2^-8 max|v| -- output
+rounding to BF16, probabilities rounded to BF16 before the product with V, row sum from the
+unrounded probabilities.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as OA
+from paper_2604_06916_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2604_06916_b200 import binding
+    binding.lib()
+    return binding
+
+
+def f64(t):
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def check(B, q, k, v, rows=None):
+    out = B.sol_attention_bf16(q, k, v)
+    torch.cuda.synchronize()
+    assert B.sol_last_device_status() == 0
+    qn, kn, vn = f64(q), f64(k), f64(v)
+    ref = OA.attention(qn, kn, vn, rows=rows)
+    got = f64(out) if rows is None else f64(out)[:, rows]
+    tol = OA.attention_tolerance(ref, vn)
+    err = np.abs(got - ref)
+    worst = float((err / tol).max())
+    assert worst <= 1.0, f"max err/tol {worst:.3f} at {np.unravel_index((err / tol).argmax(), err.shape)}"
+    return worst
+
+
+@pytest.mark.parametrize("batch,seq,heads", [(1, 128, 1), (1, 256, 1), (1, 640, 2), (2, 384, 3)])
+def test_whole_tiles(B, batch, seq, heads):
+    _, q, k, v = workloads.make_qkv(batch, seq, heads, seq + heads, "cuda")
+    check(B, q, k, v)
+
+
+@pytest.mark.parametrize("seq_q,seq_kv", [(1, 1), (5, 3), (200, 333), (129, 127), (130, 16), (64, 1000)])
+def test_ragged_sequences_and_cross_lengths(B, seq_q, seq_kv):
+    _, q, _, _ = workloads.make_qkv(2, seq_q, 2, 11, "cuda")
+    _, _, k, v = workloads.make_qkv(2, seq_kv, 2, 12, "cuda")
+    check(B, q, k, v)
+
+
+def test_sharp_softmax_moves_the_running_max(B):
+    # large scores: the row maximum keeps moving from tile to tile, so O is rescaled in TMEM many times
+    _, q, k, v = workloads.make_qkv(1, 1024, 2, 21, "cuda", q_gain=6.0)
+    check(B, q, k, v)
+
+
+def test_dense_tensors_and_output_view(B):
+    _, q, k, v = workloads.make_qkv(2, 300, 2, 31, "cuda")
+    qd, kd, vd = q.contiguous(), k.contiguous(), v.contiguous()
+    want = B.sol_attention_bf16(q, k, v)
+    got = B.sol_attention_bf16(qd, kd, vd)
+    assert torch.equal(want, got)
+    # output into a column slice of a wider buffer; the rest of the buffer is not touched
+    wide = torch.full((2, 300, 3 * 256), 7.0, dtype=torch.bfloat16, device="cuda")
+    view = wide[:, :, 256:512].unflatten(2, (2, 128))
+    B.sol_attention_bf16(q, k, v, out=view)
+    torch.cuda.synchronize()
+    assert torch.equal(view, want)
+    assert torch.all(wide[:, :, :256] == 7.0) and torch.all(wide[:, :, 512:] == 7.0)
+
+
+def test_value_of_one_gives_one_and_single_hot_key(B):
+    _, q, k, v = workloads.make_qkv(1, 512, 1, 41, "cuda")
+    ones = torch.ones_like(v)
+    assert torch.all(B.sol_attention_bf16(q, k, ones) == 1.0)
+    # one key aligned with every query and much longer than the rest: the output is that key's value row
+    k2 = k.clone()
+    k2[0, 300, 0] = 0
+    q2 = torch.zeros_like(q)
+    q2[..., 5] = 8.0
+    k2[..., 5] = 0
+    k2[0, 300, 0, 5] = 64.0
+    out = B.sol_attention_bf16(q2, k2, v)
+    assert torch.equal(out[0, :, 0], v[0, 300, 0].expand(512, 128))
+
+
+def test_flux_geometry_sampled_rows(B):
+    # the bench's shape: 8 samples x 4608 tokens x 24 heads; the oracle computes 3 query rows per tile position
+    _, q, k, v = workloads.make_qkv(8, 4608, 24, 51, "cuda")
+    out = B.sol_attention_bf16(q, k, v)
+    torch.cuda.synchronize()
+    assert B.sol_last_device_status() == 0
+    rows = [0, 127, 128, 2303, 4500, 4607]
+    for b, h in [(0, 0), (3, 11), (7, 23)]:
+        ref = OA.attention(f64(q[b:b + 1, :, h:h + 1]), f64(k[b:b + 1, :, h:h + 1]), f64(v[b:b + 1, :, h:h + 1]), rows=rows)
+        got = f64(out[b:b + 1, :, h:h + 1])[:, rows]
+        tol = OA.attention_tolerance(ref, f64(v[b:b + 1, :, h:h + 1]))
+        assert np.all(np.abs(got - ref) <= tol)
+    # and every output against the library routine within a looser screen (both round P to BF16)
+    lib = torch.nn.functional.scaled_dot_product_attention(q.transpose(1, 2), k.transpose(1, 2), v.transpose(1, 2))
+    d = (out.transpose(1, 2).float() - lib.float()).abs().max().item()
+    assert d <= 2.0 ** -6 * 2.5, d
