@@ -3,16 +3,18 @@
 // The linear layers around it run in NVFP4; attention itself stays in BF16 in both the FP4 and the
 // BF16 path of the method, so this kernel is what a whole-block forward needs besides the linears.
 //
-// One CTA per 128 query rows of one (batch, head); K and V stream through a two-stage ring of
-// 128-row tiles.  Per K/V tile j:
-//     S_j = Q K_j^T            tcgen05.mma kind::f16, 128 x 128 x 128, accumulator in TMEM (two S buffers)
+// One CTA per 128 query rows of one (batch, head), two CTAs per SM.  Per 128-key tile j:
+//     S_j = Q K_j^T            tcgen05.mma kind::f16, 128 x 128 x 128, accumulator in TMEM
 //     softmax                  one thread per query row (= TMEM lane): tcgen05.ld of the row, running
-//                              max m and sum l (online softmax), p = exp2(s c - m), P as BF16 into
-//                              shared memory in the K-major 128-byte-swizzled operand layout
+//                              max m and sum l (online softmax), p = exp2(s c - m); P goes back into
+//                              the columns S occupied, as packed BF16 pairs (tcgen05.st)
 //     O  = alpha O + P V_j     O rescaled in TMEM by the row's alpha when its max moved (tcgen05.ld /
-//                              st), then tcgen05.mma with V as an MN-major operand (V is [kv][d])
-// S_{j+1} is issued before P_j V_j, so the tensor pipe works on the next scores while the softmax
-// warps work on this tile.  The epilogue divides by l and leaves through TMA stores.
+//                              st), then tcgen05.mma with A = P from TMEM and V as an MN-major
+//                              shared-memory operand (V is [kv][d])
+// Inside a CTA the three steps of a tile run one after the other; the SM's second CTA fills the
+// tensor pipe while this one is in its softmax, and the other way round: 96 KB of shared memory
+// (Q, one K tile, one V tile) and 256 TMEM columns (S/P and O) per CTA make room for two.
+// The epilogue divides by l and leaves through TMA stores (staged where Q was).
 //
 // Warps: 0 = TMA producer, 1 = TMEM owner and MMA issuer, 2..5 = softmax / epilogue (one per TMEM
 // lane quadrant).  Every mbarrier wait is bounded.
@@ -30,12 +32,11 @@ constexpr int kBQ = 128;                // query rows per CTA
 constexpr int kBKV = 128;               // keys per tile
 constexpr int kBox = 128 * 128;         // bytes of a [128 rows][64 BF16] box
 constexpr int kTile = 2 * kBox;         // a [128][128] BF16 tile: box of columns 0..63, box of 64..127
-constexpr int kKvStages = 2;
 constexpr int kThreads = 192;
-constexpr int kSmem = kTile * (2 + 2 * kKvStages) + 256;
-constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256;
-static_assert(kSmem <= 232448, "shared memory budget");
+constexpr int kSmem = 3 * kTile + 256;
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kColS = 0, kColO = 128;   // P overwrites columns [0, 64) of S
+static_assert(2 * (kSmem + 1024) <= 233472, "two CTAs per SM");
 
 struct Params {
     int seq_kv;
@@ -57,7 +58,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const Params p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -67,14 +68,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         return;
     }
     const uint32_t sQ = smem_base;                        // Q, later the output staging buffer
-    const uint32_t sK = smem_base + kTile;                // kKvStages tiles
-    const uint32_t sV = sK + kKvStages * kTile;
-    const uint32_t sP = sV + kKvStages * kTile;
-    const uint32_t bar_base = sP + kTile;
+    const uint32_t sK = smem_base + kTile;
+    const uint32_t sV = sK + kTile;
+    const uint32_t bar_base = sV + kTile;
     uint8_t *bar_gen = smem_raw + (bar_base - smem_base);
     auto bar = [&](int i) { return bar_base + 8u * i; };
-    constexpr int kQFull = 0, kKFull = 1, kKEmpty = 3, kVFull = 5, kVEmpty = 7, kSFull = 9, kSFree = 11, kPFull = 13,
-                  kPvDone = 14, kNumBars = 15;
+    constexpr int kQFull = 0, kKFull = 1, kKEmpty = 2, kVFull = 3, kVEmpty = 4, kSFull = 5, kPFull = 6, kPvDone = 7,
+                  kNumBars = 8;
     uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * kNumBars);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * kNumBars + 4);
 
@@ -83,7 +83,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int n_tiles = (p.seq_kv + kBKV - 1) / kBKV;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kNumBars; ++i) ptx::mbar_init(bar(i), (i == kSFree || i == kSFree + 1 || i == kPFull) ? 4 : 1);
+        for (int i = 0; i < kNumBars; ++i) ptx::mbar_init(bar(i), i == kPFull ? 4 : 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tm_q);
@@ -108,16 +108,15 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ptx::tma_load_3d(sQ, &tm_q, x0, q0, batch, bar(kQFull));
             ptx::tma_load_3d(sQ + kBox, &tm_q, x0 + 64, q0, batch, bar(kQFull));
             for (int j = 0; j < n_tiles; ++j) {
-                const int st = j & 1;
-                const uint32_t par = static_cast<uint32_t>(j >> 1) & 1u;
-                if (!wait_bounded(bar(kKEmpty + st), par ^ 1u, abort_flag, p.status, 0xB10u | st)) break;
-                ptx::mbar_arrive_expect_tx(bar(kKFull + st), kTile);
-                ptx::tma_load_3d(sK + st * kTile, &tm_k, x0, j * kBKV, batch, bar(kKFull + st));
-                ptx::tma_load_3d(sK + st * kTile + kBox, &tm_k, x0 + 64, j * kBKV, batch, bar(kKFull + st));
-                if (!wait_bounded(bar(kVEmpty + st), par ^ 1u, abort_flag, p.status, 0xB20u | st)) break;
-                ptx::mbar_arrive_expect_tx(bar(kVFull + st), kTile);
-                ptx::tma_load_3d(sV + st * kTile, &tm_v, x0, j * kBKV, batch, bar(kVFull + st));
-                ptx::tma_load_3d(sV + st * kTile + kBox, &tm_v, x0 + 64, j * kBKV, batch, bar(kVFull + st));
+                const uint32_t par = static_cast<uint32_t>(j) & 1u;
+                if (!wait_bounded(bar(kKEmpty), par ^ 1u, abort_flag, p.status, 0xB10u)) break;
+                ptx::mbar_arrive_expect_tx(bar(kKFull), kTile);
+                ptx::tma_load_3d(sK, &tm_k, x0, j * kBKV, batch, bar(kKFull));
+                ptx::tma_load_3d(sK + kBox, &tm_k, x0 + 64, j * kBKV, batch, bar(kKFull));
+                if (!wait_bounded(bar(kVEmpty), par ^ 1u, abort_flag, p.status, 0xB20u)) break;
+                ptx::mbar_arrive_expect_tx(bar(kVFull), kTile);
+                ptx::tma_load_3d(sV, &tm_v, x0, j * kBKV, batch, bar(kVFull));
+                ptx::tma_load_3d(sV + kBox, &tm_v, x0 + 64, j * kBKV, batch, bar(kVFull));
             }
         }
         __syncwarp();
@@ -128,46 +127,29 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(128 >> 3) << 17) |
                                       (static_cast<uint32_t>(128 >> 4) << 24);
             const uint32_t idesc_pv = idesc_qk | (1u << 16);
-            auto issue_qk = [&](int j) {
-                const int st = j & 1;
-                const uint32_t d_tmem = tmem_base + kColS + st * 128;
+            bool ok = wait_bounded(bar(kQFull), 0, abort_flag, p.status, 0xB30u);
+            for (int j = 0; ok && j < n_tiles; ++j) {
+                const uint32_t par = static_cast<uint32_t>(j) & 1u;
+                if (!wait_bounded(bar(kKFull), par, abort_flag, p.status, 0xB40u)) break;
+                ptx::tc_fence_after_sync();
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {  // 16 elements of d per instruction
                     const uint64_t a = ptx::smem_desc_sw128(sQ + (i >> 2) * kBox) + 2u * (i & 3);
-                    const uint64_t b = ptx::smem_desc_sw128(sK + st * kTile + (i >> 2) * kBox) + 2u * (i & 3);
-                    ptx::mma_bf16(d_tmem, a, b, idesc_qk, i > 0);
+                    const uint64_t b = ptx::smem_desc_sw128(sK + (i >> 2) * kBox) + 2u * (i & 3);
+                    ptx::mma_bf16(tmem_base + kColS, a, b, idesc_qk, i > 0);
                 }
-                ptx::tc_commit(bar(kSFull + st));
-                ptx::tc_commit(bar(kKEmpty + st));
-            };
-            bool ok = wait_bounded(bar(kQFull), 0, abort_flag, p.status, 0xB30u) &&
-                      wait_bounded(bar(kKFull), 0, abort_flag, p.status, 0xB31u);
-            if (ok) {
-                ptx::tc_fence_after_sync();
-                issue_qk(0);
-            }
-            for (int j = 0; ok && j < n_tiles; ++j) {
-                if (j + 1 < n_tiles) {  // the next tile's scores first: they overlap this tile's softmax
-                    const int st = (j + 1) & 1;
-                    const uint32_t u = static_cast<uint32_t>(j + 1) >> 1;
-                    if (!wait_bounded(bar(kKFull + st), u & 1u, abort_flag, p.status, 0xB40u | st)) break;
-                    if (u > 0 && !wait_bounded(bar(kSFree + st), (u - 1) & 1u, abort_flag, p.status, 0xB50u | st)) break;
-                    ptx::tc_fence_after_sync();
-                    issue_qk(j + 1);
-                }
-                const int st = j & 1;
-                if (!wait_bounded(bar(kPFull), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, 0xB60u)) break;
-                if (!wait_bounded(bar(kVFull + st), static_cast<uint32_t>(j >> 1) & 1u, abort_flag, p.status, 0xB70u | st))
-                    break;
+                ptx::tc_commit(bar(kSFull));   // also: the previous tile's P.V has completed
+                ptx::tc_commit(bar(kKEmpty));
+                if (!wait_bounded(bar(kPFull), par, abort_flag, p.status, 0xB60u)) break;
+                if (!wait_bounded(bar(kVFull), par, abort_flag, p.status, 0xB70u)) break;
                 ptx::tc_fence_after_sync();
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {  // 16 keys per instruction
-                    const uint64_t a = ptx::smem_desc_sw128(sP + (i >> 2) * kBox) + 2u * (i & 3);
-                    const uint64_t b = ptx::smem_desc_sw128_mn(sV + st * kTile + i * 2048, kBox, 1024);
-                    ptx::mma_bf16(tmem_base + kColO, a, b, idesc_pv, (j | i) != 0);
+                for (int i = 0; i < 8; ++i) {  // 16 keys per instruction: 8 columns of packed P
+                    const uint64_t b = ptx::smem_desc_sw128_mn(sV + i * 2048, kBox, 1024);
+                    ptx::mma_bf16_a_tmem(tmem_base + kColO, tmem_base + kColS + 8 * i, b, idesc_pv, (j | i) != 0);
                 }
-                ptx::tc_commit(bar(kPvDone));
-                ptx::tc_commit(bar(kVEmpty + st));
+                ptx::tc_commit(bar(kVEmpty));
+                if (j + 1 == n_tiles) ptx::tc_commit(bar(kPvDone));
             }
         }
         __syncwarp();
@@ -176,35 +158,37 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const int quad = warp & 3;
         const int r = quad * 32 + lane;                       // row of the tile = TMEM lane
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-        const uint32_t p_row = sP + r * 128;
         const uint32_t sw = static_cast<uint32_t>(r & 7);
         float m = -INFINITY, l = 0.0f;
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
-            const int st = j & 1;
-            if (!wait_bounded(bar(kSFull + st), static_cast<uint32_t>(j >> 1) & 1u, abort_flag, p.status, 0xB80u | st)) {
+            // S_j is complete, and with it every earlier MMA: O holds the sum over tiles 0..j-1
+            if (!wait_bounded(bar(kSFull), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, 0xB80u)) {
                 ok = false;
                 break;
             }
             ptx::tc_fence_after_sync();
             uint32_t s[4][32];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(t_lane + kColS + st * 128 + 32 * c, s[c]);
+            for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(t_lane + kColS + 32 * c, s[c]);
             ptx::tmem_ld_wait();
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(kSFree + st));  // the scores are in registers
             const int valid = p.seq_kv - j * kBKV;              // keys of this tile that exist (>= 1)
-            float mx = -INFINITY;
+            if (valid < kBKV) {  // the last tile of a ragged sequence: keys that do not exist score -inf
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (c * 32 + e >= valid) s[c][e] = 0xFF800000u;
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    float v = __uint_as_float(s[c][e]);
-                    if (c * 32 + e >= valid) v = -INFINITY;
-                    s[c][e] = __float_as_uint(v);
-                    mx = fmaxf(mx, v);
+                for (int e = 0; e < 32; e += 2) {
+                    mx0 = fmaxf(mx0, __uint_as_float(s[c][e]));
+                    mx1 = fmaxf(mx1, __uint_as_float(s[c][e + 1]));
                 }
+            const float mx = fmaxf(mx0, mx1);
             const float m_new = fmaxf(m, mx * p.scale_log2);
             const float alpha = ex2(m - m_new);   // 0 on the first tile (m = -inf)
             float sum = 0.0f;
@@ -219,41 +203,26 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 }
             l = fmaf(l, alpha, sum);
             m = m_new;
-            if (j > 0) {
-                // the previous P.V has completed: P's buffer is free and O may be rescaled
-                if (!wait_bounded(bar(kPvDone), static_cast<uint32_t>(j - 1) & 1u, abort_flag, p.status, 0xB90u)) {
-                    ok = false;
-                    break;
-                }
-                ptx::tc_fence_after_sync();
-                if (__any_sync(0xFFFFFFFFu, alpha != 1.0f)) {
+            if (j > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.0f)) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
-                        ptx::tmem_ld_32x32(t_lane + kColO + 32 * c, o);
-                        ptx::tmem_ld_wait();
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    ptx::tmem_ld_32x32(t_lane + kColO + 32 * c, o);
+                    ptx::tmem_ld_wait();
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        ptx::tmem_st_32x32(t_lane + kColO + 32 * c, o);
-                    }
-                    ptx::tc_wait_st();
+                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                    ptx::tmem_st_32x32(t_lane + kColO + 32 * c, o);
                 }
             }
-            // P row: 128 BF16 = 16 chunks of 16 bytes; chunk ch lives in box ch / 8 at position (ch % 8) ^ (row % 8)
+            // P row: keys 2c and 2c+1 in column c, over the row's own scores (all of them are in registers)
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int ch = c * 4 + q;
-                    const uint32_t addr = p_row + (ch >> 3) * kBox + ((static_cast<uint32_t>(ch & 7) ^ sw) << 4);
-                    sts128(addr, s[c][4 * q], s[c][4 * q + 1], s[c][4 * q + 2], s[c][4 * q + 3]);
-                }
-            ptx::fence_proxy_async_smem();
+            for (int c = 0; c < 4; ++c) ptx::tmem_st_32x16(t_lane + kColS + 16 * c, s[c]);
+            ptx::tc_wait_st();
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar(kPFull));
         }
-        if (ok && wait_bounded(bar(kPvDone), static_cast<uint32_t>(n_tiles - 1) & 1u, abort_flag, p.status, 0xBA0u)) {
+        if (ok && wait_bounded(bar(kPvDone), 0, abort_flag, p.status, 0xBA0u)) {
             ptx::tc_fence_after_sync();
             const float inv = 1.0f / l;
             const uint32_t o_row = sQ + r * 128;  // Q is no longer read: every MMA has completed
