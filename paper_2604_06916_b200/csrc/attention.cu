@@ -33,10 +33,18 @@ constexpr int kBKV = 128;               // keys per tile
 constexpr int kBox = 128 * 128;         // bytes of a [128 rows][64 BF16] box
 constexpr int kTile = 2 * kBox;         // a [128][128] BF16 tile: box of columns 0..63, box of 64..127
 constexpr int kThreads = 192;
+constexpr float kLazyLog2 = 8.0f;        // slack of the softmax reference maximum, in powers of two
 constexpr int kSmem = 3 * kTile + 256;
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kColS = 0, kColO = 128;   // P overwrites columns [0, 64) of S
 static_assert(2 * (kSmem + 1024) <= 233472, "two CTAs per SM");
+
+#ifdef SOL_TUNING
+__device__ long long g_attn_trace[12][64];
+#define ATTN_TRACE(type, idx) do { if ((blockIdx.x | blockIdx.y | blockIdx.z) == 0 && (idx) < 64 && (threadIdx.x & 31) == 0) g_attn_trace[type][idx] = clock64(); } while (0)
+#else
+#define ATTN_TRACE(type, idx) do { } while (0)
+#endif
 
 struct Params {
     int seq_kv;
@@ -110,10 +118,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             for (int j = 0; j < n_tiles; ++j) {
                 const uint32_t par = static_cast<uint32_t>(j) & 1u;
                 if (!wait_bounded(bar(kKEmpty), par ^ 1u, abort_flag, p.status, 0xB10u)) break;
+                ATTN_TRACE(10, j);
                 ptx::mbar_arrive_expect_tx(bar(kKFull), kTile);
                 ptx::tma_load_3d(sK, &tm_k, x0, j * kBKV, batch, bar(kKFull));
                 ptx::tma_load_3d(sK + kBox, &tm_k, x0 + 64, j * kBKV, batch, bar(kKFull));
                 if (!wait_bounded(bar(kVEmpty), par ^ 1u, abort_flag, p.status, 0xB20u)) break;
+                ATTN_TRACE(11, j);
                 ptx::mbar_arrive_expect_tx(bar(kVFull), kTile);
                 ptx::tma_load_3d(sV, &tm_v, x0, j * kBKV, batch, bar(kVFull));
                 ptx::tma_load_3d(sV + kBox, &tm_v, x0 + 64, j * kBKV, batch, bar(kVFull));
@@ -132,6 +142,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 const uint32_t par = static_cast<uint32_t>(j) & 1u;
                 if (!wait_bounded(bar(kKFull), par, abort_flag, p.status, 0xB40u)) break;
                 ptx::tc_fence_after_sync();
+                ATTN_TRACE(0, j);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {  // 16 elements of d per instruction
                     const uint64_t a = ptx::smem_desc_sw128(sQ + (i >> 2) * kBox) + 2u * (i & 3);
@@ -140,15 +151,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 }
                 ptx::tc_commit(bar(kSFull));   // also: the previous tile's P.V has completed
                 ptx::tc_commit(bar(kKEmpty));
+                ATTN_TRACE(1, j);
                 if (!wait_bounded(bar(kPFull), par, abort_flag, p.status, 0xB60u)) break;
                 if (!wait_bounded(bar(kVFull), par, abort_flag, p.status, 0xB70u)) break;
                 ptx::tc_fence_after_sync();
+                ATTN_TRACE(2, j);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {  // 16 keys per instruction: 8 columns of packed P
                     const uint64_t b = ptx::smem_desc_sw128_mn(sV + i * 2048, kBox, 1024);
                     ptx::mma_bf16_a_tmem(tmem_base + kColO, tmem_base + kColS + 8 * i, b, idesc_pv, (j | i) != 0);
                 }
                 ptx::tc_commit(bar(kVEmpty));
+                ATTN_TRACE(3, j);
                 if (j + 1 == n_tiles) ptx::tc_commit(bar(kPvDone));
             }
         }
@@ -168,10 +182,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 break;
             }
             ptx::tc_fence_after_sync();
+            if (warp == 2) ATTN_TRACE(4, j);
             uint32_t s[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(t_lane + kColS + 32 * c, s[c]);
             ptx::tmem_ld_wait();
+            if (warp == 2) ATTN_TRACE(5, j);
             const int valid = p.seq_kv - j * kBKV;              // keys of this tile that exist (>= 1)
             if (valid < kBKV) {  // the last tile of a ragged sequence: keys that do not exist score -inf
 #pragma unroll
@@ -180,17 +196,26 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     for (int e = 0; e < 32; ++e)
                         if (c * 32 + e >= valid) s[c][e] = 0xFF800000u;
             }
-            float mx0 = -INFINITY, mx1 = -INFINITY;
+            float mx8[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) mx8[e] = __uint_as_float(s[0][e]);
 #pragma unroll
             for (int c = 0; c < 4; ++c)
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    mx0 = fmaxf(mx0, __uint_as_float(s[c][e]));
-                    mx1 = fmaxf(mx1, __uint_as_float(s[c][e + 1]));
-                }
-            const float mx = fmaxf(mx0, mx1);
-            const float m_new = fmaxf(m, mx * p.scale_log2);
-            const float alpha = ex2(m - m_new);   // 0 on the first tile (m = -inf)
+                for (int e = 0; e < 32; e += 8)
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        if (c + e > 0) mx8[k] = fmaxf(mx8[k], __uint_as_float(s[c][e + k]));
+            const float mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+                                   fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+            // The reference maximum m only follows the row maximum when that has grown by more than 2^8:
+            // until then the probabilities are up to 256 times larger (exact in FP32 and BF16 alike, l carries
+            // the same factor) and O, which lives in TMEM, does not have to be rescaled.
+            const float m_tile = mx * p.scale_log2;
+            const bool move = m_tile > m + kLazyLog2;
+            const float m_new = move ? m_tile : m;
+            const float alpha = move ? ex2(m - m_new) : 1.0f;   // 0 on the first tile (m = -inf)
+            if (warp == 2) ATTN_TRACE(6, j);
             float sum = 0.0f;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
@@ -203,7 +228,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 }
             l = fmaf(l, alpha, sum);
             m = m_new;
-            if (j > 0 && __any_sync(0xFFFFFFFFu, alpha != 1.0f)) {
+            if (warp == 2) ATTN_TRACE(7, j);
+            if (j > 0 && __any_sync(0xFFFFFFFFu, move)) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t o[32];
@@ -214,6 +240,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     ptx::tmem_st_32x32(t_lane + kColO + 32 * c, o);
                 }
             }
+            if (warp == 2) ATTN_TRACE(8, j);
             // P row: keys 2c and 2c+1 in column c, over the row's own scores (all of them are in registers)
 #pragma unroll
             for (int c = 0; c < 4; ++c) ptx::tmem_st_32x16(t_lane + kColS + 16 * c, s[c]);
@@ -221,6 +248,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(bar(kPFull));
+            if (warp == 2) ATTN_TRACE(9, j);
         }
         if (ok && wait_bounded(bar(kPvDone), 0, abort_flag, p.status, 0xBA0u)) {
             ptx::tc_fence_after_sync();
@@ -295,3 +323,9 @@ sol_status_t launch_attention(const void *q, const void *k, const void *v, void 
 
 }  // namespace attn
 }  // namespace sol
+
+#ifdef SOL_TUNING
+extern "C" int sol_debug_attention_trace(long long *host_out) {
+    return cudaMemcpyFromSymbol(host_out, sol::attn::g_attn_trace, sizeof(sol::attn::g_attn_trace)) == cudaSuccess ? 0 : 1;
+}
+#endif
