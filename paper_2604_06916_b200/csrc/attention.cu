@@ -3,21 +3,23 @@
 // The linear layers around it run in NVFP4; attention itself stays in BF16 in both the FP4 and the
 // BF16 path of the method, so this kernel is what a whole-block forward needs besides the linears.
 //
-// One CTA per 128 query rows of one (batch, head), two CTAs per SM.  Per 128-key tile j:
-//     S_j = Q K_j^T            tcgen05.mma kind::f16, 128 x 128 x 128, accumulator in TMEM
+// One CTA per 256 query rows of one (batch, head), one CTA per SM: two query tiles of 128 rows, each
+// with its own softmax warpgroup, share the K and V tiles, which stream through two-stage rings (a
+// tile is requested more than a whole tile period before it is used: loads take ~2 500 cycles here).
+// Per 128-key tile j and query tile t:
+//     S_t = Q_t K_j^T          tcgen05.mma kind::f16, 128 x 128 x 128, accumulator in TMEM
 //     softmax                  one thread per query row (= TMEM lane): tcgen05.ld of the row, running
 //                              max m and sum l (online softmax), p = exp2(s c - m); P goes back into
 //                              the columns S occupied, as packed BF16 pairs (tcgen05.st)
-//     O  = alpha O + P V_j     O rescaled in TMEM by the row's alpha when its max moved (tcgen05.ld /
+//     O_t = alpha O_t + P V_j  O rescaled in TMEM by the row's alpha when its max moved (tcgen05.ld /
 //                              st), then tcgen05.mma with A = P from TMEM and V as an MN-major
 //                              shared-memory operand (V is [kv][d])
-// Inside a CTA the three steps of a tile run one after the other; the SM's second CTA fills the
-// tensor pipe while this one is in its softmax, and the other way round: 96 KB of shared memory
-// (Q, one K tile, one V tile) and 256 TMEM columns (S/P and O) per CTA make room for two.
-// The epilogue divides by l and leaves through TMA stores (staged where Q was).
+// The MMA thread alternates between the two query tiles (P_0 V, next S_0, P_1 V, next S_1), so the
+// tensor pipe works for one tile while the other is in its softmax.  TMEM: S_t/P_t and O_t, 128
+// columns each.  The epilogue divides by l and leaves through TMA stores (staged where Q_t was).
 //
-// Warps: 0 = TMA producer, 1 = TMEM owner and MMA issuer, 2..5 = softmax / epilogue (one per TMEM
-// lane quadrant).  Every mbarrier wait is bounded.
+// Warps: 0 = TMA producer, 1 = TMEM owner and MMA issuer, 2..5 and 6..9 = softmax / epilogue of query
+// tile 0 and 1 (one warp per TMEM lane quadrant).  Every mbarrier wait is bounded.
 #include "gemm_common.cuh"
 #include "sol_internal.h"
 
@@ -28,16 +30,18 @@ namespace {
 using gemm::wait_bounded;
 
 constexpr int kD = 128;                 // head dimension
-constexpr int kBQ = 128;                // query rows per CTA
+constexpr int kBQ = 128;                // query rows per query tile
+constexpr int kQTiles = 2;              // query tiles per CTA
 constexpr int kBKV = 128;               // keys per tile
 constexpr int kBox = 128 * 128;         // bytes of a [128 rows][64 BF16] box
 constexpr int kTile = 2 * kBox;         // a [128][128] BF16 tile: box of columns 0..63, box of 64..127
-constexpr int kThreads = 192;
-constexpr float kLazyLog2 = 8.0f;        // slack of the softmax reference maximum, in powers of two
-constexpr int kSmem = 3 * kTile + 256;
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColO = 128;   // P overwrites columns [0, 64) of S
-static_assert(2 * (kSmem + 1024) <= 233472, "two CTAs per SM");
+constexpr int kStages = 2;              // K ring and V ring
+constexpr int kThreads = 32 * (2 + 4 * kQTiles);
+constexpr float kLazyLog2 = 8.0f;       // slack of the softmax reference maximum, in powers of two
+constexpr int kSmem = (kQTiles + 2 * kStages) * kTile + 256;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 128, kColTile = 256;   // per query tile; P overwrites columns [0, 64) of S
+static_assert(kSmem <= 232448, "shared memory budget");
 
 #ifdef SOL_TUNING
 __device__ long long g_attn_trace[12][64];
@@ -47,6 +51,7 @@ __device__ long long g_attn_trace[12][64];
 #endif
 
 struct Params {
+    int seq_q;
     int seq_kv;
     float scale_log2;      // log2(e) / sqrt(d)
     uint32_t *status;
@@ -66,7 +71,7 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const Params p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -75,23 +80,24 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (threadIdx.x == 0) atomicExch(p.status, 0xB00u);
         return;
     }
-    const uint32_t sQ = smem_base;                        // Q, later the output staging buffer
-    const uint32_t sK = smem_base + kTile;
-    const uint32_t sV = sK + kTile;
-    const uint32_t bar_base = sV + kTile;
+    const uint32_t sQ = smem_base;                        // kQTiles tiles; later the output staging buffers
+    const uint32_t sK = sQ + kQTiles * kTile;             // kStages tiles
+    const uint32_t sV = sK + kStages * kTile;
+    const uint32_t bar_base = sV + kStages * kTile;
     uint8_t *bar_gen = smem_raw + (bar_base - smem_base);
     auto bar = [&](int i) { return bar_base + 8u * i; };
-    constexpr int kQFull = 0, kKFull = 1, kKEmpty = 2, kVFull = 3, kVEmpty = 4, kSFull = 5, kPFull = 6, kPvDone = 7,
-                  kNumBars = 8;
+    // K / V rings: [stage]; S, P, PV-done: [query tile]
+    constexpr int kQFull = 0, kKFull = 1, kKEmpty = 3, kVFull = 5, kVEmpty = 7, kSFull = 9, kPFull = 11, kPvDone = 13,
+                  kNumBars = 15;
     uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * kNumBars);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * kNumBars + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int q0 = blockIdx.x * kBQ, head = blockIdx.y, batch = blockIdx.z;
+    const int q0 = blockIdx.x * (kQTiles * kBQ), head = blockIdx.y, batch = blockIdx.z;
     const int n_tiles = (p.seq_kv + kBKV - 1) / kBKV;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kNumBars; ++i) ptx::mbar_init(bar(i), i == kPFull ? 4 : 1);
+        for (int i = 0; i < kNumBars; ++i) ptx::mbar_init(bar(i), (i == kPFull || i == kPFull + 1) ? 4 : 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tm_q);
@@ -112,21 +118,25 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // ------------------------------------------------------------ TMA producer
         if (ptx::elect_one()) {
             const int x0 = head * kD;
-            ptx::mbar_arrive_expect_tx(bar(kQFull), kTile);
-            ptx::tma_load_3d(sQ, &tm_q, x0, q0, batch, bar(kQFull));
-            ptx::tma_load_3d(sQ + kBox, &tm_q, x0 + 64, q0, batch, bar(kQFull));
+            ptx::mbar_arrive_expect_tx(bar(kQFull), kQTiles * kTile);
+#pragma unroll
+            for (int t = 0; t < kQTiles; ++t) {
+                ptx::tma_load_3d(sQ + t * kTile, &tm_q, x0, q0 + t * kBQ, batch, bar(kQFull));
+                ptx::tma_load_3d(sQ + t * kTile + kBox, &tm_q, x0 + 64, q0 + t * kBQ, batch, bar(kQFull));
+            }
             for (int j = 0; j < n_tiles; ++j) {
-                const uint32_t par = static_cast<uint32_t>(j) & 1u;
-                if (!wait_bounded(bar(kKEmpty), par ^ 1u, abort_flag, p.status, 0xB10u)) break;
+                const int st = j & 1;
+                const uint32_t par = static_cast<uint32_t>(j >> 1) & 1u;
+                if (!wait_bounded(bar(kKEmpty + st), par ^ 1u, abort_flag, p.status, 0xB10u | st)) break;
                 ATTN_TRACE(10, j);
-                ptx::mbar_arrive_expect_tx(bar(kKFull), kTile);
-                ptx::tma_load_3d(sK, &tm_k, x0, j * kBKV, batch, bar(kKFull));
-                ptx::tma_load_3d(sK + kBox, &tm_k, x0 + 64, j * kBKV, batch, bar(kKFull));
-                if (!wait_bounded(bar(kVEmpty), par ^ 1u, abort_flag, p.status, 0xB20u)) break;
+                ptx::mbar_arrive_expect_tx(bar(kKFull + st), kTile);
+                ptx::tma_load_3d(sK + st * kTile, &tm_k, x0, j * kBKV, batch, bar(kKFull + st));
+                ptx::tma_load_3d(sK + st * kTile + kBox, &tm_k, x0 + 64, j * kBKV, batch, bar(kKFull + st));
+                if (!wait_bounded(bar(kVEmpty + st), par ^ 1u, abort_flag, p.status, 0xB20u | st)) break;
                 ATTN_TRACE(11, j);
-                ptx::mbar_arrive_expect_tx(bar(kVFull), kTile);
-                ptx::tma_load_3d(sV, &tm_v, x0, j * kBKV, batch, bar(kVFull));
-                ptx::tma_load_3d(sV + kBox, &tm_v, x0 + 64, j * kBKV, batch, bar(kVFull));
+                ptx::mbar_arrive_expect_tx(bar(kVFull + st), kTile);
+                ptx::tma_load_3d(sV + st * kTile, &tm_v, x0, j * kBKV, batch, bar(kVFull + st));
+                ptx::tma_load_3d(sV + st * kTile + kBox, &tm_v, x0 + 64, j * kBKV, batch, bar(kVFull + st));
             }
         }
         __syncwarp();
@@ -137,57 +147,90 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(128 >> 3) << 17) |
                                       (static_cast<uint32_t>(128 >> 4) << 24);
             const uint32_t idesc_pv = idesc_qk | (1u << 16);
-            bool ok = wait_bounded(bar(kQFull), 0, abort_flag, p.status, 0xB30u);
-            for (int j = 0; ok && j < n_tiles; ++j) {
-                const uint32_t par = static_cast<uint32_t>(j) & 1u;
-                if (!wait_bounded(bar(kKFull), par, abort_flag, p.status, 0xB40u)) break;
-                ptx::tc_fence_after_sync();
-                ATTN_TRACE(0, j);
+            auto issue_qk = [&](int t, int st) {  // S_t = Q_t K^T, 16 elements of d per instruction
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {  // 16 elements of d per instruction
-                    const uint64_t a = ptx::smem_desc_sw128(sQ + (i >> 2) * kBox) + 2u * (i & 3);
-                    const uint64_t b = ptx::smem_desc_sw128(sK + (i >> 2) * kBox) + 2u * (i & 3);
-                    ptx::mma_bf16(tmem_base + kColS, a, b, idesc_qk, i > 0);
+                for (int i = 0; i < 8; ++i) {
+                    const uint64_t a = ptx::smem_desc_sw128(sQ + t * kTile + (i >> 2) * kBox) + 2u * (i & 3);
+                    const uint64_t b = ptx::smem_desc_sw128(sK + st * kTile + (i >> 2) * kBox) + 2u * (i & 3);
+                    ptx::mma_bf16(tmem_base + t * kColTile + kColS, a, b, idesc_qk, i > 0);
                 }
-                ptx::tc_commit(bar(kSFull));   // also: the previous tile's P.V has completed
+                ptx::tc_commit(bar(kSFull + t));   // also: every earlier MMA of this tile has completed
+            };
+            auto issue_pv = [&](int t, int st, bool acc) {  // O_t += P_t V, 16 keys (8 columns of packed P) per instruction
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint64_t b = ptx::smem_desc_sw128_mn(sV + st * kTile + i * 2048, kBox, 1024);
+                    ptx::mma_bf16_a_tmem(tmem_base + t * kColTile + kColO, tmem_base + t * kColTile + kColS + 8 * i, b,
+                                         idesc_pv, acc || i > 0);
+                }
+            };
+            bool ok = wait_bounded(bar(kQFull), 0, abort_flag, p.status, 0xB30u) &&
+                      wait_bounded(bar(kKFull), 0, abort_flag, p.status, 0xB31u);
+            if (ok) {
+                ptx::tc_fence_after_sync();
+                issue_qk(0, 0);
+                issue_qk(1, 0);
                 ptx::tc_commit(bar(kKEmpty));
-                ATTN_TRACE(1, j);
+            }
+            for (int j = 0; ok && j < n_tiles; ++j) {
+                const int st = j & 1, nst = st ^ 1;
+                const uint32_t par = static_cast<uint32_t>(j) & 1u;            // per-tile barriers flip every tile
+                const uint32_t ring = static_cast<uint32_t>(j >> 1) & 1u;      // ring barriers every second tile
+                const bool more = j + 1 < n_tiles;
+                // query tile 0: P_0 V_j, then the next scores
                 if (!wait_bounded(bar(kPFull), par, abort_flag, p.status, 0xB60u)) break;
-                if (!wait_bounded(bar(kVFull), par, abort_flag, p.status, 0xB70u)) break;
+                if (!wait_bounded(bar(kVFull + st), ring, abort_flag, p.status, 0xB70u | st)) break;
                 ptx::tc_fence_after_sync();
                 ATTN_TRACE(2, j);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {  // 16 keys per instruction: 8 columns of packed P
-                    const uint64_t b = ptx::smem_desc_sw128_mn(sV + i * 2048, kBox, 1024);
-                    ptx::mma_bf16_a_tmem(tmem_base + kColO, tmem_base + kColS + 8 * i, b, idesc_pv, (j | i) != 0);
+                issue_pv(0, st, j > 0);
+                if (more) {
+                    if (!wait_bounded(bar(kKFull + nst), static_cast<uint32_t>((j + 1) >> 1) & 1u, abort_flag, p.status,
+                                      0xB40u | nst))
+                        break;
+                    ptx::tc_fence_after_sync();
+                    ATTN_TRACE(0, j + 1);
+                    issue_qk(0, nst);
+                } else {
+                    ptx::tc_commit(bar(kPvDone));
                 }
-                ptx::tc_commit(bar(kVEmpty));
+                // query tile 1
+                if (!wait_bounded(bar(kPFull + 1), par, abort_flag, p.status, 0xB61u)) break;
+                ptx::tc_fence_after_sync();
+                issue_pv(1, st, j > 0);
+                ptx::tc_commit(bar(kVEmpty + st));
+                if (more) {
+                    issue_qk(1, nst);
+                    ptx::tc_commit(bar(kKEmpty + nst));
+                } else {
+                    ptx::tc_commit(bar(kPvDone + 1));
+                }
                 ATTN_TRACE(3, j);
-                if (j + 1 == n_tiles) ptx::tc_commit(bar(kPvDone));
             }
         }
         __syncwarp();
     } else {
         // ------------------------------------------------------------ softmax and epilogue: thread = query row
+        const int t = (warp - 2) >> 2;                        // query tile of this warpgroup
         const int quad = warp & 3;
         const int r = quad * 32 + lane;                       // row of the tile = TMEM lane
-        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        const uint32_t t_lane = tmem_base + t * kColTile + (static_cast<uint32_t>(quad * 32) << 16);
         const uint32_t sw = static_cast<uint32_t>(r & 7);
+        const bool tracer = warp == 2;
         float m = -INFINITY, l = 0.0f;
         bool ok = true;
         for (int j = 0; j < n_tiles; ++j) {
-            // S_j is complete, and with it every earlier MMA: O holds the sum over tiles 0..j-1
-            if (!wait_bounded(bar(kSFull), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, 0xB80u)) {
+            // S_j is complete, and with it every earlier MMA of this tile: O holds the sum over tiles 0..j-1
+            if (!wait_bounded(bar(kSFull + t), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, 0xB80u | t)) {
                 ok = false;
                 break;
             }
             ptx::tc_fence_after_sync();
-            if (warp == 2) ATTN_TRACE(4, j);
+            if (tracer) ATTN_TRACE(4, j);
             uint32_t s[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) ptx::tmem_ld_32x32(t_lane + kColS + 32 * c, s[c]);
             ptx::tmem_ld_wait();
-            if (warp == 2) ATTN_TRACE(5, j);
+            if (tracer) ATTN_TRACE(5, j);
             const int valid = p.seq_kv - j * kBKV;              // keys of this tile that exist (>= 1)
             if (valid < kBKV) {  // the last tile of a ragged sequence: keys that do not exist score -inf
 #pragma unroll
@@ -215,7 +258,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const bool move = m_tile > m + kLazyLog2;
             const float m_new = move ? m_tile : m;
             const float alpha = move ? ex2(m - m_new) : 1.0f;   // 0 on the first tile (m = -inf)
-            if (warp == 2) ATTN_TRACE(6, j);
+            if (tracer) ATTN_TRACE(6, j);
             float sum = 0.0f;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
@@ -228,7 +271,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 }
             l = fmaf(l, alpha, sum);
             m = m_new;
-            if (warp == 2) ATTN_TRACE(7, j);
+            if (tracer) ATTN_TRACE(7, j);
             if (j > 0 && __any_sync(0xFFFFFFFFu, move)) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -240,20 +283,20 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     ptx::tmem_st_32x32(t_lane + kColO + 32 * c, o);
                 }
             }
-            if (warp == 2) ATTN_TRACE(8, j);
+            if (tracer) ATTN_TRACE(8, j);
             // P row: keys 2c and 2c+1 in column c, over the row's own scores (all of them are in registers)
 #pragma unroll
             for (int c = 0; c < 4; ++c) ptx::tmem_st_32x16(t_lane + kColS + 16 * c, s[c]);
             ptx::tc_wait_st();
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(bar(kPFull));
-            if (warp == 2) ATTN_TRACE(9, j);
+            if (lane == 0) ptx::mbar_arrive(bar(kPFull + t));
+            if (tracer) ATTN_TRACE(9, j);
         }
-        if (ok && wait_bounded(bar(kPvDone), 0, abort_flag, p.status, 0xBA0u)) {
+        if (ok && wait_bounded(bar(kPvDone + t), 0, abort_flag, p.status, 0xBA0u | t)) {
             ptx::tc_fence_after_sync();
             const float inv = 1.0f / l;
-            const uint32_t o_row = sQ + r * 128;  // Q is no longer read: every MMA has completed
+            const uint32_t o_row = sQ + t * kTile + r * 128;  // Q_t is no longer read: its MMAs have completed
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t o[32];
@@ -271,9 +314,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
             ptx::fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) {  // this warp's 32 rows, two boxes of 64 columns (clipped at the end of the sequence)
-                ptx::tma_store_3d(&tm_o, head * kD, q0 + quad * 32, batch, sQ + quad * 32 * 128);
-                ptx::tma_store_3d(&tm_o, head * kD + 64, q0 + quad * 32, batch, sQ + kBox + quad * 32 * 128);
+            const int row0 = q0 + t * kBQ + quad * 32;
+            if (lane == 0 && row0 < p.seq_q) {  // this warp's 32 rows, two boxes of 64 columns (clipped at the end of the sequence)
+                ptx::tma_store_3d(&tm_o, head * kD, row0, batch, sQ + t * kTile + quad * 32 * 128);
+                ptx::tma_store_3d(&tm_o, head * kD + 64, row0, batch, sQ + t * kTile + kBox + quad * 32 * 128);
                 ptx::tma_store_commit();
                 ptx::tma_store_wait_all<0>();
             }
@@ -304,6 +348,7 @@ sol_status_t launch_attention(const void *q, const void *k, const void *v, void 
         !make(&tm_o, out, seq_q, ld_out, 32))
         return SOL_ERR_CUDA;
     Params p{};
+    p.seq_q = static_cast<int>(seq_q);
     p.seq_kv = static_cast<int>(seq_kv);
     p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(kD));
     p.status = device_status_word();
@@ -315,7 +360,7 @@ sol_status_t launch_attention(const void *q, const void *k, const void *v, void 
             return SOL_ERR_CUDA;
         configured[dev] = true;
     }
-    const dim3 grid(static_cast<unsigned>((seq_q + kBQ - 1) / kBQ), static_cast<unsigned>(heads),
+    const dim3 grid(static_cast<unsigned>((seq_q + kQTiles * kBQ - 1) / (kQTiles * kBQ)), static_cast<unsigned>(heads),
                     static_cast<unsigned>(batch));
     attention_kernel<<<grid, kThreads, kSmem, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
     return launch_status();
