@@ -127,6 +127,27 @@ def calibrated_rows(cfg, layer_index: int, target_s: float, fixed: int) -> int:
     return max(256, min(cfg.layers[layer_index].M, (rows // 128) * 128))
 
 
+def attention_numbers(B, n_s, seq, heads, loop_ms, peaks, peak_src):
+    """Ours against torch's scaled-dot-product attention on one fused q/k/v projection output."""
+    import torch
+    import torch.nn.functional as F
+    from paper_2604_06916_b200 import workloads
+    _, q, k, v = workloads.make_qkv(n_s, seq, heads, 3, "cuda")
+    out = torch.empty((n_s, seq, heads, 128), dtype=torch.bfloat16, device="cuda")
+    t_ours = loop_ms(lambda: B.sol_attention_bf16(q, k, v, out=out))
+    qt, kt, vt = q.transpose(1, 2), k.transpose(1, 2), v.transpose(1, 2)
+    t_lib = loop_ms(lambda: F.scaled_dot_product_attention(qt, kt, vt))
+    fl = 4.0 * n_s * heads * seq * seq * 128
+    tf = fl / (t_ours * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"]
+    return {"shape": {"samples": n_s, "tokens": seq, "heads": heads, "head_dim": 128}, "ms": t_ours, "tflops": tf,
+            "torch_sdpa_ms": t_lib, "torch_sdpa_tflops": fl / (t_lib * 1e-3) / 1e12,
+            "roofline": {"bound": "tensor", "kernel": "attention_kernel", "achieved": tf, "peak": peak, "unit": "TFLOP/s",
+                         "frac": tf / peak, "traffic": None,
+                         "peak_source": peak_src + " (bf16 burst); the softmax's 2 x 16 K exponentials per tile on the SFU "
+                                                   "(16 per clock per SM) take as long as the tile's MMAs"}}
+
+
 def run_reference(args):
     from paper_2604_06916_b200 import workloads
 
@@ -497,6 +518,13 @@ def run_ours(args):
                                  "traffic": None, "peak_source": peak_src}}
         del lq, sc, sh
 
+    # ---- BF16 attention of the same block geometry (samples x tokens x hidden / 128 heads), ours and torch's
+    attention = None
+    if world == 1 and not args.lean and cfg.name.startswith("flux1_12b_g"):
+        l0 = cfg.layers[0]
+        rps = workloads.SWEEP_TOKENS if l0.M % workloads.SWEEP_TOKENS == 0 else l0.M
+        attention = attention_numbers(B, l0.M // rps, rps, l0.K // 128, loop_ms, peaks, peak_src)
+
     # ---- stage-1 selection and rank metrics at the paper's sizes (48 prompts per epoch, N = 96, K = 24):
     # two launches of one block per prompt, a few microseconds each (launch latency, not throughput)
     selection = None
@@ -599,7 +627,7 @@ def run_ours(args):
                                "peak_source": peak_src},
         "stack_tflops_delayed_scale": world * flops / (ms_static / args.steps * 1e-3) / 1e12,
         "mxfp4_stack_tflops": world * flops / (ms_mx / args.steps * 1e-3) / 1e12,
-        "weight_refresh": refresh, "mlp_pair_nvfp4_intermediate": mlp_pair, "single_stream_pair_nvfp4_intermediate": single_pair, "layernorm_quantize": ln_quant, "stage1_selection": selection,
+        "weight_refresh": refresh, "mlp_pair_nvfp4_intermediate": mlp_pair, "single_stream_pair_nvfp4_intermediate": single_pair, "layernorm_quantize": ln_quant, "attention_bf16": attention, "stage1_selection": selection,
         "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
         "gpu_launches": kernels_per_layer * len(layers) * args.steps,
         "bf16_vs_torch_matmul_note": "MEASURED_PEAKS bf16 (torch.matmul 8192^3): %.0f burst / %.0f sustained TF" % (
@@ -693,7 +721,14 @@ def run_only(args):
         y1 = torch.empty((M, l1.N), dtype=torch.bfloat16, device="cuda")
         y2 = torch.empty((M, H), dtype=torch.bfloat16, device="cuda")
 
+        attn_out = torch.empty((M, H), dtype=torch.bfloat16, device="cuda")
+        use_ours = {"on": True}
+
         def attention(qkv):
+            if use_ours["on"]:  # this library's kernel reads the fused projection in place and writes [M, H]
+                q, k, v = (qkv.view(n_s, rps, -1)[:, :, i * H:(i + 1) * H].unflatten(2, (heads, hd)) for i in range(3))
+                B.sol_attention_bf16(q, k, v, out=attn_out.view(n_s, rps, heads, hd))
+                return attn_out
             q, k, v = qkv.view(n_s, rps, 3, heads, hd).permute(2, 0, 3, 1, 4)
             o = F.scaled_dot_product_attention(q, k, v)
             return o.transpose(1, 2).reshape(M, H)
@@ -723,7 +758,9 @@ def run_only(args):
         state.copy_(amax_in / 2688.0)
         t_cat.copy_(torch.maximum(amax_cat, B.sol_amax_bf16(attention(y_qkv)) * 2688.0) / 2688.0)
         res = {}
-        for name, fn in (("nvfp4", block_fp4), ("bf16", block_bf16)):
+        for name, fn, ours in (("nvfp4", block_fp4, True), ("bf16", block_bf16, True),
+                               ("nvfp4_torch_attention", block_fp4, False), ("bf16_torch_attention", block_bf16, False)):
+            use_ours["on"] = ours
             for _ in range(max(1, args.warmup)):
                 fn()
             torch.cuda.synchronize()
@@ -735,20 +772,51 @@ def run_only(args):
             torch.cuda.synchronize()
             res[name] = e0.elapsed_time(e1) / args.steps
             res[name + "_out"] = out
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            attention(y_qkv)
-        e1.record()
-        torch.cuda.synchronize()
-        t_attn = e0.elapsed_time(e1) / args.steps
+        t_attn_by = {}
+        for ours in (True, False):
+            use_ours["on"] = ours
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                attention(y_qkv)
+            e1.record()
+            torch.cuda.synchronize()
+            t_attn_by[ours] = e0.elapsed_time(e1) / args.steps
+        t_attn = t_attn_by[True]
         B.sol_last_device_status()
         diff = (res["nvfp4_out"].float() - res["bf16_out"].float())
         rel = float(diff.pow(2).mean().sqrt() / res["bf16_out"].float().pow(2).mean().sqrt())
         print(json.dumps({"only": "single_block", "M": M, "hidden": H, "nvfp4_ms": res["nvfp4"], "bf16_ms": res["bf16"],
                           "speedup": res["bf16"] / res["nvfp4"], "attention_ms_in_both": t_attn,
+                          "attention": "sol_attention_bf16 (this library)",
+                          "with_torch_attention": {"nvfp4_ms": res["nvfp4_torch_attention"], "bf16_ms": res["bf16_torch_attention"],
+                                                   "speedup": res["bf16_torch_attention"] / res["nvfp4_torch_attention"],
+                                                   "attention_ms": t_attn_by[False]},
                           "speedup_without_attention": (res["bf16"] - t_attn) / (res["nvfp4"] - t_attn),
                           "rel_rms_difference_of_outputs": rel}))
+        return
+    if args.only == "attention":
+        cfg = workloads.CONFIGS[args.workload]
+        l0 = cfg.layers[0]
+        rps = workloads.SWEEP_TOKENS if l0.M % workloads.SWEEP_TOKENS == 0 else l0.M
+        n_s = args.rows // rps if args.rows > 0 else l0.M // rps
+        peaks, peak_src = load_peaks()
+
+        def loop_ms(fn):
+            for _ in range(max(1, args.warmup)):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / args.steps
+
+        res = attention_numbers(B, max(1, n_s), rps, l0.K // 128, loop_ms, peaks, peak_src)
+        B.sol_last_device_status()
+        print(json.dumps({"only": "attention", **res}))
         return
     if args.only == "layernorm_quantize":
         cfg = workloads.CONFIGS[args.workload]
@@ -829,7 +897,7 @@ def run_only(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair' / 'mxfp4:<layer>' / 'layernorm_quantize' / 'single_block'")
+    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair' / 'mxfp4:<layer>' / 'layernorm_quantize' / 'single_block' / 'attention'")
     ap.add_argument("--rows", type=int, default=0, help="profile mode: override M")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
