@@ -24,6 +24,8 @@
  *     row pitches multiples of 8 elements.  Inputs must be finite.
  *   - Only sm_100 devices are supported (SOL_ERR_UNSUPPORTED_ARCH otherwise); there is
  *     no CPU path.
+ *   - A launch the CUDA runtime rejects returns SOL_ERR_CUDA; with the environment variable
+ *     SOL_NVFP4_VERBOSE set, the runtime's error string is also printed to stderr.
  *
  * NVFP4 storage
  *   data   : uint8 [rows, K/2]; byte j of a row holds element 2j in its low nibble and

@@ -1,5 +1,7 @@
 // Host-side helpers shared by the entry points: argument checks, device query, launch checks.
 #pragma once
+#include <cstdio>
+#include <cstdlib>
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -26,7 +28,10 @@ const DeviceInfo *current_device_info();
 sol_status_t check_arch(const DeviceInfo **info_out);
 
 inline sol_status_t launch_status() {
-    return cudaGetLastError() == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess && getenv("SOL_NVFP4_VERBOSE") != nullptr)
+        fprintf(stderr, "sol_nvfp4: launch failed: %s\n", cudaGetErrorString(e));
+    return e == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
 }
 
 // Device status word written by bounded waits (0 = fine).
