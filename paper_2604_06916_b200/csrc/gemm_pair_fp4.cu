@@ -474,6 +474,9 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                             ptx::tc_store_32x32b_x4(sf_t + 20 + 8 * c, v[2 * kSfChunksK + c]);
                         }
                         ptx::tc_wait_st();
+                        // the stage's next contents arrive through the async proxy: order these generic-proxy
+                        // reads of the scale tiles before it (the release chain to the producer starts here)
+                        ptx::fence_proxy_async_smem();
                         ptx::tc_fence_before_sync();
                         __syncwarp();
                         if (elected) ptx::mbar_arrive_cluster(ready0 + 8u * sf_buf);
