@@ -254,6 +254,25 @@ sol_status_t sol_attention_bf16(const void *q, const void *k, const void *v, voi
                                 void *stream);
 
 /*
+ * The same attention over two token streams that are projected separately and attend jointly, as in
+ * the double-stream blocks of the FLUX.1 model of Section 4.1 (text tokens and image tokens): the
+ * joint sequence is the first stream's tokens followed by the second's; queries, keys and values
+ * are read from, and outputs written to, each stream's own tensors -- no concatenated copy exists.
+ *   first, second   host pointers to the two descriptions below (read during the call only);
+ *                   q, k, v, out: device pointers laid out as in sol_attention_bf16, `seq` tokens each
+ *   first->seq % 256 == 0 (the first stream fills whole query-tile pairs); second->seq is free
+ * Errors as for sol_attention_bf16, plus SOL_ERR_BAD_SHAPE for a first stream that is not a multiple
+ * of 256 tokens.
+ */
+typedef struct {
+    const void *q, *k, *v;
+    void *out;
+    int64_t seq, ld_q, ld_k, ld_v, ld_out;
+} sol_attention_stream_t;
+sol_status_t sol_attention_bf16_joint(const sol_attention_stream_t *first, const sol_attention_stream_t *second,
+                                      int64_t batch, int64_t heads, void *stream);
+
+/*
  * BF16 linear, the full-precision stage-2 reference (Section 3.4):
  *     Y[m,n] = bf16_rne( sum_k x[m,k] * w[n,k] + bias[n] ),  FP32 accumulate.
  */

@@ -36,6 +36,15 @@ def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray, rows=None) -> np.ndar
     return out
 
 
+def attention_joint(first, second):
+    """Two token streams that attend jointly (first stream's tokens, then the second's): (q, k, v) each
+    [B, S_i, H, d].  The plain definition on the concatenated sequence, split back per stream."""
+    q, k, v = (np.concatenate((a, b), axis=1) for a, b in zip(first, second))
+    out = attention(q, k, v)
+    n = first[0].shape[1]
+    return out[:, :n], out[:, n:]
+
+
 def attention_tolerance(ref: np.ndarray, v: np.ndarray) -> np.ndarray:
     """Bound for a kernel that rounds the probabilities and the output to BF16 and sums in FP32.
 

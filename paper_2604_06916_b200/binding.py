@@ -25,7 +25,7 @@ EXPORTS = [
     "nvfp4_requantize_lora", "nvfp4_requantize_lora_batch", "nvfp4_linear_quantized_out",
     "solrl_select_contrastive", "solrl_rank_consistency", "sol_mxfp4_scale_bytes", "mxfp4_quantize",
     "mxfp4_linear", "nvfp4_linear_split_out", "nvfp4_quantize_into",
-    "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale", "nvfp4_layernorm_quantize", "sol_attention_bf16",
+    "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale", "nvfp4_layernorm_quantize", "sol_attention_bf16", "sol_attention_bf16_joint",
 ]
 
 _lib = None
@@ -91,6 +91,8 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_quantize_linear_delayed.restype = i32
     L.nvfp4_quantize_linear_delayed.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, sz, vp]
     L.sol_roll_tensor_scale.restype, L.sol_roll_tensor_scale.argtypes = i32, [vp, vp]
+    L.sol_attention_bf16_joint.restype = i32
+    L.sol_attention_bf16_joint.argtypes = [ctypes.POINTER(AttentionStream), ctypes.POINTER(AttentionStream), i64, i64, vp]
     L.sol_attention_bf16.restype = i32
     L.sol_attention_bf16.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, vp]
     L.nvfp4_layernorm_quantize.restype = i32
@@ -319,6 +321,54 @@ def nvfp4_layernorm_quantize(x, scale, shift, rows_per_sample: int, tensor_scale
                                           float(eps), _ptr(tensor_scale), _ptr(q), _ptr(sf), _ptr(amax_out), _stream()),
            "nvfp4_layernorm_quantize")
     return q, sf
+
+
+class AttentionStream(ctypes.Structure):
+    """sol_attention_stream_t of the C header."""
+    _fields_ = [("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("out", ctypes.c_void_p),
+                ("seq", ctypes.c_int64), ("ld_q", ctypes.c_int64), ("ld_k", ctypes.c_int64), ("ld_v", ctypes.c_int64),
+                ("ld_out", ctypes.c_int64)]
+
+
+def _token_pitch(t: torch.Tensor) -> int:
+    """Elements between consecutive tokens of a [B, S, H, 128] view (a dimension of extent 1 has no meaningful stride)."""
+    if t.shape[1] > 1:
+        return t.stride(1)
+    return t.stride(0) if t.shape[0] > 1 else t.shape[2] * 128
+
+
+def _check_attention_view(name: str, t: torch.Tensor):
+    if t.dtype != torch.bfloat16 or t.dim() != 4 or t.shape[3] != 128:
+        raise ValueError(f"{name} must be a [B, S, H, 128] BF16 tensor")
+    if t.stride(3) != 1 or (t.shape[2] > 1 and t.stride(2) != 128) or \
+            (t.shape[0] > 1 and t.shape[1] > 1 and t.stride(0) != t.shape[1] * t.stride(1)):
+        raise ValueError(f"{name}: heads and head dimension must be contiguous, batches stacked densely")
+
+
+def sol_attention_bf16_joint(first, second, out=None):
+    """Joint attention of two token streams: first = (q, k, v) of the stream whose tokens come first.
+
+    Every tensor is a [B, S_stream, H, 128] view as in sol_attention_bf16; S of the first stream is a
+    multiple of 256.  Returns (out_first, out_second), each [B, S_stream, H, 128].
+    """
+    streams = []
+    outs = list(out) if out is not None else [None, None]
+    for i, (q, k, v) in enumerate((first, second)):
+        for name, t in (("q", q), ("k", k), ("v", v)):
+            _check_attention_view(name, t)
+        if q.shape != k.shape or q.shape != v.shape:
+            raise ValueError("q, k and v of a stream must have one shape")
+        if outs[i] is None:
+            outs[i] = torch.empty(tuple(q.shape), dtype=torch.bfloat16, device=q.device)
+        _check_attention_view("out", outs[i])
+        streams.append(AttentionStream(_ptr(q), _ptr(k), _ptr(v), _ptr(outs[i]), q.shape[1], _token_pitch(q),
+                                       _token_pitch(k), _token_pitch(v), _token_pitch(outs[i])))
+    B_, _, H, _ = first[0].shape
+    if second[0].shape[0] != B_ or second[0].shape[2] != H:
+        raise ValueError("both streams must share batch and heads")
+    _check(lib().sol_attention_bf16_joint(ctypes.byref(streams[0]), ctypes.byref(streams[1]), B_, H, _stream()),
+           "sol_attention_bf16_joint")
+    return outs[0], outs[1]
 
 
 def sol_attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor | None = None):

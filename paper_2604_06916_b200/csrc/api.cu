@@ -492,8 +492,33 @@ sol_status_t sol_attention_bf16(const void *q, const void *k, const void *v, voi
     const DeviceInfo *dev = nullptr;
     sol_status_t st = check_arch(&dev);
     if (st != SOL_OK) return st;
-    return attn::launch_attention(q, k, v, out, batch, seq_q, seq_kv, heads, ld_q, ld_k, ld_v, ld_out,
-                                  static_cast<cudaStream_t>(stream));
+    const attn::Stream b{q, k, v, out, seq_q, seq_kv, ld_q, ld_k, ld_v, ld_out};
+    return attn::launch_attention(nullptr, b, batch, heads, static_cast<cudaStream_t>(stream));
+}
+
+sol_status_t sol_attention_bf16_joint(const sol_attention_stream_t *first, const sol_attention_stream_t *second,
+                                      int64_t batch, int64_t heads, void *stream) {
+    if (first == nullptr || second == nullptr) return SOL_ERR_NULL_POINTER;
+    const sol_attention_stream_t *both[2] = {first, second};
+    const int64_t cols = heads * 128;
+    if (batch <= 0 || heads <= 0 || batch > 65535 || heads > 65535) return SOL_ERR_BAD_SHAPE;
+    for (const sol_attention_stream_t *s : both) {
+        if (s->q == nullptr || s->k == nullptr || s->v == nullptr || s->out == nullptr) return SOL_ERR_NULL_POINTER;
+        if (s->seq <= 0 || s->seq > (1LL << 24) || s->ld_q < cols || s->ld_k < cols || s->ld_v < cols || s->ld_out < cols)
+            return SOL_ERR_BAD_SHAPE;
+        if (!aligned16(s->q) || !aligned16(s->k) || !aligned16(s->v) || !aligned16(s->out) || s->ld_q % 8 != 0 ||
+            s->ld_k % 8 != 0 || s->ld_v % 8 != 0 || s->ld_out % 8 != 0)
+            return SOL_ERR_ALIGNMENT;
+    }
+    if (first->seq % 256 != 0) return SOL_ERR_BAD_SHAPE;  // the first stream must fill whole query-tile pairs
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    const attn::Stream a{first->q, first->k, first->v, first->out, first->seq, first->seq,
+                         first->ld_q, first->ld_k, first->ld_v, first->ld_out};
+    const attn::Stream b{second->q, second->k, second->v, second->out, second->seq, second->seq,
+                         second->ld_q, second->ld_k, second->ld_v, second->ld_out};
+    return attn::launch_attention(&a, b, batch, heads, static_cast<cudaStream_t>(stream));
 }
 
 sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,

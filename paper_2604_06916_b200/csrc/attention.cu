@@ -51,8 +51,10 @@ __device__ long long g_attn_trace[12][64];
 #endif
 
 struct Params {
-    int seq_q;
+    int seq_q;             // query rows and keys of the joint sequence (stream a first, then stream b)
     int seq_kv;
+    int q_split;           // rows / keys that come from stream a (0: one stream); multiples of 256 and 128
+    int kv_split;
     float scale_log2;      // log2(e) / sqrt(d)
     uint32_t *status;
 };
@@ -72,8 +74,10 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const Params p) {
+attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ CUtensorMap tm_ka,
+                 const __grid_constant__ CUtensorMap tm_va, const __grid_constant__ CUtensorMap tm_oa,
+                 const __grid_constant__ CUtensorMap tm_qb, const __grid_constant__ CUtensorMap tm_kb,
+                 const __grid_constant__ CUtensorMap tm_vb, const __grid_constant__ CUtensorMap tm_ob, const Params p) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t smem_base = ptx::smem_u32(smem_raw);
     if (smem_base & 1023u) {  // the swizzled operand layout needs 1024-byte alignment
@@ -93,17 +97,23 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * kNumBars + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int q0 = blockIdx.x * (kQTiles * kBQ), head = blockIdx.y, batch = blockIdx.z;
+    const int q0_joint = blockIdx.x * (kQTiles * kBQ), head = blockIdx.y, batch = blockIdx.z;
     const int n_tiles = (p.seq_kv + kBKV - 1) / kBKV;
+    // the CTA's queries come from one stream (the split is a multiple of the CTA's 256 rows)
+    const bool q_in_a = q0_joint < p.q_split;
+    const CUtensorMap *tm_q = q_in_a ? &tm_qa : &tm_qb;
+    const CUtensorMap *tm_o = q_in_a ? &tm_oa : &tm_ob;
+    const int q0 = q_in_a ? q0_joint : q0_joint - p.q_split;                 // row within its stream
+    const int q_rows = q_in_a ? p.q_split : p.seq_q - p.q_split;             // rows of that stream
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kNumBars; ++i) ptx::mbar_init(bar(i), (i == kPFull || i == kPFull + 1) ? 4 : 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
-        ptx::prefetch_tmap(&tm_q);
-        ptx::prefetch_tmap(&tm_k);
-        ptx::prefetch_tmap(&tm_v);
-        ptx::prefetch_tmap(&tm_o);
+        ptx::prefetch_tmap(tm_q);
+        ptx::prefetch_tmap(tm_o);
+        ptx::prefetch_tmap(&tm_kb);
+        ptx::prefetch_tmap(&tm_vb);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(tmem_ptr_smem), kTmemCols);
@@ -121,8 +131,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ptx::mbar_arrive_expect_tx(bar(kQFull), kQTiles * kTile);
 #pragma unroll
             for (int t = 0; t < kQTiles; ++t) {
-                ptx::tma_load_3d(sQ + t * kTile, &tm_q, x0, q0 + t * kBQ, batch, bar(kQFull));
-                ptx::tma_load_3d(sQ + t * kTile + kBox, &tm_q, x0 + 64, q0 + t * kBQ, batch, bar(kQFull));
+                ptx::tma_load_3d(sQ + t * kTile, tm_q, x0, q0 + t * kBQ, batch, bar(kQFull));
+                ptx::tma_load_3d(sQ + t * kTile + kBox, tm_q, x0 + 64, q0 + t * kBQ, batch, bar(kQFull));
             }
             for (int j = 0; j < n_tiles; ++j) {
                 const int st = j & 1;
@@ -130,13 +140,18 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 if (!wait_bounded(bar(kKEmpty + st), par ^ 1u, abort_flag, p.status, 0xB10u | st)) break;
                 ATTN_TRACE(10, j);
                 ptx::mbar_arrive_expect_tx(bar(kKFull + st), kTile);
-                ptx::tma_load_3d(sK + st * kTile, &tm_k, x0, j * kBKV, batch, bar(kKFull + st));
-                ptx::tma_load_3d(sK + st * kTile + kBox, &tm_k, x0 + 64, j * kBKV, batch, bar(kKFull + st));
+                // key tile j of the joint sequence: stream a up to the split (a multiple of the tile), then stream b
+                const bool kv_in_a = j * kBKV < p.kv_split;
+                const int kv0 = kv_in_a ? j * kBKV : j * kBKV - p.kv_split;
+                const CUtensorMap *tm_k = kv_in_a ? &tm_ka : &tm_kb;
+                const CUtensorMap *tm_v = kv_in_a ? &tm_va : &tm_vb;
+                ptx::tma_load_3d(sK + st * kTile, tm_k, x0, kv0, batch, bar(kKFull + st));
+                ptx::tma_load_3d(sK + st * kTile + kBox, tm_k, x0 + 64, kv0, batch, bar(kKFull + st));
                 if (!wait_bounded(bar(kVEmpty + st), par ^ 1u, abort_flag, p.status, 0xB20u | st)) break;
                 ATTN_TRACE(11, j);
                 ptx::mbar_arrive_expect_tx(bar(kVFull + st), kTile);
-                ptx::tma_load_3d(sV + st * kTile, &tm_v, x0, j * kBKV, batch, bar(kVFull + st));
-                ptx::tma_load_3d(sV + st * kTile + kBox, &tm_v, x0 + 64, j * kBKV, batch, bar(kVFull + st));
+                ptx::tma_load_3d(sV + st * kTile, tm_v, x0, kv0, batch, bar(kVFull + st));
+                ptx::tma_load_3d(sV + st * kTile + kBox, tm_v, x0 + 64, kv0, batch, bar(kVFull + st));
             }
         }
         __syncwarp();
@@ -315,9 +330,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             ptx::fence_proxy_async_smem();
             __syncwarp();
             const int row0 = q0 + t * kBQ + quad * 32;
-            if (lane == 0 && row0 < p.seq_q) {  // this warp's 32 rows, two boxes of 64 columns (clipped at the end of the sequence)
-                ptx::tma_store_3d(&tm_o, head * kD, row0, batch, sQ + t * kTile + quad * 32 * 128);
-                ptx::tma_store_3d(&tm_o, head * kD + 64, row0, batch, sQ + t * kTile + kBox + quad * 32 * 128);
+            if (lane == 0 && row0 < q_rows) {  // this warp's 32 rows, two boxes of 64 columns (clipped at the end of the stream)
+                ptx::tma_store_3d(tm_o, head * kD, row0, batch, sQ + t * kTile + quad * 32 * 128);
+                ptx::tma_store_3d(tm_o, head * kD + 64, row0, batch, sQ + t * kTile + kBox + quad * 32 * 128);
                 ptx::tma_store_commit();
                 ptx::tma_store_wait_all<0>();
             }
@@ -335,21 +350,23 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
 }  // namespace
 
-sol_status_t launch_attention(const void *q, const void *k, const void *v, void *out, int64_t batch, int64_t seq_q,
-                              int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v, int64_t ld_out,
-                              cudaStream_t stream) {
-    CUtensorMap tm_q, tm_k, tm_v, tm_o;
+sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, cudaStream_t stream) {
+    CUtensorMap tm[8];
     const uint64_t cols = static_cast<uint64_t>(heads) * kD;
-    auto make = [&](CUtensorMap *tm, const void *base, int64_t seq, int64_t ld, uint32_t box_rows) {
-        return make_tmap_3d_bf16(tm, base, cols, static_cast<uint64_t>(seq), static_cast<uint64_t>(batch),
+    auto make = [&](CUtensorMap *t, const void *base, int64_t seq, int64_t ld, uint32_t box_rows) {
+        return make_tmap_3d_bf16(t, base, cols, static_cast<uint64_t>(seq), static_cast<uint64_t>(batch),
                                  static_cast<uint64_t>(ld) * 2, static_cast<uint64_t>(seq) * ld * 2, 64, box_rows);
     };
-    if (!make(&tm_q, q, seq_q, ld_q, kBQ) || !make(&tm_k, k, seq_kv, ld_k, kBKV) || !make(&tm_v, v, seq_kv, ld_v, kBKV) ||
-        !make(&tm_o, out, seq_q, ld_out, 32))
-        return SOL_ERR_CUDA;
+    auto make4 = [&](CUtensorMap *t, const Stream &s) {
+        return make(t, s.q, s.seq_q, s.ld_q, kBQ) && make(t + 1, s.k, s.seq_kv, s.ld_k, kBKV) &&
+               make(t + 2, s.v, s.seq_kv, s.ld_v, kBKV) && make(t + 3, s.out, s.seq_q, s.ld_out, 32);
+    };
+    if (!make4(tm + 4, b) || !make4(tm, a != nullptr ? *a : b)) return SOL_ERR_CUDA;  // one stream: the a maps are never used
     Params p{};
-    p.seq_q = static_cast<int>(seq_q);
-    p.seq_kv = static_cast<int>(seq_kv);
+    p.q_split = a != nullptr ? static_cast<int>(a->seq_q) : 0;
+    p.kv_split = a != nullptr ? static_cast<int>(a->seq_kv) : 0;
+    p.seq_q = p.q_split + static_cast<int>(b.seq_q);
+    p.seq_kv = p.kv_split + static_cast<int>(b.seq_kv);
     p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(kD));
     p.status = device_status_word();
     static bool configured[64] = {};
@@ -360,9 +377,9 @@ sol_status_t launch_attention(const void *q, const void *k, const void *v, void 
             return SOL_ERR_CUDA;
         configured[dev] = true;
     }
-    const dim3 grid(static_cast<unsigned>((seq_q + kQTiles * kBQ - 1) / (kQTiles * kBQ)), static_cast<unsigned>(heads),
+    const dim3 grid(static_cast<unsigned>((p.seq_q + kQTiles * kBQ - 1) / (kQTiles * kBQ)), static_cast<unsigned>(heads),
                     static_cast<unsigned>(batch));
-    attention_kernel<<<grid, kThreads, kSmem, stream>>>(tm_q, tm_k, tm_v, tm_o, p);
+    attention_kernel<<<grid, kThreads, kSmem, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], tm[7], p);
     return launch_status();
 }
 

@@ -114,9 +114,13 @@ bool make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t
                        uint64_t pitch2_bytes, uint32_t box0, uint32_t box1);
 
 namespace attn {
-sol_status_t launch_attention(const void *q, const void *k, const void *v, void *out, int64_t batch, int64_t seq_q,
-                              int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v, int64_t ld_out,
-                              cudaStream_t stream);
+struct Stream {   // one token stream of an attention call: [batch, seq, heads, 128] views with token pitches
+    const void *q, *k, *v;
+    void *out;
+    int64_t seq_q, seq_kv, ld_q, ld_k, ld_v, ld_out;
+};
+// Attention over the concatenation (a, then b) of two token streams, or over b alone when a is null.
+sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, cudaStream_t stream);
 }
 
 // Scale-factor buffer in the chunked layout as a 3-D tensor [row chunk][k chunk][128 x u32]; the box

@@ -140,6 +140,13 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.sol_attention_bf16(p, p, p, p, 70000, 4, 4, 1, 128, 128, 128, 128, None) == SHAPE
     assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 1, 132, 128, 128, 128, None) == ALIGN      # pitch % 8
     assert L.sol_attention_bf16(p, p + 8, p, p, 1, 4, 4, 1, 128, 128, 128, 128, None) == ALIGN
+    from paper_2604_06916_b200.binding import AttentionStream
+    ok = AttentionStream(p, p, p, p, 256, 128, 128, 128, 128)
+    assert L.sol_attention_bf16_joint(None, ctypes.byref(ok), 1, 1, None) == NULLP
+    assert L.sol_attention_bf16_joint(ctypes.byref(AttentionStream(p, None, p, p, 256, 128, 128, 128, 128)), ctypes.byref(ok), 1, 1, None) == NULLP
+    assert L.sol_attention_bf16_joint(ctypes.byref(AttentionStream(p, p, p, p, 200, 128, 128, 128, 128)), ctypes.byref(ok), 1, 1, None) == SHAPE  # first % 256
+    assert L.sol_attention_bf16_joint(ctypes.byref(ok), ctypes.byref(AttentionStream(p, p, p, p, 0, 128, 128, 128, 128)), 1, 1, None) == SHAPE
+    assert L.sol_attention_bf16_joint(ctypes.byref(ok), ctypes.byref(AttentionStream(p, p, p, p + 8, 5, 128, 128, 128, 128)), 1, 1, None) == ALIGN
     # MXFP4
     assert L.sol_mxfp4_scale_bytes(256, 512, 0) == 256 * 16 and L.sol_mxfp4_scale_bytes(256, 512, 1) == 2 * 4 * 512
     assert L.sol_mxfp4_scale_bytes(130, 160, 1) == 2 * 2 * 512 and L.sol_mxfp4_scale_bytes(4, 48, 1) == 0

@@ -104,3 +104,23 @@ def test_flux_geometry_sampled_rows(B):
     lib = torch.nn.functional.scaled_dot_product_attention(q.transpose(1, 2), k.transpose(1, 2), v.transpose(1, 2))
     d = (out.transpose(1, 2).float() - lib.float()).abs().max().item()
     assert d <= 2.0 ** -6 * 2.5, d
+
+
+@pytest.mark.parametrize("seq_a,seq_b", [(256, 128), (512, 1000), (256, 1), (768, 4096 - 768 + 37)])
+def test_joint_streams(B, seq_a, seq_b):
+    # text-like and image-like streams from separate fused projections, attending jointly
+    _, qa, ka, va = workloads.make_qkv(2, seq_a, 2, 61, "cuda")
+    _, qb, kb, vb = workloads.make_qkv(2, seq_b, 2, 62, "cuda")
+    oa, ob = B.sol_attention_bf16_joint((qa, ka, va), (qb, kb, vb))
+    torch.cuda.synchronize()
+    assert B.sol_last_device_status() == 0
+    first, second = tuple(f64(t) for t in (qa, ka, va)), tuple(f64(t) for t in (qb, kb, vb))
+    ra, rb = OA.attention_joint(first, second)
+    vall = np.concatenate((first[2], second[2]), axis=1)
+    for got, ref in ((oa, ra), (ob, rb)):
+        tol = OA.attention_tolerance(ref, vall)
+        assert np.all(np.abs(f64(got) - ref) <= tol)
+    # the same tiles in the same order as one call on the concatenated tensors: bit for bit
+    q, k, v = (torch.cat((x, y), dim=1) for x, y in ((qa, qb), (ka, kb), (va, vb)))
+    whole = B.sol_attention_bf16(q, k, v)
+    assert torch.equal(torch.cat((oa, ob), dim=1), whole)

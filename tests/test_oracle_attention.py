@@ -85,3 +85,20 @@ def test_large_scores_do_not_overflow():
     q = np.full((1, 128), 30.0); k = np.stack([np.full(128, 30.0), np.full(128, -30.0)]); v = np.array([[1.0] * 128, [5.0] * 128])
     out = A.attention_head(q, k, v)    # scores +-1.15e5 / 11.3: exp of the raw score overflows FP64
     assert np.all(np.isfinite(out)) and np.allclose(out, 1.0)
+
+
+def test_joint_streams_are_the_concatenation():
+    rng = np.random.default_rng(6)
+    a = tuple(rnd(rng, 2, 8, 2, 16) for _ in range(3))
+    b = tuple(rnd(rng, 2, 5, 2, 16) for _ in range(3))
+    oa, ob = A.attention_joint(a, b)
+    # every query of either stream sees all 13 keys: with the second stream's values set to a constant c and
+    # the first's to 0 the output is c times the probability mass on the second stream, the same for both halves
+    a0 = (a[0], a[1], np.zeros_like(a[2]))
+    b1 = (b[0], b[1], np.ones_like(b[2]))
+    ma, mb = A.attention_joint(a0, b1)
+    assert np.all((ma > 0) & (ma < 1)) and np.all((mb > 0) & (mb < 1))
+    # and a single stream split in two gives back the single-stream result
+    q, k, v = (np.concatenate((x, y), axis=1) for x, y in zip(a, b))
+    whole = A.attention(q, k, v)
+    np.testing.assert_array_equal(np.concatenate((oa, ob), axis=1), whole)
