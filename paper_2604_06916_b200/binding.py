@@ -379,24 +379,15 @@ def sol_attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: t
     projection output qualify.  Returns [B, Sq, H, 128].
     """
     for name, t in (("q", q), ("k", k), ("v", v)):
-        if t.dtype != torch.bfloat16 or t.dim() != 4 or t.shape[3] != 128:
-            raise ValueError(f"{name} must be a [B, S, H, 128] BF16 tensor")
-        if t.stride(3) != 1 or (t.shape[2] > 1 and t.stride(2) != 128) or \
-                (t.shape[0] > 1 and t.shape[1] > 1 and t.stride(0) != t.shape[1] * t.stride(1)):
-            raise ValueError(f"{name}: heads and head dimension must be contiguous, batches stacked densely")
+        _check_attention_view(name, t)
     B, Sq, H, _ = q.shape
-
-    def pitch(t):  # elements between consecutive tokens (a dimension of extent 1 has no meaningful stride)
-        if t.shape[1] > 1:
-            return t.stride(1)
-        return t.stride(0) if t.shape[0] > 1 else t.shape[2] * 128
-
     if k.shape != v.shape or k.shape[0] != B or k.shape[2] != H:
         raise ValueError("k and v must share [B, Skv, H, 128] with q's batch and heads")
     if out is None:
         out = torch.empty((B, Sq, H, 128), dtype=torch.bfloat16, device=q.device)
-    _check(lib().sol_attention_bf16(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, Sq, k.shape[1], H, pitch(q), pitch(k),
-                                    pitch(v), pitch(out), _stream()), "sol_attention_bf16")
+    _check_attention_view("out", out)
+    _check(lib().sol_attention_bf16(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, Sq, k.shape[1], H, _token_pitch(q),
+                                    _token_pitch(k), _token_pitch(v), _token_pitch(out), _stream()), "sol_attention_bf16")
     return out
 
 
