@@ -254,6 +254,24 @@ sol_status_t sol_attention_bf16(const void *q, const void *k, const void *v, voi
                                 void *stream);
 
 /*
+ * sol_attention_bf16 whose output leaves as the quantized activations of the linear that follows it in
+ * a DiT block (the output projection; in a single-stream block the concatenated input it shares
+ * with the MLP branch): h = bf16(attention output), then nvfp4_quantize's mapping with
+ * T = *out_tscale, written into columns [dest_col0, dest_col0 + heads * 128) of the NVFP4 tensor
+ * [batch * seq_q, dest_K] (rows of all samples stacked; chunked scale layout).  Bit for bit what
+ * sol_attention_bf16 followed by nvfp4_quantize_into produces, without the BF16 round trip through HBM.
+ *   out_tscale   caller supplied (a delayed scale); amax_out: nullable running max|h| as in
+ *                nvfp4_linear_quantized_out
+ *   dest_K % 64 == 0, dest_col0 % 64 == 0, dest_col0 + heads * 128 <= dest_K
+ * Bytes outside the column range are not touched, so the rows past batch * seq_q of the destination's
+ * last 128-row scale chunk must have been zeroed once.  Everything else as sol_attention_bf16.
+ */
+sol_status_t sol_attention_nvfp4_out(const void *q, const void *k, const void *v, int64_t batch, int64_t seq_q,
+                                     int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v,
+                                     const float *out_tscale, void *q_dest, void *sf_dest, int64_t dest_K,
+                                     int64_t dest_col0, float *amax_out, void *stream);
+
+/*
  * The same attention over two token streams that are projected separately and attend jointly, as in
  * the double-stream blocks of the FLUX.1 model of Section 4.1 (text tokens and image tokens): the
  * joint sequence is the first stream's tokens followed by the second's; queries, keys and values

@@ -26,6 +26,7 @@ EXPORTS = [
     "solrl_select_contrastive", "solrl_rank_consistency", "sol_mxfp4_scale_bytes", "mxfp4_quantize",
     "mxfp4_linear", "nvfp4_linear_split_out", "nvfp4_quantize_into",
     "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale", "nvfp4_layernorm_quantize", "sol_attention_bf16", "sol_attention_bf16_joint",
+    "sol_attention_nvfp4_out",
 ]
 
 _lib = None
@@ -93,6 +94,8 @@ def lib() -> ctypes.CDLL:
     L.sol_roll_tensor_scale.restype, L.sol_roll_tensor_scale.argtypes = i32, [vp, vp]
     L.sol_attention_bf16_joint.restype = i32
     L.sol_attention_bf16_joint.argtypes = [ctypes.POINTER(AttentionStream), ctypes.POINTER(AttentionStream), i64, i64, vp]
+    L.sol_attention_nvfp4_out.restype = i32
+    L.sol_attention_nvfp4_out.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, vp, vp, vp, i64, i64, vp, vp]
     L.sol_attention_bf16.restype = i32
     L.sol_attention_bf16.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, vp]
     L.nvfp4_layernorm_quantize.restype = i32
@@ -389,6 +392,26 @@ def sol_attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: t
     _check(lib().sol_attention_bf16(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, Sq, k.shape[1], H, _token_pitch(q),
                                     _token_pitch(k), _token_pitch(v), _token_pitch(out), _stream()), "sol_attention_bf16")
     return out
+
+
+def sol_attention_nvfp4_out(q, k, v, out_tscale: torch.Tensor, dest, dest_col0: int = 0,
+                            amax_out: torch.Tensor | None = None):
+    """Attention whose output is quantized into columns [dest_col0, dest_col0 + H * 128) of `dest`.
+
+    dest = (nibbles [B * Sq, dest_K / 2] uint8, swizzled scales of a [B * Sq, dest_K] tensor); returns dest.
+    """
+    for name, t in (("q", q), ("k", k), ("v", v)):
+        _check_attention_view(name, t)
+    B, Sq, H, _ = q.shape
+    if k.shape != v.shape or k.shape[0] != B or k.shape[2] != H:
+        raise ValueError("k and v must share [B, Skv, H, 128] with q's batch and heads")
+    dq, dsf = dest
+    if dq.dtype != torch.uint8 or dq.dim() != 2 or dq.shape[0] != B * Sq or not dq.is_contiguous():
+        raise ValueError("dest nibbles must be a contiguous [B * Sq, dest_K / 2] uint8 tensor")
+    _check(lib().sol_attention_nvfp4_out(_ptr(q), _ptr(k), _ptr(v), B, Sq, k.shape[1], H, _token_pitch(q), _token_pitch(k),
+                                         _token_pitch(v), _ptr(out_tscale), _ptr(dq), _ptr(dsf), dq.shape[1] * 2, dest_col0,
+                                         _ptr(amax_out), _stream()), "sol_attention_nvfp4_out")
+    return dest
 
 
 def mxfp4_scale_bytes(rows: int, K: int, layout: int = SF_SWIZZLED_128x4) -> int:

@@ -21,6 +21,7 @@
 // Warps: 0 = TMA producer, 1 = TMEM owner and MMA issuer, 2..5 and 6..9 = softmax / epilogue of query
 // tile 0 and 1 (one warp per TMEM lane quadrant).  Every mbarrier wait is bounded.
 #include "gemm_common.cuh"
+#include "quant_math.cuh"
 #include "sol_internal.h"
 
 namespace sol {
@@ -57,6 +58,14 @@ struct Params {
     int kv_split;
     float scale_log2;      // log2(e) / sqrt(d)
     uint32_t *status;
+    // quantized output (kQuantOut): the rows of all samples stacked, [batch * seq_q, dest_K] in NVFP4
+    uint8_t *q_dest;       // packed nibbles, dest_K / 2 bytes per row
+    uint8_t *sf_dest;      // chunked scale layout of a [batch * seq_q, dest_K] tensor
+    const float *ts_out;   // tensor scale of the destination (caller supplied)
+    uint32_t *amax_out;    // nullable: running max |h| as FP32 bits
+    int dest_pitch;        // dest_K / 2
+    int dest_col0;         // first destination column of head 0
+    int dest_chunks_k;     // dest_K / 64
 };
 
 __device__ __forceinline__ float ex2(float x) {
@@ -73,6 +82,9 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// kQuantOut: the output leaves as the next linear's NVFP4 activations (h = bf16(O / l), then the
+// quantizer's FP32 sequence per 16 columns) instead of BF16 -- one stream only.
+template <bool kQuantOut>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ CUtensorMap tm_ka,
                  const __grid_constant__ CUtensorMap tm_va, const __grid_constant__ CUtensorMap tm_oa,
@@ -311,6 +323,61 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
         if (ok && wait_bounded(bar(kPvDone + t), 0, abort_flag, p.status, 0xBA0u | t)) {
             ptx::tc_fence_after_sync();
             const float inv = 1.0f / l;
+            if constexpr (kQuantOut) {
+                // thread = row: 128 columns of one head = eight 16-element blocks, quantized from registers
+                const int row = q0 + t * kBQ + r;
+                const bool row_ok = row < q_rows;
+                const int64_t m = static_cast<int64_t>(batch) * p.seq_q + row;
+                const float T = __ldcg(p.ts_out);
+                const float c6T = __fmul_rn(6.0f, T);
+                const int col0 = p.dest_col0 + head * kD;
+                uint8_t *qrow = p.q_dest + m * p.dest_pitch + (col0 >> 1);
+                uint32_t amax2 = 0, sfw[2] = {0u, 0u};
+                uint32_t codes[16];  // the row's 128 nibbles: stored in one go so that its two 32-byte sectors fill at once
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    ptx::tmem_ld_32x32(t_lane + kColO + 32 * c, o);
+                    ptx::tmem_ld_wait();
+                    uint32_t w[16];
+                    uint32_t *code = codes + 4 * c;
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        w[e] = pack_bf16(__uint_as_float(o[2 * e]) * inv, __uint_as_float(o[2 * e + 1]) * inv);
+#pragma unroll
+                    for (int blk = 0; blk < 2; ++blk) {
+                        const uint32_t *b = w + 8 * blk;
+                        uint32_t a2 = qmath::absmax2(qmath::absmax2(qmath::absmax2(b[0], b[1]), qmath::absmax2(b[2], b[3])),
+                                                     qmath::absmax2(qmath::absmax2(b[4], b[5]), qmath::absmax2(b[6], b[7])));
+                        a2 &= 0x7FFF7FFFu;
+                        amax2 = qmath::absmax2(amax2, a2);
+                        const float a = fmaxf(qmath::bf16_lo(a2), qmath::bf16_hi(a2));
+                        float rcp;
+                        const uint32_t sb = qmath::block_scale(a, c6T, T, rcp);
+                        code[2 * blk] = qmath::quantize8(b[0], b[1], b[2], b[3], rcp);
+                        code[2 * blk + 1] = qmath::quantize8(b[4], b[5], b[6], b[7], rcp);
+                        sfw[c >> 1] |= sb << (8 * ((c & 1) * 2 + blk));
+                    }
+                }
+                if (row_ok) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        *reinterpret_cast<uint4 *>(qrow + 16 * c) = make_uint4(codes[4 * c], codes[4 * c + 1], codes[4 * c + 2], codes[4 * c + 3]);
+                }
+                if (row_ok) {
+#pragma unroll
+                    for (int kc = 0; kc < 2; ++kc) {  // the four scale bytes of a (row, 64-column chunk) slot are one word
+                        const int64_t chunk = (m >> 7) * p.dest_chunks_k + (col0 >> 6) + kc;
+                        *reinterpret_cast<uint32_t *>(p.sf_dest + chunk * 512 + (m & 31) * 16 + ((m & 127) >> 5) * 4) = sfw[kc];
+                    }
+                }
+                if (p.amax_out != nullptr) {
+                    amax2 &= 0x7FFF7FFFu;
+                    uint32_t mx = row_ok ? max(amax2 & 0xFFFFu, amax2 >> 16) : 0u;
+                    mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+                    if (lane == 0 && mx) atomicMax(p.amax_out, mx << 16);
+                }
+            } else {
             const uint32_t o_row = sQ + t * kTile + r * 128;  // Q_t is no longer read: its MMAs have completed
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -336,6 +403,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
                 ptx::tma_store_commit();
                 ptx::tma_store_wait_all<0>();
             }
+            }
         }
     }
 
@@ -350,7 +418,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
 
 }  // namespace
 
-sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, cudaStream_t stream) {
+sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, const QuantDest *qd,
+                              cudaStream_t stream) {
     CUtensorMap tm[8];
     const uint64_t cols = static_cast<uint64_t>(heads) * kD;
     auto make = [&](CUtensorMap *t, const void *base, int64_t seq, int64_t ld, uint32_t box_rows) {
@@ -358,8 +427,10 @@ sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, i
                                  static_cast<uint64_t>(ld) * 2, static_cast<uint64_t>(seq) * ld * 2, 64, box_rows);
     };
     auto make4 = [&](CUtensorMap *t, const Stream &s) {
+        // a quantized destination has no BF16 output tensor: the (unused) output map is a copy of the query map
         return make(t, s.q, s.seq_q, s.ld_q, kBQ) && make(t + 1, s.k, s.seq_kv, s.ld_k, kBKV) &&
-               make(t + 2, s.v, s.seq_kv, s.ld_v, kBKV) && make(t + 3, s.out, s.seq_q, s.ld_out, 32);
+               make(t + 2, s.v, s.seq_kv, s.ld_v, kBKV) &&
+               (qd != nullptr ? make(t + 3, s.q, s.seq_q, s.ld_q, 32) : make(t + 3, s.out, s.seq_q, s.ld_out, 32));
     };
     if (!make4(tm + 4, b) || !make4(tm, a != nullptr ? *a : b)) return SOL_ERR_CUDA;  // one stream: the a maps are never used
     Params p{};
@@ -369,17 +440,27 @@ sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, i
     p.seq_kv = p.kv_split + static_cast<int>(b.seq_kv);
     p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(kD));
     p.status = device_status_word();
-    static bool configured[64] = {};
+    if (qd != nullptr) {
+        p.q_dest = static_cast<uint8_t *>(qd->q);
+        p.sf_dest = static_cast<uint8_t *>(qd->sf);
+        p.ts_out = qd->tscale;
+        p.amax_out = qd->amax_out;
+        p.dest_pitch = static_cast<int>(qd->dest_K / 2);
+        p.dest_col0 = static_cast<int>(qd->dest_col0);
+        p.dest_chunks_k = static_cast<int>(qd->dest_K / 64);
+    }
+    auto kern = qd != nullptr ? attention_kernel<true> : attention_kernel<false>;
+    static bool configured[2][64] = {};
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SOL_ERR_CUDA;
-    if (!configured[dev]) {
-        if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+    if (!configured[qd != nullptr][dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
             return SOL_ERR_CUDA;
-        configured[dev] = true;
+        configured[qd != nullptr][dev] = true;
     }
     const dim3 grid(static_cast<unsigned>((p.seq_q + kQTiles * kBQ - 1) / (kQTiles * kBQ)), static_cast<unsigned>(heads),
                     static_cast<unsigned>(batch));
-    attention_kernel<<<grid, kThreads, kSmem, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], tm[7], p);
+    kern<<<grid, kThreads, kSmem, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], tm[7], p);
     return launch_status();
 }
 

@@ -119,8 +119,16 @@ struct Stream {   // one token stream of an attention call: [batch, seq, heads, 
     void *out;
     int64_t seq_q, seq_kv, ld_q, ld_k, ld_v, ld_out;
 };
-// Attention over the concatenation (a, then b) of two token streams, or over b alone when a is null.
-sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, cudaStream_t stream);
+struct QuantDest {   // NVFP4 destination of the output: columns [dest_col0, dest_col0 + heads * 128) of a [rows, dest_K] tensor
+    void *q, *sf;
+    const float *tscale;
+    uint32_t *amax_out;
+    int64_t dest_K, dest_col0;
+};
+// Attention over the concatenation (a, then b) of two token streams, or over b alone when a is null;
+// with `qd` (one stream only) the output is quantized into `qd` instead of written as BF16.
+sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, const QuantDest *qd,
+                              cudaStream_t stream);
 }
 
 // Scale-factor buffer in the chunked layout as a 3-D tensor [row chunk][k chunk][128 x u32]; the box

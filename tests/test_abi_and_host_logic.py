@@ -140,6 +140,10 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.sol_attention_bf16(p, p, p, p, 70000, 4, 4, 1, 128, 128, 128, 128, None) == SHAPE
     assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 1, 132, 128, 128, 128, None) == ALIGN      # pitch % 8
     assert L.sol_attention_bf16(p, p + 8, p, p, 1, 4, 4, 1, 128, 128, 128, 128, None) == ALIGN
+    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, None, p, p, 128, 0, None, None) == NULLP
+    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, p, p, p, 96, 0, None, None) == SHAPE     # dest_K % 64
+    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, p, p, p, 128, 64, None, None) == SHAPE   # past the end
+    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, p, p + 8, p, 128, 0, None, None) == ALIGN
     from paper_2604_06916_b200.binding import AttentionStream
     ok = AttentionStream(p, p, p, p, 256, 128, 128, 128, 128)
     assert L.sol_attention_bf16_joint(None, ctypes.byref(ok), 1, 1, None) == NULLP

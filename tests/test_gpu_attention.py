@@ -124,3 +124,37 @@ def test_joint_streams(B, seq_a, seq_b):
     q, k, v = (torch.cat((x, y), dim=1) for x, y in ((qa, qb), (ka, kb), (va, vb)))
     whole = B.sol_attention_bf16(q, k, v)
     assert torch.equal(torch.cat((oa, ob), dim=1), whole)
+
+
+@pytest.mark.parametrize("batch,seq,heads,dest_cols,col0", [(2, 300, 2, 256, 0), (1, 1024, 3, 1024, 384), (3, 130, 1, 192, 64)])
+def test_quantized_output_equals_attention_then_quantizer(B, batch, seq, heads, dest_cols, col0):
+    # the fused epilogue must give, bit for bit, what the BF16 kernel followed by the destination-slice
+    # quantizer gives (each of which is checked against the oracle on its own); other columns stay untouched
+    _, q, k, v = workloads.make_qkv(batch, seq, heads, 71, "cuda")
+    M = batch * seq
+    o = B.sol_attention_bf16(q, k, v).reshape(M, heads * 128)
+    T = B.sol_amax_bf16(o)
+    def fresh():
+        dq = torch.full((M, dest_cols // 2), 0x5A, dtype=torch.uint8, device="cuda")
+        dsf = torch.zeros(B.scale_bytes(M, dest_cols), dtype=torch.uint8, device="cuda")
+        return dq, dsf
+    want = fresh()
+    B.nvfp4_quantize_into(o, T, want, col0)
+    got = fresh()
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    B.sol_attention_nvfp4_out(q, k, v, T, got, col0, amax_out=amax)
+    torch.cuda.synchronize()
+    assert B.sol_last_device_status() == 0
+    assert torch.equal(got[0], want[0]) and torch.equal(got[1], want[1])
+    assert amax.item() == o.float().abs().max().item()
+    # and end to end against the FP64 oracle: every dequantized value within the attention tolerance plus half
+    # the widest FP4 step (1 unit of the block scale) of the FP64 output
+    from tests.helpers import dequantize_on_device
+    cols = heads * 128
+    sub_q = got[0][:, col0 // 2:(col0 + cols) // 2].contiguous()
+    full = dequantize_on_device(got[0], got[1], M, dest_cols).float()[:, col0:col0 + cols] * T.item()
+    ref = OA.attention(f64(q), f64(k), f64(v)).reshape(M, cols)
+    step = (full.abs().reshape(M, cols // 16, 16).amax(dim=2, keepdim=True) / 6.0 * 1.0).expand(M, cols // 16, 16).reshape(M, cols)
+    tol = OA.attention_tolerance(ref.reshape(batch, seq, heads, 128), f64(v)).reshape(M, cols) + 1.01 * step.cpu().numpy() + 1e-30
+    assert sub_q.shape == (M, cols // 2)
+    assert np.all(np.abs(full.cpu().numpy().astype(np.float64) - ref) <= tol)
