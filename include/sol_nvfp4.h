@@ -363,6 +363,17 @@ sol_status_t mxfp4_linear(const void *xq, const void *xsf, const void *wq, const
                           void *y_bf16, int64_t M, int64_t N, int64_t K, int64_t ldy, void *stream);
 
 /*
+ * mxfp4_linear whose output leaves as the MXFP4 activations of the next linear (the MXFP4 form of
+ * nvfp4_linear_quantized_out): h = bf16_rne(act(Y)), then mxfp4_quantize's mapping along N.
+ *   hq_out   [M, N/2] nibbles;  hsf_out  SOL_SF_SWIZZLED_128x4 MXFP4 scales of an [M, N] tensor, every byte written
+ *   amax_out nullable running max|h| (FP32 bits, atomic max); N % 128 == 0
+ * No tensor scales anywhere: the format has none.  Errors as nvfp4_linear_quantized_out.
+ */
+sol_status_t mxfp4_linear_quantized_out(const void *xq, const void *xsf, const void *wq, const void *wsf,
+                                        const void *bias_bf16, sol_activation_t activation, void *hq_out, void *hsf_out,
+                                        float *amax_out, int64_t M, int64_t N, int64_t K, void *stream);
+
+/*
  * Stage-1 selection (Section 3.4; Section 4.1 "Rollout Generation": N = 96 candidates per prompt,
  * the 12 best and 12 worst kept, their initial noises preserved) and the group-standardised
  * advantages of the GRPO equation in Section 2, A_i = (R_i - mean) / population std.

@@ -296,6 +296,16 @@ def nvfp4_linear_quantized(qx, sfx, Tx, qw, sfw, Tw, bias_bits, act: int, T_out,
     return H, h, q, sf
 
 
+def mxfp4_linear_quantized(qx, sfx, qw, sfw, bias_bits, act: int, rows=None):
+    """The MXFP4 linear followed by an activation and the MXFP4 quantizer of the NEXT linear: H = act(Y),
+    h = H rounded once to BF16, (q, sf) = mxfp4_quantize(h).  Returns (H as FP64, h bits, nibbles, row-major scales)."""
+    Y = mxfp4_linear(qx, sfx, qw, sfw, bias_bits, rows=rows)
+    H = gelu_tanh(Y) if act == ACT_GELU_TANH else Y
+    h = round_bf16(H)
+    q, sf = mxfp4_quantize(h)
+    return H, h, q, sf
+
+
 LN_EPS = 1e-6
 
 

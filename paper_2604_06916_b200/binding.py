@@ -26,7 +26,7 @@ EXPORTS = [
     "solrl_select_contrastive", "solrl_rank_consistency", "sol_mxfp4_scale_bytes", "mxfp4_quantize",
     "mxfp4_linear", "nvfp4_linear_split_out", "nvfp4_quantize_into",
     "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale", "nvfp4_layernorm_quantize", "sol_attention_bf16", "sol_attention_bf16_joint",
-    "sol_attention_nvfp4_out",
+    "sol_attention_nvfp4_out", "mxfp4_linear_quantized_out",
 ]
 
 _lib = None
@@ -94,6 +94,8 @@ def lib() -> ctypes.CDLL:
     L.sol_roll_tensor_scale.restype, L.sol_roll_tensor_scale.argtypes = i32, [vp, vp]
     L.sol_attention_bf16_joint.restype = i32
     L.sol_attention_bf16_joint.argtypes = [ctypes.POINTER(AttentionStream), ctypes.POINTER(AttentionStream), i64, i64, vp]
+    L.mxfp4_linear_quantized_out.restype = i32
+    L.mxfp4_linear_quantized_out.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, vp, i64, i64, i64, vp]
     L.sol_attention_nvfp4_out.restype = i32
     L.sol_attention_nvfp4_out.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, vp, vp, vp, i64, i64, vp, vp]
     L.sol_attention_bf16.restype = i32
@@ -488,6 +490,19 @@ def nvfp4_linear_quantized_out(xq, xsf, x_tscale, wq, wsf, w_tscale, bias, activ
     _check(lib().nvfp4_linear_quantized_out(_ptr(xq), _ptr(xsf), _ptr(x_tscale), _ptr(wq), _ptr(wsf), _ptr(w_tscale),
                                             _ptr(bias), activation, _ptr(out_tscale), _ptr(hq), _ptr(hsf),
                                             _ptr(amax_out), M, N, K, _stream()), "nvfp4_linear_quantized_out")
+    return hq, hsf
+
+
+def mxfp4_linear_quantized_out(xq, xsf, wq, wsf, bias, activation: int, amax_out: torch.Tensor | None = None, out=None):
+    """MXFP4 linear whose output leaves as (nibbles [M, N/2], swizzled E8M0 scales) for the next MXFP4 linear."""
+    M, K = xq.shape[0], xq.shape[1] * 2
+    N = wq.shape[0]
+    if out is None:
+        out = (torch.empty((M, N // 2), dtype=torch.uint8, device=xq.device),
+               torch.empty(mxfp4_scale_bytes(M, N), dtype=torch.uint8, device=xq.device))
+    hq, hsf = out
+    _check(lib().mxfp4_linear_quantized_out(_ptr(xq), _ptr(xsf), _ptr(wq), _ptr(wsf), _ptr(bias), activation, _ptr(hq),
+                                            _ptr(hsf), _ptr(amax_out), M, N, K, _stream()), "mxfp4_linear_quantized_out")
     return hq, hsf
 
 

@@ -382,6 +382,25 @@ sol_status_t mxfp4_linear(const void *xq, const void *xsf, const void *wq, const
                                       static_cast<cudaStream_t>(stream), dev);
 }
 
+sol_status_t mxfp4_linear_quantized_out(const void *xq, const void *xsf, const void *wq, const void *wsf,
+                                        const void *bias_bf16, sol_activation_t activation, void *hq_out, void *hsf_out,
+                                        float *amax_out, int64_t M, int64_t N, int64_t K, void *stream) {
+    if (xq == nullptr || xsf == nullptr || wq == nullptr || wsf == nullptr || hq_out == nullptr || hsf_out == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(M, K) || N <= 0 || N % 128 != 0 || N > (1LL << 24)) return SOL_ERR_BAD_SHAPE;
+    if (activation != SOL_ACT_NONE && activation != SOL_ACT_GELU_TANH) return SOL_ERR_BAD_LAYOUT;
+    if (!aligned16(xq) || !aligned16(xsf) || !aligned16(wq) || !aligned16(wsf) || !aligned16(hq_out) ||
+        !aligned16(hsf_out) || (bias_bf16 != nullptr && !aligned16(bias_bf16)) ||
+        (reinterpret_cast<uintptr_t>(amax_out) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return gemm::launch_pair256_mxfp4_quant_out(xq, xsf, wq, wsf, bias_bf16, activation == SOL_ACT_GELU_TANH ? 1 : 0,
+                                                hq_out, hsf_out, reinterpret_cast<uint32_t *>(amax_out), M, N, K,
+                                                static_cast<cudaStream_t>(stream), dev);
+}
+
 sol_status_t solrl_select_contrastive(const float *rewards, const uint64_t *seeds, int64_t P, int64_t N, int64_t K,
                                       int32_t *idx_out, uint64_t *seeds_out, float *advantages_out, void *stream) {
     if (rewards == nullptr || idx_out == nullptr || (seeds_out != nullptr && seeds == nullptr)) return SOL_ERR_NULL_POINTER;

@@ -173,8 +173,77 @@ __device__ __forceinline__ void epilogue_quant_store(const CUtensorMap *tm_q, co
     }
 }
 
+// The MXFP4 form of the same: two 32-element blocks per 64-column chunk, each with the E8M0 scale
+// 2^(floor(log2 amax) - 2) taken from the exponent field of the block maximum, codes by an exact
+// power-of-two scaling; no tensor scale.  A scale chunk of the destination spans 128 columns, so the
+// chunk's two scale bytes are one 2-byte store into the lower or upper half of a (row, chunk) slot.
+__device__ __forceinline__ void epilogue_quant_store_mx(const CUtensorMap *tm_q, const Params &p, const uint32_t (&lo)[32],
+                                                        const uint32_t (&hi)[32], int m0, int quad_in_tile, int row_tile,
+                                                        int nc, float alpha, uint32_t sbuf, uint32_t sbias, int lane,
+                                                        uint32_t &amax2) {
+    const bool gelu = p.act != 0;
+    if (lane == 0) ptx::tma_store_wait_read<0>();
+    __syncwarp();
+    uint32_t sfw = 0;
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk) {
+        uint32_t hw[16];  // thirty-two BF16 values of h
+        uint32_t bm = 0;
+#pragma unroll
+        for (int g4 = 0; g4 < 4; ++g4) {
+            const int g = blk * 4 + g4;
+            uint32_t bw[4];
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(bw[0]), "=r"(bw[1]), "=r"(bw[2]), "=r"(bw[3])
+                         : "r"(sbias + g * 16));
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t a0 = g < 4 ? lo[g * 8 + 2 * e] : hi[(g - 4) * 8 + 2 * e];
+                const uint32_t a1 = g < 4 ? lo[g * 8 + 2 * e + 1] : hi[(g - 4) * 8 + 2 * e + 1];
+                float y0 = fmaf(__uint_as_float(a0), alpha, __uint_as_float(bw[e] << 16));
+                float y1 = fmaf(__uint_as_float(a1), alpha, __uint_as_float(bw[e] & 0xFFFF0000u));
+                if (gelu) {
+                    y0 = gelu_tanh(y0);
+                    y1 = gelu_tanh(y1);
+                }
+                __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
+                const uint32_t w = *reinterpret_cast<uint32_t *>(&pk);
+                hw[g4 * 4 + e] = w;
+                bm = qmath::absmax2(bm, w);
+            }
+        }
+        amax2 = qmath::absmax2(amax2, bm);
+        bm &= 0x7FFF7FFFu;
+        const uint32_t e8 = max(bm & 0xFFFFu, bm >> 16) >> 7;   // biased exponent of the block maximum
+        const uint32_t sb = e8 > 2u ? e8 - 2u : 0u;             // shared exponent floor(log2 amax) - 2, clamped at -127
+        const float inv = __uint_as_float((254u - sb) << 23);   // 2^(127 - sb), exact
+        sfw |= sb << (8 * blk);
+#pragma unroll
+        for (int h8 = 0; h8 < 2; ++h8) {
+            const uint32_t q0 = qmath::quantize8(hw[8 * h8], hw[8 * h8 + 1], hw[8 * h8 + 2], hw[8 * h8 + 3], inv);
+            const uint32_t q1 = qmath::quantize8(hw[8 * h8 + 4], hw[8 * h8 + 5], hw[8 * h8 + 6], hw[8 * h8 + 7], inv);
+            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sbuf + lane * 32 + blk * 16 + h8 * 8), "r"(q0), "r"(q1)
+                         : "memory");
+        }
+    }
+    const bool unit_ok = nc < p.N && !(kTuning && (p.dbg & kDbgNoStore));
+    if (unit_ok && row_tile * 128 < p.M) {
+        if (m0 + lane >= p.M) sfw = 0;  // rows past M inside the last 128-row chunk are padding and read as 0
+        const int64_t chunk = static_cast<int64_t>(row_tile) * p.dest_chunks_k + (nc >> 7);
+        *reinterpret_cast<uint16_t *>(p.sf_out + chunk * 512 + lane * 16 + quad_in_tile * 4 + ((nc >> 6) & 1) * 2) =
+            static_cast<uint16_t>(sfw);
+    }
+    ptx::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        if (unit_ok && m0 < p.M) ptx::tma_store_2d(tm_q, nc >> 1, m0, sbuf);
+        ptx::tma_store_commit();
+    }
+}
+
 // kMx: MXFP4 operands (32-element blocks, E8M0 scales: a 512-byte scale chunk spans 128 elements of K,
-// so a k-tile has two chunks per 128 rows instead of four, and no tensor scales) -- BF16 output only.
+// so a k-tile has two chunks per 128 rows instead of four, and no tensor scales) -- BF16 output, or
+// (kOutQuant) the next linear's MXFP4 activations.
 template <int kOut, bool kMx>
 __global__ void __launch_bounds__(kThreadsFp4, 1)
 gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
@@ -516,7 +585,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         const uint32_t sbuf = epi_base + e * kEpiBufBytes;
         const uint32_t sbias = bias_base + e * 256;
         const float alpha = kMx ? 1.0f : __fmul_rn(__ldcg(p.ts_a), __ldcg(p.ts_b));
-        const float Tq = kOut != kOutBf16 ? __ldcg(p.ts_out) : 1.0f;
+        const float Tq = (kOut != kOutBf16 && !kMx) ? __ldcg(p.ts_out) : 1.0f;
         const float c6T = __fmul_rn(6.0f, Tq);
         uint32_t amax2 = 0;
         for (int t = pair, it = 0; t < total_tiles; t += num_pairs, ++it) {
@@ -574,6 +643,9 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             const int dst_shift = kOut == kOutSplit ? p.dest_col0 - p.n_split : 0;
             if (as_bf16)
                 epilogue_store(&tm_y, p, a_lo, a_hi, m0, n0 + first * 64, alpha, sbuf, sbias, lane);
+            else if constexpr (kMx)
+                epilogue_quant_store_mx(&tm_q, p, a_lo, a_hi, m0, quad, row_tile, n0 + first * 64, alpha, sbuf, sbias, lane,
+                                        amax2);
             else
                 epilogue_quant_store(&tm_q, p, a_lo, a_hi, m0, quad, row_tile, n0 + first * 64,
                                      n0 + first * 64 + dst_shift, alpha, Tq, c6T, sbuf, sbias, lane, amax2);
@@ -588,6 +660,13 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     epilogue_store(&tm_y, p, b_ot, b_sh, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
                 else
                     epilogue_store(&tm_y, p, b_sh, b_ot, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
+            } else if constexpr (kMx) {
+                if (x == 0)
+                    epilogue_quant_store_mx(&tm_q, p, b_ot, b_sh, m0, quad, row_tile, n0 + second * 64, alpha, sbuf,
+                                            sbias + 128, lane, amax2);
+                else
+                    epilogue_quant_store_mx(&tm_q, p, b_sh, b_ot, m0, quad, row_tile, n0 + second * 64, alpha, sbuf,
+                                            sbias + 128, lane, amax2);
             } else {
                 if (x == 0)
                     epilogue_quant_store(&tm_q, p, b_ot, b_sh, m0, quad, row_tile, n0 + second * 64,
@@ -670,16 +749,16 @@ sol_status_t launch_pair256(int out_mode, bool mx, const void *xq, const void *x
     p.act = qo.act;
     p.n_split = static_cast<int>(qo.n_split);
     p.dest_col0 = static_cast<int>(qo.dest_col0);
-    p.dest_chunks_k = static_cast<int>(qo.dest_K >> 6);
+    p.dest_chunks_k = static_cast<int>(mx ? qo.dest_K >> 7 : qo.dest_K >> 6);  // a scale chunk spans 64 (NVFP4) or 128 columns
 #ifdef SOL_TUNING
     if (const char *e = getenv("SOL_DBG")) p.dbg = static_cast<uint32_t>(atoi(e));
 #endif
-    auto kern = mx ? gemm_pair_fp4_kernel<kOutBf16, true>
+    auto kern = mx ? (out_mode == kOutQuant ? gemm_pair_fp4_kernel<kOutQuant, true> : gemm_pair_fp4_kernel<kOutBf16, true>)
                 : out_mode == kOutBf16 ? gemm_pair_fp4_kernel<kOutBf16, false>
                 : out_mode == kOutQuant ? gemm_pair_fp4_kernel<kOutQuant, false>
                                         : gemm_pair_fp4_kernel<kOutSplit, false>;
-    static bool configured[4][64] = {};
-    const int slot = mx ? 3 : out_mode;
+    static bool configured[5][64] = {};
+    const int slot = mx ? (out_mode == kOutQuant ? 4 : 3) : out_mode;
     if (dev->device < 64 && !configured[slot][dev->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return SOL_ERR_CUDA;
@@ -727,6 +806,18 @@ sol_status_t launch_pair256_mxfp4(const void *xq, const void *xsf, const void *w
                                   const DeviceInfo *dev) {
     return launch_pair256(kOutBf16, true, xq, xsf, nullptr, wq, wsf, nullptr, bias, y, ldy, QuantOut{}, M, N, K, stream,
                           dev);
+}
+
+sol_status_t launch_pair256_mxfp4_quant_out(const void *xq, const void *xsf, const void *wq, const void *wsf,
+                                            const void *bias, int act, void *hq, void *hsf, uint32_t *amax_out, int64_t M,
+                                            int64_t N, int64_t K, cudaStream_t stream, const DeviceInfo *dev) {
+    QuantOut qo;
+    qo.act = act;
+    qo.hq = hq;
+    qo.hsf = hsf;
+    qo.amax_out = amax_out;
+    qo.dest_K = N;
+    return launch_pair256(kOutQuant, true, xq, xsf, nullptr, wq, wsf, nullptr, bias, nullptr, 0, qo, M, N, K, stream, dev);
 }
 
 sol_status_t launch_pair256_nvfp4_quant_out(const void *xq, const void *xsf, const float *xts, const void *wq,

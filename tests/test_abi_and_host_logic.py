@@ -140,6 +140,9 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.sol_attention_bf16(p, p, p, p, 70000, 4, 4, 1, 128, 128, 128, 128, None) == SHAPE
     assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 1, 132, 128, 128, 128, None) == ALIGN      # pitch % 8
     assert L.sol_attention_bf16(p, p + 8, p, p, 1, 4, 4, 1, 128, 128, 128, 128, None) == ALIGN
+    assert L.mxfp4_linear_quantized_out(p, p, p, None, None, 0, p, p, None, 4, 128, 64, None) == NULLP
+    assert L.mxfp4_linear_quantized_out(p, p, p, p, None, 0, p, p, None, 4, 192, 64, None) == SHAPE      # N % 128
+    assert L.mxfp4_linear_quantized_out(p, p, p, p, None, 0, p + 8, p, None, 4, 128, 64, None) == ALIGN
     assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, None, p, p, 128, 0, None, None) == NULLP
     assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, p, p, p, 96, 0, None, None) == SHAPE     # dest_K % 64
     assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, p, p, p, 128, 64, None, None) == SHAPE   # past the end

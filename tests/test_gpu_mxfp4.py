@@ -128,3 +128,70 @@ def test_flux_layers_sampled_rows(B, index):
     assert np.array_equal(wsf.cpu().numpy(), oracle.mx_sf_swizzle(want_sfw, K))
     Y = oracle.mxfp4_linear(want_qx, want_sfx, want_qw, want_sfw, bits_of(bias))
     check_linear(bits_of(y[rows_t]), Y, f"{cfg.name}/{layer.name} mxfp4")
+
+
+@pytest.mark.parametrize("M,N,K", [(256, 256, 64), (128, 384, 256), (300, 512, 448), (64, 128, 32), (520, 1024, 512)])
+def test_quantized_output_integer_exact_bit_for_bit(B, M, N, K):
+    rng = np.random.default_rng(M * 5 + N + K)
+    qx = rng.integers(0, 256, size=(M, K // 2), dtype=np.uint8)
+    qw = rng.integers(0, 256, size=(N, K // 2), dtype=np.uint8)
+    sfx = (rng.integers(-2, 3, size=(M, K // 32)) + 127).astype(np.uint8)
+    sfw = (rng.integers(-2, 3, size=(N, K // 32)) + 127).astype(np.uint8)
+    H, h, q_star, sf_star = oracle.mxfp4_linear_quantized(qx, sfx, qw, sfw, None, oracle.ACT_NONE)
+    if np.abs(H).max() * 4 >= 2 ** 24:
+        pytest.skip("sum too large for an exact FP32 accumulator")
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    hq, hsf = B.mxfp4_linear_quantized_out(dev(qx), dev(oracle.mx_sf_swizzle(sfx, K)), dev(qw),
+                                           dev(oracle.mx_sf_swizzle(sfw, K)), None, B.ACT_NONE, amax_out=amax)
+    B.sol_last_device_status()
+    assert np.array_equal(hq.cpu().numpy(), q_star)
+    assert np.array_equal(hsf.cpu().numpy(), oracle.mx_sf_swizzle(sf_star, N))      # padding rows are 0
+    assert amax.item() == np.abs(oracle.bits_to_f64(h)).max()
+
+
+@pytest.mark.parametrize("M,N,K", [(384, 512, 1024), (1000, 384, 96), (4608, 1536, 3072)])
+def test_quantized_output_equals_linear_then_quantizer(B, M, N, K):
+    # without an activation the fused epilogue rounds the same FP32 accumulator to BF16 and applies the same
+    # quantizer arithmetic as mxfp4_linear followed by mxfp4_quantize (both checked against the oracle above)
+    g = torch.Generator(device="cuda").manual_seed(M + N + K)
+    X = workloads.make_activation("student_t", M, K, g, "cuda")
+    W = (torch.randn(N, K, generator=g, device="cuda") * K ** -0.5).to(torch.bfloat16)
+    bias = (torch.randn(N, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    xq, xsf = B.mxfp4_quantize(X)
+    wq, wsf = B.mxfp4_quantize(W)
+    y = B.mxfp4_linear(xq, xsf, wq, wsf, bias)
+    want_q, want_sf = B.mxfp4_quantize(y)
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    hq, hsf = B.mxfp4_linear_quantized_out(xq, xsf, wq, wsf, bias, B.ACT_NONE, amax_out=amax)
+    B.sol_last_device_status()
+    assert torch.equal(hq, want_q) and torch.equal(hsf, want_sf)
+    assert amax.item() == y.float().abs().max().item()
+
+
+def test_quantized_output_with_gelu_against_oracle(B):
+    M, N, K = 300, 256, 512
+    g = torch.Generator(device="cuda").manual_seed(99)
+    X = workloads.make_activation("student_t", M, K, g, "cuda")
+    W = (torch.randn(N, K, generator=g, device="cuda") * K ** -0.5).to(torch.bfloat16)
+    bias = (torch.randn(N, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    qx, sfx = oracle.mxfp4_quantize(bits_of(X))
+    qw, sfw = oracle.mxfp4_quantize(bits_of(W))
+    H, h, q_star, sf_star = oracle.mxfp4_linear_quantized(qx, sfx, qw, sfw, bits_of(bias), oracle.ACT_GELU_TANH)
+    hq, hsf = B.mxfp4_linear_quantized_out(dev(qx), dev(oracle.mx_sf_swizzle(sfx, K)), dev(qw),
+                                           dev(oracle.mx_sf_swizzle(sfw, K)), bias, B.ACT_GELU_TANH)
+    B.sol_last_device_status()
+    sf_rm = hsf.cpu().numpy()[mx_offsets(np.arange(M), N)]
+    # scale bytes: the block maximum may sit on either side of a power of two in a few blocks, never further
+    d = np.abs(sf_rm.astype(np.int32) - sf_star.astype(np.int32))
+    assert d.max() <= 1 and (d == 0).mean() >= 0.99
+    # every dequantized value within the format's widest half step (1 unit of the emitted scale), or its
+    # saturation distance, plus the linear's tolerance (GELU's slope is below 1.13) of the FP64 result
+    deq = oracle.mxfp4_dequantize(hq.cpu().numpy(), sf_rm)
+    scale = np.repeat(np.ldexp(1.0, sf_rm.astype(np.int32) - 127), 32, axis=1)
+    Y = oracle.mxfp4_linear(qx, sfx, qw, sfw, bits_of(bias))
+    tol = 1.2 * oracle.linear_tolerance(Y) + 2.0 ** -8 * np.abs(H)
+    # (a block maximum up to 8 units saturates at the largest code, 6 units)
+    reach = np.maximum(1.0 * scale, np.abs(H) - 6.0 * scale)
+    assert np.all(np.abs(deq - H) <= reach * (1 + 2.0 ** -6) + tol)
+    # and it is the oracle's own output almost everywhere
+    assert (hq.cpu().numpy() == q_star).mean() >= 0.98

@@ -170,3 +170,26 @@ def test_linear_integer_exact_and_structure():
     A = oracle.mxfp4_dequantize(qx, (ex + 127).astype(np.uint8))
     Bm = oracle.mxfp4_dequantize(qw, (ew + 127).astype(np.uint8))
     assert np.allclose(Y, A @ Bm.T, rtol=1e-13, atol=0)
+
+
+def test_linear_quantized_is_linear_then_round_then_quantizer():
+    # the composition the fused GPU epilogue is checked against: every step is one the tests above pin
+    rng = np.random.default_rng(17)
+    M, N, K = 6, 64, 64
+    qx = rng.integers(0, 256, size=(M, K // 2), dtype=np.uint8)
+    qw = rng.integers(0, 256, size=(N, K // 2), dtype=np.uint8)
+    sfx = (rng.integers(-1, 2, size=(M, K // 32)) + 127).astype(np.uint8)
+    sfw = (rng.integers(-1, 2, size=(N, K // 32)) + 127).astype(np.uint8)
+    H, h, q, sf = oracle.mxfp4_linear_quantized(qx, sfx, qw, sfw, None, oracle.ACT_NONE)
+    Y = oracle.mxfp4_linear(qx, sfx, qw, sfw)
+    assert np.array_equal(H, Y) and np.array_equal(h, oracle.round_bf16(Y))
+    q2, sf2 = oracle.mxfp4_quantize(h)
+    assert np.array_equal(q, q2) and np.array_equal(sf, sf2)
+    # with the activation the pre-quantizer values are GELU of the linear
+    Hg, hg, _, _ = oracle.mxfp4_linear_quantized(qx, sfx, qw, sfw, None, oracle.ACT_GELU_TANH)
+    assert np.array_equal(Hg, oracle.gelu_tanh(Y)) and np.array_equal(hg, oracle.round_bf16(oracle.gelu_tanh(Y)))
+    # dequantizing recovers every h to within the block's widest half step (1 unit) or its saturation distance
+    deq = oracle.mxfp4_dequantize(q, sf)
+    unit = np.repeat(np.ldexp(1.0, sf.astype(np.int32) - 127), 32, axis=1)
+    hv = oracle.bits_to_f64(h)
+    assert np.all(np.abs(deq - hv) <= np.maximum(unit, np.abs(hv) - 6 * unit) + 1e-12)
