@@ -434,6 +434,32 @@ def run_ours(args):
                     "note": "unfused = BF16 intermediate, dynamic amax + quantizer per layer, no separate GELU pass "
                             "counted; fused = nvfp4_linear_quantized_out (GELU, calibrated T) feeding nvfp4_linear"}
         del xq, xsf, hq, hsf
+        # the same pair in MXFP4 (no amax pass in either form: the format has no tensor scale)
+        w1mx, w2mx = B.mxfp4_quantize(d1["W"]), B.mxfp4_quantize(d2["W"])
+        xmx = (torch.empty((l1.M, l1.K // 2), dtype=torch.uint8, device=dev),
+               torch.empty(B.mxfp4_scale_bytes(l1.M, l1.K), dtype=torch.uint8, device=dev))
+        hmx = (torch.empty((l1.M, l1.N // 2), dtype=torch.uint8, device=dev),
+               torch.empty(B.mxfp4_scale_bytes(l1.M, l1.N), dtype=torch.uint8, device=dev))
+
+        def mx_unfused():
+            B.mxfp4_quantize(d1["X"], B.SF_SWIZZLED_128x4, out=xmx)
+            B.mxfp4_linear(xmx[0], xmx[1], w1mx[0], w1mx[1], d1["bias"], out=d1["Y"])
+            B.mxfp4_quantize(d1["Y"], B.SF_SWIZZLED_128x4, out=hmx)
+            B.mxfp4_linear(hmx[0], hmx[1], w2mx[0], w2mx[1], d2["bias"], out=d2["Y"])
+
+        def mx_fused():
+            B.mxfp4_quantize(d1["X"], B.SF_SWIZZLED_128x4, out=xmx)
+            B.mxfp4_linear_quantized_out(xmx[0], xmx[1], w1mx[0], w1mx[1], d1["bias"], B.ACT_GELU_TANH, out=hmx)
+            B.mxfp4_linear(hmx[0], hmx[1], w2mx[0], w2mx[1], d2["bias"], out=d2["Y"])
+
+        t_mu, t_mf = loop_ms(mx_unfused), loop_ms(mx_fused)
+        t_mu, t_mf = min(t_mu, loop_ms(mx_unfused)), min(t_mf, loop_ms(mx_fused))
+        B.sol_last_device_status()
+        mlp_pair["mxfp4"] = {"unfused_ms": t_mu, "fused_ms": t_mf, "speedup": t_mu / t_mf,
+                             "fused_tflops": pair_flops / t_mf / 1e9, "unfused_tflops": pair_flops / t_mu / 1e9,
+                             "note": "unfused = BF16 intermediate and a quantizer pass (no GELU pass counted); fused = "
+                                     "mxfp4_linear_quantized_out (GELU) feeding mxfp4_linear"}
+        del w1mx, w2mx, xmx, hmx
 
     # ---- single-stream block pair with the concatenated intermediate kept in NVFP4: the first linear's
     # q/k/v columns leave as BF16, its MLP columns pass GELU and are quantized straight into the second
