@@ -25,12 +25,6 @@ namespace {
 constexpr int kLnMaxWarps = 16;          // upper bound of warps per block (the launcher uses 4)
 constexpr int kLnMaxBlocksPerLane = 8;   // 8 x 32 lanes x 16 elements = 4096
 
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
-}
-
 // One row (bytes, a multiple of 16, 16-byte aligned on both sides) global -> shared, completing on `bar`.
 __device__ __forceinline__ void bulk_load_row(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
