@@ -238,36 +238,36 @@ sol_status_t nvfp4_layernorm_quantize(const void *x_bf16, int64_t M, int64_t K, 
  * Scaled-dot-product attention of a DiT block in BF16 (the rollout models of Section 4.1 are
  * diffusion transformers; the method quantizes their linear layers, Section 3, and leaves attention
  * in BF16 in the FP4 and in the BF16 path alike):
- *     out[b, s, h, :] = sum_t softmax_t( q[b,s,h,:] . k[b,t,h,:] / sqrt(128) ) v[b,t,h,:]
- * No mask, no dropout, head dimension 128.  Scores and sums in FP32, probabilities rounded to BF16
+ *     out[b, s, h, :] = sum_t softmax_t( q[b,s,h,:] . k[b,t,h,:] / sqrt(head_dim) ) v[b,t,h,:]
+ * No mask, no dropout; head_dim is 128 (FLUX.1) or 64 (SD3.5).  Scores and sums in FP32, probabilities rounded to BF16
  * before the product with V, output rounded to BF16.
- *   q, out   [batch, seq_q, heads, 128] BF16: element (b, s, h, d) at ((b * seq_q + s) * ld + h * 128 + d),
- *            ld_q / ld_out elements between consecutive tokens (>= heads * 128, multiple of 8), so q, k
+ *   q, out   [batch, seq_q, heads, head_dim] BF16: element (b, s, h, d) at ((b * seq_q + s) * ld + h * head_dim + d),
+ *            ld_q / ld_out elements between consecutive tokens (>= heads * head_dim, multiple of 8), so q, k
  *            and v may be column slices of one fused projection output
- *   k, v     [batch, seq_kv, heads, 128] BF16, the same way with ld_k / ld_v
+ *   k, v     [batch, seq_kv, heads, head_dim] BF16, the same way with ld_k / ld_v
  * All pointers are device pointers, 16-byte aligned, owned by the caller; out must not alias an input.
- * Errors: SOL_ERR_NULL_POINTER, SOL_ERR_BAD_SHAPE (a non-positive extent, ld < heads * 128, heads or batch
- * above 65535), SOL_ERR_ALIGNMENT, SOL_ERR_UNSUPPORTED_ARCH, SOL_ERR_CUDA; nothing is launched on an error.
+ * Errors: SOL_ERR_NULL_POINTER, SOL_ERR_BAD_SHAPE (a non-positive extent, another head_dim, ld < heads * head_dim,
+ * heads or batch above 65535), SOL_ERR_ALIGNMENT, SOL_ERR_UNSUPPORTED_ARCH, SOL_ERR_CUDA; nothing is launched on an error.
  */
 sol_status_t sol_attention_bf16(const void *q, const void *k, const void *v, void *out, int64_t batch, int64_t seq_q,
-                                int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v, int64_t ld_out,
-                                void *stream);
+                                int64_t seq_kv, int64_t heads, int64_t head_dim, int64_t ld_q, int64_t ld_k, int64_t ld_v,
+                                int64_t ld_out, void *stream);
 
 /*
  * sol_attention_bf16 whose output leaves as the quantized activations of the linear that follows it in
  * a DiT block (the output projection; in a single-stream block the concatenated input it shares
  * with the MLP branch): h = bf16(attention output), then nvfp4_quantize's mapping with
- * T = *out_tscale, written into columns [dest_col0, dest_col0 + heads * 128) of the NVFP4 tensor
+ * T = *out_tscale, written into columns [dest_col0, dest_col0 + heads * head_dim) of the NVFP4 tensor
  * [batch * seq_q, dest_K] (rows of all samples stacked; chunked scale layout).  Bit for bit what
  * sol_attention_bf16 followed by nvfp4_quantize_into produces, without the BF16 round trip through HBM.
  *   out_tscale   caller supplied (a delayed scale); amax_out: nullable running max|h| as in
  *                nvfp4_linear_quantized_out
- *   dest_K % 64 == 0, dest_col0 % 64 == 0, dest_col0 + heads * 128 <= dest_K
+ *   dest_K % 64 == 0, dest_col0 % 64 == 0, dest_col0 + heads * head_dim <= dest_K
  * Bytes outside the column range are not touched, so the rows past batch * seq_q of the destination's
  * last 128-row scale chunk must have been zeroed once.  Everything else as sol_attention_bf16.
  */
 sol_status_t sol_attention_nvfp4_out(const void *q, const void *k, const void *v, int64_t batch, int64_t seq_q,
-                                     int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v,
+                                     int64_t seq_kv, int64_t heads, int64_t head_dim, int64_t ld_q, int64_t ld_k, int64_t ld_v,
                                      const float *out_tscale, void *q_dest, void *sf_dest, int64_t dest_K,
                                      int64_t dest_col0, float *amax_out, void *stream);
 
@@ -288,7 +288,7 @@ typedef struct {
     int64_t seq, ld_q, ld_k, ld_v, ld_out;
 } sol_attention_stream_t;
 sol_status_t sol_attention_bf16_joint(const sol_attention_stream_t *first, const sol_attention_stream_t *second,
-                                      int64_t batch, int64_t heads, void *stream);
+                                      int64_t batch, int64_t heads, int64_t head_dim, void *stream);
 
 /*
  * BF16 linear, the full-precision stage-2 reference (Section 3.4):

@@ -93,13 +93,13 @@ def lib() -> ctypes.CDLL:
     L.nvfp4_quantize_linear_delayed.argtypes = [vp, i64, vp, vp, vp, vp, vp, i64, i64, i64, i64, vp, vp, sz, vp]
     L.sol_roll_tensor_scale.restype, L.sol_roll_tensor_scale.argtypes = i32, [vp, vp]
     L.sol_attention_bf16_joint.restype = i32
-    L.sol_attention_bf16_joint.argtypes = [ctypes.POINTER(AttentionStream), ctypes.POINTER(AttentionStream), i64, i64, vp]
+    L.sol_attention_bf16_joint.argtypes = [ctypes.POINTER(AttentionStream), ctypes.POINTER(AttentionStream), i64, i64, i64, vp]
     L.mxfp4_linear_quantized_out.restype = i32
     L.mxfp4_linear_quantized_out.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, vp, i64, i64, i64, vp]
     L.sol_attention_nvfp4_out.restype = i32
-    L.sol_attention_nvfp4_out.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, vp, vp, vp, i64, i64, vp, vp]
+    L.sol_attention_nvfp4_out.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, vp, vp, vp, i64, i64, vp, vp]
     L.sol_attention_bf16.restype = i32
-    L.sol_attention_bf16.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, vp]
+    L.sol_attention_bf16.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, i64, vp]
     L.nvfp4_layernorm_quantize.restype = i32
     L.nvfp4_layernorm_quantize.argtypes = [vp, i64, i64, i64, vp, vp, i64, ctypes.c_float, vp, vp, vp, vp, vp]
     L.sol_last_device_status.restype = i32
@@ -336,16 +336,16 @@ class AttentionStream(ctypes.Structure):
 
 
 def _token_pitch(t: torch.Tensor) -> int:
-    """Elements between consecutive tokens of a [B, S, H, 128] view (a dimension of extent 1 has no meaningful stride)."""
+    """Elements between consecutive tokens of a [B, S, H, D] view (a dimension of extent 1 has no meaningful stride)."""
     if t.shape[1] > 1:
         return t.stride(1)
-    return t.stride(0) if t.shape[0] > 1 else t.shape[2] * 128
+    return t.stride(0) if t.shape[0] > 1 else t.shape[2] * t.shape[3]
 
 
 def _check_attention_view(name: str, t: torch.Tensor):
-    if t.dtype != torch.bfloat16 or t.dim() != 4 or t.shape[3] != 128:
-        raise ValueError(f"{name} must be a [B, S, H, 128] BF16 tensor")
-    if t.stride(3) != 1 or (t.shape[2] > 1 and t.stride(2) != 128) or \
+    if t.dtype != torch.bfloat16 or t.dim() != 4 or t.shape[3] not in (64, 128):
+        raise ValueError(f"{name} must be a [B, S, H, D] BF16 tensor with D = 64 or 128")
+    if t.stride(3) != 1 or (t.shape[2] > 1 and t.stride(2) != t.shape[3]) or \
             (t.shape[0] > 1 and t.shape[1] > 1 and t.stride(0) != t.shape[1] * t.stride(1)):
         raise ValueError(f"{name}: heads and head dimension must be contiguous, batches stacked densely")
 
@@ -353,8 +353,8 @@ def _check_attention_view(name: str, t: torch.Tensor):
 def sol_attention_bf16_joint(first, second, out=None):
     """Joint attention of two token streams: first = (q, k, v) of the stream whose tokens come first.
 
-    Every tensor is a [B, S_stream, H, 128] view as in sol_attention_bf16; S of the first stream is a
-    multiple of 256.  Returns (out_first, out_second), each [B, S_stream, H, 128].
+    Every tensor is a [B, S_stream, H, D] view as in sol_attention_bf16; S of the first stream is a
+    multiple of 256.  Returns (out_first, out_second), each [B, S_stream, H, D].
     """
     streams = []
     outs = list(out) if out is not None else [None, None]
@@ -368,49 +368,49 @@ def sol_attention_bf16_joint(first, second, out=None):
         _check_attention_view("out", outs[i])
         streams.append(AttentionStream(_ptr(q), _ptr(k), _ptr(v), _ptr(outs[i]), q.shape[1], _token_pitch(q),
                                        _token_pitch(k), _token_pitch(v), _token_pitch(outs[i])))
-    B_, _, H, _ = first[0].shape
-    if second[0].shape[0] != B_ or second[0].shape[2] != H:
-        raise ValueError("both streams must share batch and heads")
-    _check(lib().sol_attention_bf16_joint(ctypes.byref(streams[0]), ctypes.byref(streams[1]), B_, H, _stream()),
+    B_, _, H, D = first[0].shape
+    if second[0].shape[0] != B_ or second[0].shape[2] != H or second[0].shape[3] != D:
+        raise ValueError("both streams must share batch, heads and head dimension")
+    _check(lib().sol_attention_bf16_joint(ctypes.byref(streams[0]), ctypes.byref(streams[1]), B_, H, D, _stream()),
            "sol_attention_bf16_joint")
     return outs[0], outs[1]
 
 
 def sol_attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: torch.Tensor | None = None):
-    """softmax(q k^T / sqrt(128)) v per batch element and head.
+    """softmax(q k^T / sqrt(D)) v per batch element and head, D = 64 or 128.
 
-    q [B, Sq, H, 128], k and v [B, Skv, H, 128], BF16; the last two dimensions contiguous, the batch
+    q [B, Sq, H, D], k and v [B, Skv, H, D], BF16; the last two dimensions contiguous, the batch
     dimension densely on top of the token dimension (stride(0) == S * stride(1)) -- views into a fused
-    projection output qualify.  Returns [B, Sq, H, 128].
+    projection output qualify.  Returns [B, Sq, H, D].
     """
     for name, t in (("q", q), ("k", k), ("v", v)):
         _check_attention_view(name, t)
-    B, Sq, H, _ = q.shape
-    if k.shape != v.shape or k.shape[0] != B or k.shape[2] != H:
-        raise ValueError("k and v must share [B, Skv, H, 128] with q's batch and heads")
+    B, Sq, H, D = q.shape
+    if k.shape != v.shape or k.shape[0] != B or k.shape[2] != H or k.shape[3] != D:
+        raise ValueError("k and v must share [B, Skv, H, D] with q's batch, heads and head dimension")
     if out is None:
-        out = torch.empty((B, Sq, H, 128), dtype=torch.bfloat16, device=q.device)
+        out = torch.empty((B, Sq, H, D), dtype=torch.bfloat16, device=q.device)
     _check_attention_view("out", out)
-    _check(lib().sol_attention_bf16(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, Sq, k.shape[1], H, _token_pitch(q),
+    _check(lib().sol_attention_bf16(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, Sq, k.shape[1], H, D, _token_pitch(q),
                                     _token_pitch(k), _token_pitch(v), _token_pitch(out), _stream()), "sol_attention_bf16")
     return out
 
 
 def sol_attention_nvfp4_out(q, k, v, out_tscale: torch.Tensor, dest, dest_col0: int = 0,
                             amax_out: torch.Tensor | None = None):
-    """Attention whose output is quantized into columns [dest_col0, dest_col0 + H * 128) of `dest`.
+    """Attention whose output is quantized into columns [dest_col0, dest_col0 + H * D) of `dest`.
 
     dest = (nibbles [B * Sq, dest_K / 2] uint8, swizzled scales of a [B * Sq, dest_K] tensor); returns dest.
     """
     for name, t in (("q", q), ("k", k), ("v", v)):
         _check_attention_view(name, t)
-    B, Sq, H, _ = q.shape
-    if k.shape != v.shape or k.shape[0] != B or k.shape[2] != H:
-        raise ValueError("k and v must share [B, Skv, H, 128] with q's batch and heads")
+    B, Sq, H, D = q.shape
+    if k.shape != v.shape or k.shape[0] != B or k.shape[2] != H or k.shape[3] != D:
+        raise ValueError("k and v must share [B, Skv, H, D] with q's batch, heads and head dimension")
     dq, dsf = dest
     if dq.dtype != torch.uint8 or dq.dim() != 2 or dq.shape[0] != B * Sq or not dq.is_contiguous():
         raise ValueError("dest nibbles must be a contiguous [B * Sq, dest_K / 2] uint8 tensor")
-    _check(lib().sol_attention_nvfp4_out(_ptr(q), _ptr(k), _ptr(v), B, Sq, k.shape[1], H, _token_pitch(q), _token_pitch(k),
+    _check(lib().sol_attention_nvfp4_out(_ptr(q), _ptr(k), _ptr(v), B, Sq, k.shape[1], H, D, _token_pitch(q), _token_pitch(k),
                                          _token_pitch(v), _ptr(out_tscale), _ptr(dq), _ptr(dsf), dq.shape[1] * 2, dest_col0,
                                          _ptr(amax_out), _stream()), "sol_attention_nvfp4_out")
     return dest

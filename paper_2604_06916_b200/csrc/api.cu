@@ -498,10 +498,11 @@ sol_status_t nvfp4_layernorm_quantize(const void *x_bf16, int64_t M, int64_t K, 
 }
 
 sol_status_t sol_attention_bf16(const void *q, const void *k, const void *v, void *out, int64_t batch, int64_t seq_q,
-                                int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v, int64_t ld_out,
-                                void *stream) {
+                                int64_t seq_kv, int64_t heads, int64_t head_dim, int64_t ld_q, int64_t ld_k, int64_t ld_v,
+                                int64_t ld_out, void *stream) {
     if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return SOL_ERR_NULL_POINTER;
-    const int64_t cols = heads * 128;
+    if (head_dim != 64 && head_dim != 128) return SOL_ERR_BAD_SHAPE;
+    const int64_t cols = heads * head_dim;
     if (batch <= 0 || seq_q <= 0 || seq_kv <= 0 || heads <= 0 || batch > 65535 || heads > 65535 ||
         seq_q > (1LL << 24) || seq_kv > (1LL << 24) || ld_q < cols || ld_k < cols || ld_v < cols || ld_out < cols)
         return SOL_ERR_BAD_SHAPE;
@@ -512,16 +513,17 @@ sol_status_t sol_attention_bf16(const void *q, const void *k, const void *v, voi
     sol_status_t st = check_arch(&dev);
     if (st != SOL_OK) return st;
     const attn::Stream b{q, k, v, out, seq_q, seq_kv, ld_q, ld_k, ld_v, ld_out};
-    return attn::launch_attention(nullptr, b, batch, heads, nullptr, static_cast<cudaStream_t>(stream));
+    return attn::launch_attention(nullptr, b, batch, heads, head_dim, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 sol_status_t sol_attention_nvfp4_out(const void *q, const void *k, const void *v, int64_t batch, int64_t seq_q,
-                                     int64_t seq_kv, int64_t heads, int64_t ld_q, int64_t ld_k, int64_t ld_v,
+                                     int64_t seq_kv, int64_t heads, int64_t head_dim, int64_t ld_q, int64_t ld_k, int64_t ld_v,
                                      const float *out_tscale, void *q_dest, void *sf_dest, int64_t dest_K,
                                      int64_t dest_col0, float *amax_out, void *stream) {
     if (q == nullptr || k == nullptr || v == nullptr || out_tscale == nullptr || q_dest == nullptr || sf_dest == nullptr)
         return SOL_ERR_NULL_POINTER;
-    const int64_t cols = heads * 128;
+    if (head_dim != 64 && head_dim != 128) return SOL_ERR_BAD_SHAPE;
+    const int64_t cols = heads * head_dim;
     if (batch <= 0 || seq_q <= 0 || seq_kv <= 0 || heads <= 0 || batch > 65535 || heads > 65535 ||
         seq_q > (1LL << 24) || seq_kv > (1LL << 24) || ld_q < cols || ld_k < cols || ld_v < cols || dest_K <= 0 ||
         dest_K % 64 != 0 || dest_col0 < 0 || dest_col0 % 64 != 0 || dest_col0 + cols > dest_K || dest_K > (1LL << 24) ||
@@ -536,14 +538,15 @@ sol_status_t sol_attention_nvfp4_out(const void *q, const void *k, const void *v
     if (st != SOL_OK) return st;
     const attn::Stream b{q, k, v, nullptr, seq_q, seq_kv, ld_q, ld_k, ld_v, cols};
     const attn::QuantDest qd{q_dest, sf_dest, out_tscale, reinterpret_cast<uint32_t *>(amax_out), dest_K, dest_col0};
-    return attn::launch_attention(nullptr, b, batch, heads, &qd, static_cast<cudaStream_t>(stream));
+    return attn::launch_attention(nullptr, b, batch, heads, head_dim, &qd, static_cast<cudaStream_t>(stream));
 }
 
 sol_status_t sol_attention_bf16_joint(const sol_attention_stream_t *first, const sol_attention_stream_t *second,
-                                      int64_t batch, int64_t heads, void *stream) {
+                                      int64_t batch, int64_t heads, int64_t head_dim, void *stream) {
     if (first == nullptr || second == nullptr) return SOL_ERR_NULL_POINTER;
+    if (head_dim != 64 && head_dim != 128) return SOL_ERR_BAD_SHAPE;
     const sol_attention_stream_t *both[2] = {first, second};
-    const int64_t cols = heads * 128;
+    const int64_t cols = heads * head_dim;
     if (batch <= 0 || heads <= 0 || batch > 65535 || heads > 65535) return SOL_ERR_BAD_SHAPE;
     for (const sol_attention_stream_t *s : both) {
         if (s->q == nullptr || s->k == nullptr || s->v == nullptr || s->out == nullptr) return SOL_ERR_NULL_POINTER;
@@ -561,7 +564,7 @@ sol_status_t sol_attention_bf16_joint(const sol_attention_stream_t *first, const
                          first->ld_q, first->ld_k, first->ld_v, first->ld_out};
     const attn::Stream b{second->q, second->k, second->v, second->out, second->seq, second->seq,
                          second->ld_q, second->ld_k, second->ld_v, second->ld_out};
-    return attn::launch_attention(&a, b, batch, heads, nullptr, static_cast<cudaStream_t>(stream));
+    return attn::launch_attention(&a, b, batch, heads, head_dim, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 sol_status_t nvfp4_quantize_linear(const void *x_bf16, int64_t ldx, const void *wq, const void *wsf,

@@ -30,19 +30,17 @@ namespace {
 
 using gemm::wait_bounded;
 
-constexpr int kD = 128;                 // head dimension
 constexpr int kBQ = 128;                // query rows per query tile
 constexpr int kQTiles = 2;              // query tiles per CTA
 constexpr int kBKV = 128;               // keys per tile
 constexpr int kBox = 128 * 128;         // bytes of a [128 rows][64 BF16] box
-constexpr int kTile = 2 * kBox;         // a [128][128] BF16 tile: box of columns 0..63, box of 64..127
 constexpr int kStages = 2;              // K ring and V ring
 constexpr int kThreads = 32 * (2 + 4 * kQTiles);
 constexpr float kLazyLog2 = 8.0f;       // slack of the softmax reference maximum, in powers of two
-constexpr int kSmem = (kQTiles + 2 * kStages) * kTile + 256;
+constexpr int smem_bytes(int head_dim) { return (kQTiles + 2 * kStages) * (head_dim / 64) * kBox + 256; }
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 128, kColTile = 256;   // per query tile; P overwrites columns [0, 64) of S
-static_assert(kSmem <= 232448, "shared memory budget");
+static_assert(smem_bytes(128) <= 232448, "shared memory budget");
 
 #ifdef SOL_TUNING
 __device__ long long g_attn_trace[12][64];
@@ -82,14 +80,17 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// kD: head dimension, 64 or 128 (a tile of kD columns is kD / 64 boxes of [128 rows][64 BF16]).
 // kQuantOut: the output leaves as the next linear's NVFP4 activations (h = bf16(O / l), then the
 // quantizer's FP32 sequence per 16 columns) instead of BF16 -- one stream only.
-template <bool kQuantOut>
+template <int kD, bool kQuantOut>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constant__ CUtensorMap tm_ka,
                  const __grid_constant__ CUtensorMap tm_va, const __grid_constant__ CUtensorMap tm_oa,
                  const __grid_constant__ CUtensorMap tm_qb, const __grid_constant__ CUtensorMap tm_kb,
                  const __grid_constant__ CUtensorMap tm_vb, const __grid_constant__ CUtensorMap tm_ob, const Params p) {
+    constexpr int kBoxes = kD / 64;
+    constexpr int kTile = kBoxes * kBox;    // bytes of a [128][kD] BF16 tile
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t smem_base = ptx::smem_u32(smem_raw);
     if (smem_base & 1023u) {  // the swizzled operand layout needs 1024-byte alignment
@@ -143,8 +144,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
             ptx::mbar_arrive_expect_tx(bar(kQFull), kQTiles * kTile);
 #pragma unroll
             for (int t = 0; t < kQTiles; ++t) {
-                ptx::tma_load_3d(sQ + t * kTile, tm_q, x0, q0 + t * kBQ, batch, bar(kQFull));
-                ptx::tma_load_3d(sQ + t * kTile + kBox, tm_q, x0 + 64, q0 + t * kBQ, batch, bar(kQFull));
+#pragma unroll
+                for (int bx = 0; bx < kBoxes; ++bx)
+                    ptx::tma_load_3d(sQ + t * kTile + bx * kBox, tm_q, x0 + 64 * bx, q0 + t * kBQ, batch, bar(kQFull));
             }
             for (int j = 0; j < n_tiles; ++j) {
                 const int st = j & 1;
@@ -157,26 +159,28 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
                 const int kv0 = kv_in_a ? j * kBKV : j * kBKV - p.kv_split;
                 const CUtensorMap *tm_k = kv_in_a ? &tm_ka : &tm_kb;
                 const CUtensorMap *tm_v = kv_in_a ? &tm_va : &tm_vb;
-                ptx::tma_load_3d(sK + st * kTile, tm_k, x0, kv0, batch, bar(kKFull + st));
-                ptx::tma_load_3d(sK + st * kTile + kBox, tm_k, x0 + 64, kv0, batch, bar(kKFull + st));
+#pragma unroll
+                for (int bx = 0; bx < kBoxes; ++bx)
+                    ptx::tma_load_3d(sK + st * kTile + bx * kBox, tm_k, x0 + 64 * bx, kv0, batch, bar(kKFull + st));
                 if (!wait_bounded(bar(kVEmpty + st), par ^ 1u, abort_flag, p.status, 0xB20u | st)) break;
                 ATTN_TRACE(11, j);
                 ptx::mbar_arrive_expect_tx(bar(kVFull + st), kTile);
-                ptx::tma_load_3d(sV + st * kTile, tm_v, x0, kv0, batch, bar(kVFull + st));
-                ptx::tma_load_3d(sV + st * kTile + kBox, tm_v, x0 + 64, kv0, batch, bar(kVFull + st));
+#pragma unroll
+                for (int bx = 0; bx < kBoxes; ++bx)
+                    ptx::tma_load_3d(sV + st * kTile + bx * kBox, tm_v, x0 + 64 * bx, kv0, batch, bar(kVFull + st));
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (ptx::elect_one()) {
-            // BF16 x BF16 -> FP32, M = 128, N = 128; bit 16: B is MN-major (V)
-            const uint32_t idesc_qk = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(128 >> 3) << 17) |
-                                      (static_cast<uint32_t>(128 >> 4) << 24);
-            const uint32_t idesc_pv = idesc_qk | (1u << 16);
+            // BF16 x BF16 -> FP32, M = 128; scores N = 128 keys, output N = kD with B MN-major (bit 16: V is [kv][d])
+            const uint32_t idesc_base = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(128 >> 4) << 24);
+            const uint32_t idesc_qk = idesc_base | (static_cast<uint32_t>(kBKV >> 3) << 17);
+            const uint32_t idesc_pv = idesc_base | (static_cast<uint32_t>(kD >> 3) << 17) | (1u << 16);
             auto issue_qk = [&](int t, int st) {  // S_t = Q_t K^T, 16 elements of d per instruction
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+                for (int i = 0; i < kD / 16; ++i) {
                     const uint64_t a = ptx::smem_desc_sw128(sQ + t * kTile + (i >> 2) * kBox) + 2u * (i & 3);
                     const uint64_t b = ptx::smem_desc_sw128(sK + st * kTile + (i >> 2) * kBox) + 2u * (i & 3);
                     ptx::mma_bf16(tmem_base + t * kColTile + kColS, a, b, idesc_qk, i > 0);
@@ -301,7 +305,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
             if (tracer) ATTN_TRACE(7, j);
             if (j > 0 && __any_sync(0xFFFFFFFFu, move)) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < kD / 32; ++c) {
                     uint32_t o[32];
                     ptx::tmem_ld_32x32(t_lane + kColO + 32 * c, o);
                     ptx::tmem_ld_wait();
@@ -324,7 +328,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
             ptx::tc_fence_after_sync();
             const float inv = 1.0f / l;
             if constexpr (kQuantOut) {
-                // thread = row: 128 columns of one head = eight 16-element blocks, quantized from registers
+                // thread = row: the kD columns of one head are whole 16-element blocks, quantized from registers
                 const int row = q0 + t * kBQ + r;
                 const bool row_ok = row < q_rows;
                 const int64_t m = static_cast<int64_t>(batch) * p.seq_q + row;
@@ -332,10 +336,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
                 const float c6T = __fmul_rn(6.0f, T);
                 const int col0 = p.dest_col0 + head * kD;
                 uint8_t *qrow = p.q_dest + m * p.dest_pitch + (col0 >> 1);
-                uint32_t amax2 = 0, sfw[2] = {0u, 0u};
-                uint32_t codes[16];  // the row's 128 nibbles: stored in one go so that its two 32-byte sectors fill at once
+                uint32_t amax2 = 0, sfw[kD / 64] = {};
+                uint32_t codes[kD / 8];  // the row's nibbles: stored in one go so that its 32-byte sectors fill at once
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < kD / 32; ++c) {
                     uint32_t o[32];
                     ptx::tmem_ld_32x32(t_lane + kColO + 32 * c, o);
                     ptx::tmem_ld_wait();
@@ -361,12 +365,12 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
                 }
                 if (row_ok) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
+                    for (int c = 0; c < kD / 32; ++c)
                         *reinterpret_cast<uint4 *>(qrow + 16 * c) = make_uint4(codes[4 * c], codes[4 * c + 1], codes[4 * c + 2], codes[4 * c + 3]);
                 }
                 if (row_ok) {
 #pragma unroll
-                    for (int kc = 0; kc < 2; ++kc) {  // the four scale bytes of a (row, 64-column chunk) slot are one word
+                    for (int kc = 0; kc < kD / 64; ++kc) {  // the four scale bytes of a (row, 64-column chunk) slot are one word
                         const int64_t chunk = (m >> 7) * p.dest_chunks_k + (col0 >> 6) + kc;
                         *reinterpret_cast<uint32_t *>(p.sf_dest + chunk * 512 + (m & 31) * 16 + ((m & 127) >> 5) * 4) = sfw[kc];
                     }
@@ -380,7 +384,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
             } else {
             const uint32_t o_row = sQ + t * kTile + r * 128;  // Q_t is no longer read: its MMAs have completed
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < kD / 32; ++c) {
                 uint32_t o[32];
                 ptx::tmem_ld_32x32(t_lane + kColO + 32 * c, o);
                 ptx::tmem_ld_wait();
@@ -397,9 +401,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
             ptx::fence_proxy_async_smem();
             __syncwarp();
             const int row0 = q0 + t * kBQ + quad * 32;
-            if (lane == 0 && row0 < q_rows) {  // this warp's 32 rows, two boxes of 64 columns (clipped at the end of the stream)
-                ptx::tma_store_3d(tm_o, head * kD, row0, batch, sQ + t * kTile + quad * 32 * 128);
-                ptx::tma_store_3d(tm_o, head * kD + 64, row0, batch, sQ + t * kTile + kBox + quad * 32 * 128);
+            if (lane == 0 && row0 < q_rows) {  // this warp's 32 rows, boxes of 64 columns (clipped at the end of the stream)
+#pragma unroll
+                for (int bx = 0; bx < kBoxes; ++bx)
+                    ptx::tma_store_3d(tm_o, head * kD + 64 * bx, row0, batch, sQ + t * kTile + bx * kBox + quad * 32 * 128);
                 ptx::tma_store_commit();
                 ptx::tma_store_wait_all<0>();
             }
@@ -418,10 +423,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
 
 }  // namespace
 
-sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, const QuantDest *qd,
-                              cudaStream_t stream) {
+sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, int64_t head_dim,
+                              const QuantDest *qd, cudaStream_t stream) {
     CUtensorMap tm[8];
-    const uint64_t cols = static_cast<uint64_t>(heads) * kD;
+    const uint64_t cols = static_cast<uint64_t>(heads) * static_cast<uint64_t>(head_dim);
     auto make = [&](CUtensorMap *t, const void *base, int64_t seq, int64_t ld, uint32_t box_rows) {
         return make_tmap_3d_bf16(t, base, cols, static_cast<uint64_t>(seq), static_cast<uint64_t>(batch),
                                  static_cast<uint64_t>(ld) * 2, static_cast<uint64_t>(seq) * ld * 2, 64, box_rows);
@@ -438,7 +443,7 @@ sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, i
     p.kv_split = a != nullptr ? static_cast<int>(a->seq_kv) : 0;
     p.seq_q = p.q_split + static_cast<int>(b.seq_q);
     p.seq_kv = p.kv_split + static_cast<int>(b.seq_kv);
-    p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(kD));
+    p.scale_log2 = 1.4426950408889634f / sqrtf(static_cast<float>(head_dim));
     p.status = device_status_word();
     if (qd != nullptr) {
         p.q_dest = static_cast<uint8_t *>(qd->q);
@@ -449,18 +454,22 @@ sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, i
         p.dest_col0 = static_cast<int>(qd->dest_col0);
         p.dest_chunks_k = static_cast<int>(qd->dest_K / 64);
     }
-    auto kern = qd != nullptr ? attention_kernel<true> : attention_kernel<false>;
-    static bool configured[2][64] = {};
+    const bool quant = qd != nullptr, wide = head_dim == 128;
+    auto kern = wide ? (quant ? attention_kernel<128, true> : attention_kernel<128, false>)
+                     : (quant ? attention_kernel<64, true> : attention_kernel<64, false>);
+    const int smem = smem_bytes(static_cast<int>(head_dim));
+    static bool configured[4][64] = {};
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SOL_ERR_CUDA;
-    if (!configured[qd != nullptr][dev]) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess)
+    const int slot = (wide ? 2 : 0) + (quant ? 1 : 0);
+    if (!configured[slot][dev]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return SOL_ERR_CUDA;
-        configured[qd != nullptr][dev] = true;
+        configured[slot][dev] = true;
     }
     const dim3 grid(static_cast<unsigned>((p.seq_q + kQTiles * kBQ - 1) / (kQTiles * kBQ)), static_cast<unsigned>(heads),
                     static_cast<unsigned>(batch));
-    kern<<<grid, kThreads, kSmem, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], tm[7], p);
+    kern<<<grid, kThreads, smem, stream>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], tm[6], tm[7], p);
     return launch_status();
 }
 

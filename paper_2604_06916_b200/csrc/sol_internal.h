@@ -114,12 +114,12 @@ bool make_tmap_3d_bf16(CUtensorMap *out, const void *base, uint64_t d0, uint64_t
                        uint64_t pitch2_bytes, uint32_t box0, uint32_t box1);
 
 namespace attn {
-struct Stream {   // one token stream of an attention call: [batch, seq, heads, 128] views with token pitches
+struct Stream {   // one token stream of an attention call: [batch, seq, heads, head_dim] views with token pitches
     const void *q, *k, *v;
     void *out;
     int64_t seq_q, seq_kv, ld_q, ld_k, ld_v, ld_out;
 };
-struct QuantDest {   // NVFP4 destination of the output: columns [dest_col0, dest_col0 + heads * 128) of a [rows, dest_K] tensor
+struct QuantDest {   // NVFP4 destination of the output: columns [dest_col0, dest_col0 + heads * head_dim) of a [rows, dest_K] tensor
     void *q, *sf;
     const float *tscale;
     uint32_t *amax_out;
@@ -127,8 +127,8 @@ struct QuantDest {   // NVFP4 destination of the output: columns [dest_col0, des
 };
 // Attention over the concatenation (a, then b) of two token streams, or over b alone when a is null;
 // with `qd` (one stream only) the output is quantized into `qd` instead of written as BF16.
-sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, const QuantDest *qd,
-                              cudaStream_t stream);
+sol_status_t launch_attention(const Stream *a, const Stream &b, int64_t batch, int64_t heads, int64_t head_dim,
+                              const QuantDest *qd, cudaStream_t stream);
 }
 
 // Scale-factor buffer in the chunked layout as a 3-D tensor [row chunk][k chunk][128 x u32]; the box

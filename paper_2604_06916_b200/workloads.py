@@ -142,23 +142,23 @@ def make_lora(N: int, K: int, seed: int, device="cpu", rank: int = LORA_RANK):
     return A, B
 
 
-def make_qkv(batch: int, seq: int, heads: int, seed: int, device="cpu", q_gain: float = 1.0):
-    """One fused projection output [batch, seq, 3 * heads * 128] in BF16 and its q, k, v views.
+def make_qkv(batch: int, seq: int, heads: int, seed: int, device="cpu", q_gain: float = 1.0, head_dim: int = 128):
+    """One fused projection output [batch, seq, 3 * heads * head_dim] in BF16 and its q, k, v views.
 
     q and k are unit normal per element (the models named in Section 4.1 RMS-normalise both per head
     before attention, so q.k / sqrt(d) has unit variance); v is normal with standard deviation 0.5.
-    `q_gain` > 1 sharpens the softmax.  The views are [batch, seq, heads, 128] with a token pitch of
-    3 * heads * 128 elements, as attention sees them after a fused q/k/v linear.
+    `q_gain` > 1 sharpens the softmax.  The views are [batch, seq, heads, head_dim] with a token pitch of
+    3 * heads * head_dim elements, as attention sees them after a fused q/k/v linear.
     """
     g = torch.Generator(device=device).manual_seed(7000 + seed)
-    width = heads * 128
+    width = heads * head_dim
     fused = torch.empty((batch, seq, 3 * width), dtype=torch.bfloat16, device=device)
     for b in range(batch):
         z = torch.randn((seq, 3 * width), generator=g, device=device, dtype=torch.float32)
         z[:, :width] *= q_gain
         z[:, 2 * width:] *= 0.5
         fused[b] = z.to(torch.bfloat16)
-    q, k, v = (fused[:, :, i * width:(i + 1) * width].unflatten(2, (heads, 128)) for i in range(3))
+    q, k, v = (fused[:, :, i * width:(i + 1) * width].unflatten(2, (heads, head_dim)) for i in range(3))
     return fused, q, k, v
 
 

@@ -134,26 +134,27 @@ def test_argument_validation_happens_before_any_cuda_call(lib):
     assert L.nvfp4_layernorm_quantize(p, 4, 64, 64, p, p, 0, 1e-6, p, p, p, None, None) == SHAPE
     assert L.nvfp4_layernorm_quantize(p, 4, 64, 64, p + 8, p, 4, 1e-6, p, p, p, None, None) == ALIGN
     # attention
-    assert L.sol_attention_bf16(p, p, None, p, 1, 4, 4, 1, 128, 128, 128, 128, None) == NULLP
-    assert L.sol_attention_bf16(p, p, p, p, 1, 0, 4, 1, 128, 128, 128, 128, None) == SHAPE
-    assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 2, 128, 256, 256, 256, None) == SHAPE      # pitch < heads * 128
-    assert L.sol_attention_bf16(p, p, p, p, 70000, 4, 4, 1, 128, 128, 128, 128, None) == SHAPE
-    assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 1, 132, 128, 128, 128, None) == ALIGN      # pitch % 8
-    assert L.sol_attention_bf16(p, p + 8, p, p, 1, 4, 4, 1, 128, 128, 128, 128, None) == ALIGN
+    assert L.sol_attention_bf16(p, p, None, p, 1, 4, 4, 1, 128, 128, 128, 128, 128, None) == NULLP
+    assert L.sol_attention_bf16(p, p, p, p, 1, 0, 4, 1, 128, 128, 128, 128, 128, None) == SHAPE
+    assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 2, 128, 128, 256, 256, 256, None) == SHAPE      # pitch < heads * head_dim
+    assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 1, 96, 128, 128, 128, 128, None) == SHAPE       # head_dim
+    assert L.sol_attention_bf16(p, p, p, p, 70000, 4, 4, 1, 128, 128, 128, 128, 128, None) == SHAPE
+    assert L.sol_attention_bf16(p, p, p, p, 1, 4, 4, 1, 128, 132, 128, 128, 128, None) == ALIGN      # pitch % 8
+    assert L.sol_attention_bf16(p, p + 8, p, p, 1, 4, 4, 1, 128, 128, 128, 128, 128, None) == ALIGN
     assert L.mxfp4_linear_quantized_out(p, p, p, None, None, 0, p, p, None, 4, 128, 64, None) == NULLP
     assert L.mxfp4_linear_quantized_out(p, p, p, p, None, 0, p, p, None, 4, 192, 64, None) == SHAPE      # N % 128
     assert L.mxfp4_linear_quantized_out(p, p, p, p, None, 0, p + 8, p, None, 4, 128, 64, None) == ALIGN
-    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, None, p, p, 128, 0, None, None) == NULLP
-    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, p, p, p, 96, 0, None, None) == SHAPE     # dest_K % 64
-    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, p, p, p, 128, 64, None, None) == SHAPE   # past the end
-    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, p, p + 8, p, 128, 0, None, None) == ALIGN
+    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, 128, None, p, p, 128, 0, None, None) == NULLP
+    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, 128, p, p, p, 96, 0, None, None) == SHAPE     # dest_K % 64
+    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, 128, p, p, p, 128, 64, None, None) == SHAPE   # past the end
+    assert L.sol_attention_nvfp4_out(p, p, p, 1, 4, 4, 1, 128, 128, 128, 128, p, p + 8, p, 128, 0, None, None) == ALIGN
     from paper_2604_06916_b200.binding import AttentionStream
     ok = AttentionStream(p, p, p, p, 256, 128, 128, 128, 128)
-    assert L.sol_attention_bf16_joint(None, ctypes.byref(ok), 1, 1, None) == NULLP
-    assert L.sol_attention_bf16_joint(ctypes.byref(AttentionStream(p, None, p, p, 256, 128, 128, 128, 128)), ctypes.byref(ok), 1, 1, None) == NULLP
-    assert L.sol_attention_bf16_joint(ctypes.byref(AttentionStream(p, p, p, p, 200, 128, 128, 128, 128)), ctypes.byref(ok), 1, 1, None) == SHAPE  # first % 256
-    assert L.sol_attention_bf16_joint(ctypes.byref(ok), ctypes.byref(AttentionStream(p, p, p, p, 0, 128, 128, 128, 128)), 1, 1, None) == SHAPE
-    assert L.sol_attention_bf16_joint(ctypes.byref(ok), ctypes.byref(AttentionStream(p, p, p, p + 8, 5, 128, 128, 128, 128)), 1, 1, None) == ALIGN
+    assert L.sol_attention_bf16_joint(None, ctypes.byref(ok), 1, 1, 128, None) == NULLP
+    assert L.sol_attention_bf16_joint(ctypes.byref(AttentionStream(p, None, p, p, 256, 128, 128, 128, 128)), ctypes.byref(ok), 1, 1, 128, None) == NULLP
+    assert L.sol_attention_bf16_joint(ctypes.byref(AttentionStream(p, p, p, p, 200, 128, 128, 128, 128)), ctypes.byref(ok), 1, 1, 128, None) == SHAPE  # first % 256
+    assert L.sol_attention_bf16_joint(ctypes.byref(ok), ctypes.byref(AttentionStream(p, p, p, p, 0, 128, 128, 128, 128)), 1, 1, 128, None) == SHAPE
+    assert L.sol_attention_bf16_joint(ctypes.byref(ok), ctypes.byref(AttentionStream(p, p, p, p + 8, 5, 128, 128, 128, 128)), 1, 1, 128, None) == ALIGN
     # MXFP4
     assert L.sol_mxfp4_scale_bytes(256, 512, 0) == 256 * 16 and L.sol_mxfp4_scale_bytes(256, 512, 1) == 2 * 4 * 512
     assert L.sol_mxfp4_scale_bytes(130, 160, 1) == 2 * 2 * 512 and L.sol_mxfp4_scale_bytes(4, 48, 1) == 0

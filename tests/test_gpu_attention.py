@@ -1,4 +1,4 @@
-"""GPU parity: BF16 attention (head dimension 128) through the C ABI against the FP64 oracle.
+"""GPU parity: BF16 attention (head dimension 128 or 64) through the C ABI against the FP64 oracle.
 
 Tolerance (derived in oracle.attention.attention_tolerance): 2^-8 |O| + 2^-8 max|v| -- output
 rounding to BF16, probabilities rounded to BF16 before the product with V, row sum from the
@@ -158,3 +158,40 @@ def test_quantized_output_equals_attention_then_quantizer(B, batch, seq, heads, 
     tol = OA.attention_tolerance(ref.reshape(batch, seq, heads, 128), f64(v)).reshape(M, cols) + 1.01 * step.cpu().numpy() + 1e-30
     assert sub_q.shape == (M, cols // 2)
     assert np.all(np.abs(full.cpu().numpy().astype(np.float64) - ref) <= tol)
+
+
+@pytest.mark.parametrize("batch,seq_q,seq_kv,heads", [(1, 128, 128, 1), (2, 640, 640, 3), (2, 200, 333, 2), (1, 1, 1, 1),
+                                                       (1, 4096 + 154, 4096 + 154, 2)])
+def test_head_dimension_64(B, batch, seq_q, seq_kv, heads):
+    # the SD3.5 geometry: 64-wide heads (38 of them there; 4096 image + 154 text tokens at 1024 pixels)
+    _, q, _, _ = workloads.make_qkv(batch, seq_q, heads, 81, "cuda", head_dim=64)
+    _, _, k, v = workloads.make_qkv(batch, seq_kv, heads, 82, "cuda", head_dim=64)
+    if seq_q > 2048:   # the oracle on sampled query rows only
+        rows = [0, 127, 128, 255, 256, 2000, 4095, 4096, seq_q - 1]
+        check(B, q, k, v, rows=rows)
+    else:
+        check(B, q, k, v)
+
+
+def test_head_dimension_64_joint_and_quantized_output(B):
+    _, qa, ka, va = workloads.make_qkv(2, 256, 2, 83, "cuda", head_dim=64)
+    _, qb, kb, vb = workloads.make_qkv(2, 300, 2, 84, "cuda", head_dim=64)
+    oa, ob = B.sol_attention_bf16_joint((qa, ka, va), (qb, kb, vb))
+    q, k, v = (torch.cat((x, y), dim=1) for x, y in ((qa, qb), (ka, kb), (va, vb)))
+    whole = B.sol_attention_bf16(q, k, v)
+    assert torch.equal(torch.cat((oa, ob), dim=1), whole)
+    ref = OA.attention(f64(q), f64(k), f64(v))
+    assert np.all(np.abs(f64(whole) - ref) <= OA.attention_tolerance(ref, f64(v)))
+    # quantizing epilogue against the BF16 kernel followed by the slice quantizer, bit for bit
+    M, cols = 2 * 556, 2 * 64
+    o = whole.reshape(M, cols)
+    T = B.sol_amax_bf16(o)
+    def fresh():
+        return (torch.full((M, 192 // 2), 0x5A, dtype=torch.uint8, device="cuda"),
+                torch.zeros(B.scale_bytes(M, 192), dtype=torch.uint8, device="cuda"))
+    want, got = fresh(), fresh()
+    B.nvfp4_quantize_into(o, T, want, 64)
+    B.sol_attention_nvfp4_out(q, k, v, T, got, 64)
+    torch.cuda.synchronize()
+    assert B.sol_last_device_status() == 0
+    assert torch.equal(got[0], want[0]) and torch.equal(got[1], want[1])
