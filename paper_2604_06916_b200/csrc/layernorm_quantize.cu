@@ -128,9 +128,11 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
             w[i][0] = v0.x; w[i][1] = v0.y; w[i][2] = v0.z; w[i][3] = v0.w;
             w[i][4] = v1.x; w[i][5] = v1.y; w[i][6] = v1.z; w[i][7] = v1.w;
         }
+        // every lane orders its reads of the slot before the bulk copy that refills it (the copy writes
+        // through the async proxy, which an mbarrier or a warp barrier alone does not order behind generic reads)
+        ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0 && r + 2 * stride < last) {   // the slot is free again: fetch the row after next
-            ptx::fence_proxy_async_smem();
             ptx::mbar_arrive_expect_tx(bar0 + 8u * slot, row_bytes);
             bulk_load_row(ring + slot * row_bytes, x + (r + 2 * stride) * ld, row_bytes, bar0 + 8u * slot);
         }
