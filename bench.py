@@ -871,10 +871,12 @@ def run_only(args):
         sh = (torch.randn(M // rps, l0.K, generator=gen, device="cuda") * 0.2).to(torch.bfloat16)
         ts = torch.full((1,), 0.004, dtype=torch.float32, device="cuda")
         times = []
+        out = (torch.empty((M, l0.K // 2), dtype=torch.uint8, device="cuda"),
+               torch.empty(B.scale_bytes(M, l0.K), dtype=torch.uint8, device="cuda"))
         for it in range(args.warmup + args.steps):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            B.nvfp4_layernorm_quantize(X, sc, sh, rps, ts)
+            B.nvfp4_layernorm_quantize(X, sc, sh, rps, ts, out=out)
             e1.record()
             torch.cuda.synchronize()
             if it >= args.warmup:
