@@ -92,6 +92,14 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def rolled_scale(B, torch, amax):
+    """T for a running amax word, derived by the library's own kernel (sol_roll_tensor_scale)."""
+    state = torch.zeros(2, dtype=torch.float32, device=amax.device)
+    state[1:].copy_(amax)
+    B.sol_roll_tensor_scale(state)
+    return state[:1].clone()
+
+
 def flops_of(layers) -> float:
     return float(sum(2.0 * l.M * l.N * l.K for l in layers))
 
@@ -178,6 +186,73 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- GPU arm
+class LegTimer:
+    """Times named legs in long contiguous regions, rotated so that no leg always follows the same one.
+
+    A leg's region repeats its K-step block until the region has run for at least `min_s` seconds (the
+    GPU then sits in its power-capped steady state), with one CUDA event per block on the launching
+    stream; regions are bracketed by barrier + synchronize and the per-step time is the max over ranks.
+    Each of `rounds` rounds visits every leg once and starts at a different leg.
+    """
+
+    def __init__(self, torch, replicas, dev, dist, sampler, steps, min_s, rounds):
+        self.torch, self.replicas, self.dev, self.dist = torch, replicas, dev, dist
+        self.sampler, self.steps, self.min_s, self.rounds = sampler, steps, min_s, rounds
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def region(self, fn, blocks):
+        torch = self.torch
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(blocks + 1)]
+        self.barrier()
+        w0 = time.time()
+        ev[0].record()
+        for b in range(blocks):
+            for _ in range(self.steps):
+                fn()
+            ev[b + 1].record()
+        self.barrier()
+        w1 = time.time()
+        total_ms = ev[0].elapsed_time(ev[-1])
+        ms, _, _ = self.replicas.aggregate(total_ms / (blocks * self.steps), 1.0, self.dev)  # max over ranks
+        return ms, total_ms * 1e-3, (w0, w1)
+
+    def run(self, legs, warmup):
+        """legs: ordered {name: fn}.  Returns {name: {ms_per_step (mean over rounds), per_round, spread, blocks,
+        region_s, clocks}}."""
+        names = list(legs)
+        blocks = {}
+        for n in names:                       # warm-up, and the block count that makes a region >= min_s
+            for _ in range(warmup):
+                legs[n]()
+            ms, _, _ = self.region(legs[n], 1)
+            blocks[n] = max(1, int(self.min_s * 1e3 / (ms * self.steps)) + 1)
+        out = {n: {"per_round": [], "region_s": [], "windows": []} for n in names}
+        for rnd in range(self.rounds):
+            k = rnd % len(names)
+            for n in names[k:] + names[:k]:
+                ms, secs, win = self.region(legs[n], blocks[n])
+                out[n]["per_round"].append(ms)
+                out[n]["region_s"].append(secs)
+                out[n]["windows"].append(win)
+        for n in names:
+            r = out[n]
+            r["ms_per_step"] = sum(r["per_round"]) / len(r["per_round"])
+            r["spread"] = (max(r["per_round"]) - min(r["per_round"])) / r["ms_per_step"]
+            r["blocks"] = blocks[n]
+        return out
+
+
+def clock_normalised(flops, ms, sm_mhz, flop_per_clk_sm):
+    """Share of the tensor pipe's issue rate at the sampled clock: flops / (148 SM x flop/clk x f x t)."""
+    if not sm_mhz:
+        return None
+    return flops / (148.0 * flop_per_clk_sm * sm_mhz * 1e6 * ms * 1e-3)
+
+
 def run_ours(args):
     import torch
     from paper_2604_06916_b200 import binding as B
@@ -186,6 +261,10 @@ def run_ours(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world:
+        raise SystemExit(f"bench.py --gpus {args.gpus} needs {args.gpus} ranks but WORLD_SIZE is {world}: launch it as "
+                         f"`python -m torch.distributed.run --nnodes=1 --nproc-per-node {args.gpus} --master-addr 127.0.0.1 "
+                         f"--master-port <port> bench.py --gpus {args.gpus} ...` (independent replicas, one per GPU)")
     torch.cuda.set_device(local_rank)
     dist = None
     if world > 1:
@@ -197,54 +276,39 @@ def run_ours(args):
         int(args.workload.split("_g")[-1]))
     layers = cfg.layers
     dev = torch.device("cuda", local_rank)
+    warm = max(3, args.warmup)
+
+    def make_data(cfg_):
+        acts, data_ = {}, []
+        for i, l in enumerate(cfg_.layers):
+            X, W, bias = workloads.make_layer(cfg_, i, dev)
+            if l.K in acts:
+                X = acts[l.K]          # one activation tensor per distinct K (all larger than L2)
+            else:
+                acts[l.K] = X
+            wq, wsf, wts = B.nvfp4_quantize_weight(W)
+            Y = torch.empty((l.M, l.N), dtype=torch.bfloat16, device=dev)
+            ws = torch.empty(B.linear_workspace_bytes(l.M, l.N, l.K), dtype=torch.uint8, device=dev)
+            data_.append(dict(l=l, X=X, W=W, bias=bias, wq=wq, wsf=wsf, wts=wts, Y=Y, ws=ws))
+        return data_
 
     # ---- inputs (resident in HBM), weights quantized once
-    acts = {}
-    data = []
-    for i, l in enumerate(layers):
-        X, W, bias = workloads.make_layer(cfg, i, dev)
-        if l.K in acts:
-            X = acts[l.K]          # one activation tensor per distinct K (all larger than L2)
-        else:
-            acts[l.K] = X
-        wq, wsf, wts = B.nvfp4_quantize_weight(W)
-        Y = torch.empty((l.M, l.N), dtype=torch.bfloat16, device=dev)
-        ws = torch.empty(B.linear_workspace_bytes(l.M, l.N, l.K), dtype=torch.uint8, device=dev)
-        data.append(dict(l=l, X=X, W=W, bias=bias, wq=wq, wsf=wsf, wts=wts, Y=Y, ws=ws))
+    data = make_data(cfg)
     torch.cuda.synchronize()
 
-    def fp4_step():
-        for d in data:
-            B.nvfp4_quantize_linear(d["X"], d["wq"], d["wsf"], d["wts"], d["bias"], workspace=d["ws"], out=d["Y"])
+    def fp4_step_of(data_):
+        def step():
+            for d in data_:
+                B.nvfp4_quantize_linear(d["X"], d["wq"], d["wsf"], d["wts"], d["bias"], workspace=d["ws"], out=d["Y"])
+        return step
 
-    def bf16_step():
-        for d in data:
-            B.bf16_linear(d["X"], d["W"], d["bias"], out=d["Y"])
+    def bf16_step_of(data_):
+        def step():
+            for d in data_:
+                B.bf16_linear(d["X"], d["W"], d["bias"], out=d["Y"])
+        return step
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, steps):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(steps):
-            fn()
-        e1.record()
-        barrier()
-        ms, _, _ = replicas.aggregate(e0.elapsed_time(e1), 1.0, dev)  # max over ranks
-        return ms
-
-    for _ in range(max(3, args.warmup)):
-        fp4_step()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    ms_fp4 = timed(fp4_step, args.steps)
-    clocks = sampler.stop() if rank == 0 else None
-    B.sol_last_device_status()
+    fp4_step, bf16_step = fp4_step_of(data), bf16_step_of(data)
 
     # the same FP4 stack with a delayed tensor scale: no amax pass -- the quantizer collects max|x| as a
     # by-product and the scale is rolled forward once per step and layer (one tiny kernel)
@@ -260,12 +324,6 @@ def run_ours(args):
                                             workspace=d["ws"], out=d["Y"])
             B.sol_roll_tensor_scale(state)
 
-    for _ in range(3):
-        fp4_static_step()
-    ms_static = timed(fp4_static_step, args.steps)
-    B.sol_last_device_status()
-    del static
-
     # the MXFP4 variant of the stack (32-element blocks, E8M0 scales): no tensor scale, hence no amax pass
     mx = []
     for d in data:
@@ -279,22 +337,72 @@ def run_ours(args):
             B.mxfp4_quantize(d["X"], out=(xq, xsf))
             B.mxfp4_linear(xq, xsf, wq_mx, wsf_mx, d["bias"], out=d["Y"])
 
-    for _ in range(3):
-        mxfp4_step()
-    ms_mx = timed(mxfp4_step, args.steps)
+    # the FP4 stack through the three separate entries with an event behind every kernel: the split of the
+    # step into amax / quantizer / GEMM, taken inside a long loop (same clock state as the step itself)
+    split_buf = []
+    for d in data:
+        l = d["l"]
+        split_buf.append((d, torch.empty(1, dtype=torch.float32, device=dev),
+                          torch.empty((l.M, l.K // 2), dtype=torch.uint8, device=dev),
+                          torch.empty(B.scale_bytes(l.M, l.K), dtype=torch.uint8, device=dev)))
+    split_events = []
+
+    def fp4_split_step():
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3 * len(split_buf) + 1)]
+        ev[0].record()
+        for i, (d, xts, xq, xsf) in enumerate(split_buf):
+            B.sol_amax_bf16(d["X"], out=xts)
+            ev[3 * i + 1].record()
+            B.nvfp4_quantize(d["X"], xts, out=(xq, xsf))
+            ev[3 * i + 2].record()
+            B.nvfp4_linear(xq, xsf, xts, d["wq"], d["wsf"], d["wts"], d["bias"], out=d["Y"])
+            ev[3 * i + 3].record()
+        split_events.append(ev)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    timer = LegTimer(torch, replicas, dev, dist, sampler, args.steps, args.min_leg_s, args.rounds)
+    legs = {"nvfp4": fp4_step, "nvfp4_delayed_scale": fp4_static_step, "mxfp4": mxfp4_step, "bf16": bf16_step}
+    res = timer.run(legs, warm)
     B.sol_last_device_status()
-    del mx
+    del static, mx
 
-    for _ in range(max(3, args.warmup)):
-        bf16_step()
-    ms_bf16 = timed(bf16_step, args.steps)
+    # ---- split of the step, in one more long region of the instrumented step
+    for _ in range(2):
+        fp4_split_step()
+    torch.cuda.synchronize()
+    split_events.clear()
+    split_ms, _, split_win = timer.region(fp4_split_step, max(1, int(args.min_leg_s * 1e3 / (res["nvfp4"]["ms_per_step"] * args.steps)) + 1))
+    per_layer_split = []
+    for i in range(len(split_buf)):
+        acc = [0.0, 0.0, 0.0]
+        for ev in split_events:
+            for j in range(3):
+                acc[j] += ev[3 * i + j].elapsed_time(ev[3 * i + j + 1])
+        per_layer_split.append([a / len(split_events) for a in acc])
+    del split_buf
+    split_events.clear()
     B.sol_last_device_status()
 
+    # ---- rollout-scaling sweep point (config 5): the single-stream pair at group size 16, 28 denoising-step
+    # calls per sequence, NVFP4 and BF16 sequences in rotated long regions like the legs above
+    sweep = None
+    if not args.lean and args.sweep_group > 0:
+        scfg = workloads.config_sweep(args.sweep_group)
+        sdata = make_data(scfg)
+        stimer = LegTimer(torch, replicas, dev, dist, sampler, workloads.SWEEP_STEPS, args.min_leg_s, args.rounds)
+        sres = stimer.run({"nvfp4": fp4_step_of(sdata), "bf16": bf16_step_of(sdata)}, 2)
+        B.sol_last_device_status()
+        sflops = flops_of(scfg.layers)
+        sweep = {"group": args.sweep_group, "M": scfg.layers[0].M, "calls_per_sequence": workloads.SWEEP_STEPS,
+                 "layers": [f"{l.name}:{l.M}x{l.K}->{l.N}" for l in scfg.layers], "res": sres, "flops": sflops}
+        del sdata
 
-    # ---- per-kernel durations: each kernel launched n times back to back between two events on the
-    # launching stream (events between every launch would add idle gaps of several microseconds).
-    # Every kernel's working set exceeds L2 (X >= 226 MB for the streaming kernels, Y >= 226 MB for the
-    # GEMMs); the packed X a GEMM reads is L2-warm, as it is in the step, where the quantizer wrote it.
+    # ---- per-kernel durations in isolation: each kernel launched n times back to back between two events on
+    # the launching stream.  Every kernel's working set exceeds L2 (X >= 226 MB for the streaming kernels,
+    # Y >= 226 MB for the GEMMs); the packed X a GEMM reads is L2-warm, as it is in the step.  These short
+    # loops run at burst clocks and are compared with burst peaks; the split above is what adds up to the step.
     per_layer = []
     n_detail = max(5, min(args.steps, 20))
     tot = {"amax": 0.0, "quant": 0.0, "gemm": 0.0}
@@ -309,7 +417,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / n_detail
 
-    for d in data:
+    for d, split in zip(data, per_layer_split):
         l = d["l"]
         xts = torch.empty(1, dtype=torch.float32, device=dev)
         xq = torch.empty((l.M, l.K // 2), dtype=torch.uint8, device=dev)
@@ -324,12 +432,15 @@ def run_ours(args):
         qbytes = l.M * l.K * 2 + l.M * l.K // 2 + B.scale_bytes(l.M, l.K)
         per_layer.append({
             "layer": l.name, "M": l.M, "K": l.K, "N": l.N,
-            "amax_ms": round(t_amax, 4), "quant_ms": round(t_quant, 4), "gemm_ms": round(t_gemm, 4),
-            "stack_ms": round(t_stack, 4), "bf16_ms": round(t_bf16, 4),
-            "gemm_tflops": round(fl / t_gemm / 1e9, 1), "stack_tflops": round(fl / t_stack / 1e9, 1),
-            "bf16_tflops": round(fl / t_bf16 / 1e9, 1),
-            "quant_gbs": round(qbytes / t_quant / 1e6, 1), "amax_gbs": round(l.M * l.K * 2 / t_amax / 1e6, 1),
-            "stack_speedup": round(t_bf16 / t_stack, 3),
+            "in_step_ms": {"amax": round(split[0], 4), "quant": round(split[1], 4), "gemm": round(split[2], 4)},
+            "isolated_ms": {"amax": round(t_amax, 4), "quant": round(t_quant, 4), "gemm": round(t_gemm, 4),
+                            "stack": round(t_stack, 4), "bf16": round(t_bf16, 4)},
+            "gemm_tflops_in_step": round(fl / split[2] / 1e9, 1), "gemm_tflops_isolated": round(fl / t_gemm / 1e9, 1),
+            "bf16_tflops_isolated": round(fl / t_bf16 / 1e9, 1),
+            "quant_gbs_in_step": round(qbytes / split[1] / 1e6, 1), "quant_gbs_isolated": round(qbytes / t_quant / 1e6, 1),
+            "amax_gbs_in_step": round(l.M * l.K * 2 / split[0] / 1e6, 1),
+            "amax_gbs_isolated": round(l.M * l.K * 2 / t_amax / 1e6, 1),
+            "stack_speedup_isolated": round(t_bf16 / t_stack, 3),
         })
         tot["amax"] += t_amax
         tot["quant"] += t_quant
@@ -338,14 +449,20 @@ def run_ours(args):
     B.sol_last_device_status()
 
     flops = flops_of(layers)
-    ms_step = ms_fp4 / args.steps
+    ms_step = res["nvfp4"]["ms_per_step"]
+    ms_bf16 = res["bf16"]["ms_per_step"]
     value = world * flops / (ms_step * 1e-3) / 1e12
-    bf16_value = world * flops / (ms_bf16 / args.steps * 1e-3) / 1e12
-    gemm_tflops = flops / (tot["gemm"] * 1e-3) / 1e12
-    fp4_peak = peaks["bf16_tflops_sustained"] * (NOMINAL_FP4_TFLOPS / NOMINAL_BF16_TFLOPS)
+    bf16_value = world * flops / (ms_bf16 * 1e-3) / 1e12
     quant_bytes = sum(l.M * l.K * 2 + l.M * l.K // 2 + B.scale_bytes(l.M, l.K) for l in layers)
+    amax_bytes = sum(l.M * l.K * 2 for l in layers)
     gemm_bytes = sum(l.M * l.K // 2 + B.scale_bytes(l.M, l.K) + l.N * l.K // 2 + B.scale_bytes(l.N, l.K) + 2 * l.N +
                      2 * l.M * l.N for l in layers)
+    # split of the step: the instrumented step's shares scaled to the plain step (its events cost a few
+    # microseconds each and keep consecutive kernels from overlapping their prologues)
+    split_tot = [sum(s[j] for s in per_layer_split) for j in range(3)]
+    split_scale = ms_step / sum(split_tot)
+    in_step = {"amax_ms": split_tot[0] * split_scale, "quant_ms": split_tot[1] * split_scale,
+               "gemm_ms": split_tot[2] * split_scale, "instrumented_step_ms": split_ms, "scale": split_scale}
 
     # ---- weight refresh after a policy update: merge the rank-32 adapters of every targeted projection
     # and re-quantize it.  FLUX targets to_q/k/v/out: 19 double blocks x 4 + 38 single blocks x 3 = 190
@@ -411,7 +528,7 @@ def run_ours(args):
         B.nvfp4_quantize(d1["X"], xts, out=(xq, xsf))
         B.nvfp4_linear_quantized_out(xq, xsf, xts, d1["wq"], d1["wsf"], d1["wts"], d1["bias"], B.ACT_GELU_TANH, t_out,
                                      amax_out=amax, out=(hq, hsf))
-        t_out.copy_(amax / 2688.0)          # calibration from the first call's amax (device to device)
+        t_out.copy_(rolled_scale(B, torch, amax))   # calibration from the first call's amax (device to device)
 
         def pair_unfused():
             B.nvfp4_quantize_linear(d1["X"], d1["wq"], d1["wsf"], d1["wts"], d1["bias"], workspace=d1["ws"], out=d1["Y"])
@@ -495,7 +612,8 @@ def run_ours(args):
                 B.nvfp4_quantize_linear(d2["X"], d2["wq"], d2["wsf"], d2["wts"], d2["bias"], workspace=d2["ws"], out=d2["Y"])
 
             single_fused()
-            t_cat.copy_(torch.maximum(amax, B.sol_amax_bf16(attn) * 2688.0) / 2688.0)   # calibrate T of the concat
+            # T of the concat: the larger of the two parts' scales (T is monotone in the amax)
+            t_cat.copy_(torch.maximum(rolled_scale(B, torch, amax), B.sol_amax_bf16(attn)))
             t_unf, t_fus = loop_ms(single_unfused), loop_ms(single_fused)
             t_unf, t_fus = min(t_unf, loop_ms(single_unfused)), min(t_fus, loop_ms(single_fused))
             B.sol_last_device_status()
@@ -524,7 +642,7 @@ def run_ours(args):
         lq = (torch.empty((l0.M, l0.K // 2), dtype=torch.uint8, device=dev),
               torch.empty(B.scale_bytes(l0.M, l0.K), dtype=torch.uint8, device=dev))
         B.nvfp4_layernorm_quantize(Xl, sc, sh, rps, state, amax_out=amax, out=lq)
-        state.copy_(amax / 2688.0)
+        state.copy_(rolled_scale(B, torch, amax))
         t_fused = loop_ms(lambda: B.nvfp4_layernorm_quantize(Xl, sc, sh, rps, state, amax_out=amax, out=lq))
         xts_l = torch.empty(1, dtype=torch.float32, device=dev)
 
@@ -788,8 +906,8 @@ def run_only(args):
 
         use_ours["fused"] = False
         out4 = block_fp4()                       # calibrate the delayed scales from the first pass
-        state.copy_(amax_in / 2688.0)
-        t_cat.copy_(torch.maximum(amax_cat, B.sol_amax_bf16(attention(y_qkv)) * 2688.0) / 2688.0)
+        state.copy_(rolled_scale(B, torch, amax_in))
+        t_cat.copy_(torch.maximum(rolled_scale(B, torch, amax_cat), B.sol_amax_bf16(attention(y_qkv))))
         res = {}
         variants = (("nvfp4", block_fp4, True, False), ("nvfp4_attention_quantized_output", block_fp4, True, True),
                     ("bf16", block_bf16, True, False), ("nvfp4_torch_attention", block_fp4, False, False),

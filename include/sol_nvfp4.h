@@ -433,6 +433,27 @@ sol_status_t nvfp4_quantize_linear_static(const void *x_bf16, int64_t ldx, const
  */
 sol_status_t sol_last_device_status(void *stream, uint32_t *detail_out);
 
+/*
+ * (No counterpart in the paper: failure detection of the kernels themselves.)
+ *
+ * Sets, for the current device, the limit of every bounded device-side wait in SM clock cycles
+ * (default 4e9, about two seconds; `cycles` <= 0 restores the default).  Synchronous: it copies
+ * eight bytes to the device and affects kernels launched afterwards.  A wait that exceeds the limit
+ * makes its kernel leave through the normal teardown (outputs incomplete) and is reported by
+ * sol_last_device_status as SOL_ERR_TIMEOUT; the context stays usable.
+ */
+sol_status_t sol_set_wait_limit_cycles(int64_t cycles);
+
+/*
+ * Test hook for that path (no counterpart in the paper).  While `on` is non-zero on the current
+ * device, the load-issuing warps of the CTA-pair GEMM kernels (M > 128: nvfp4_linear, mxfp4_linear,
+ * bf16_linear and the entries built on them) issue no loads, so every consumer wait of such a launch
+ * runs into the wait limit: nothing traps, faults or spins without bound, the kernel returns with Y
+ * unwritten and the status word set.  Use it with a short limit (about 1e6 cycles) and switch it off
+ * again; it is not meant for anything but exercising the time-out path.
+ */
+sol_status_t sol_test_hold_loads(int on);
+
 #ifdef __cplusplus
 }
 #endif

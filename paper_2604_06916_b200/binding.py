@@ -26,7 +26,7 @@ EXPORTS = [
     "solrl_select_contrastive", "solrl_rank_consistency", "sol_mxfp4_scale_bytes", "mxfp4_quantize",
     "mxfp4_linear", "nvfp4_linear_split_out", "nvfp4_quantize_into",
     "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale", "nvfp4_layernorm_quantize", "sol_attention_bf16", "sol_attention_bf16_joint",
-    "sol_attention_nvfp4_out", "mxfp4_linear_quantized_out",
+    "sol_attention_nvfp4_out", "mxfp4_linear_quantized_out", "sol_set_wait_limit_cycles", "sol_test_hold_loads",
 ]
 
 _lib = None
@@ -102,6 +102,8 @@ def lib() -> ctypes.CDLL:
     L.sol_attention_bf16.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, i64, vp]
     L.nvfp4_layernorm_quantize.restype = i32
     L.nvfp4_layernorm_quantize.argtypes = [vp, i64, i64, i64, vp, vp, i64, ctypes.c_float, vp, vp, vp, vp, vp]
+    L.sol_set_wait_limit_cycles.restype, L.sol_set_wait_limit_cycles.argtypes = i32, [i64]
+    L.sol_test_hold_loads.restype, L.sol_test_hold_loads.argtypes = i32, [i32]
     L.sol_last_device_status.restype = i32
     L.sol_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     _lib = L
@@ -570,5 +572,17 @@ def sol_last_device_status() -> int:
     detail = ctypes.c_uint32(0)
     code = lib().sol_last_device_status(_stream(), ctypes.byref(detail))
     if code != 0:
-        raise SolError(code, f"device status word 0x{detail.value:x}")
+        err = SolError(code, f"device status word 0x{detail.value:x}")
+        err.detail = detail.value
+        raise err
     return 0
+
+
+def sol_set_wait_limit_cycles(cycles: int) -> None:
+    """Limit of every bounded device-side wait on the current device, in SM cycles (<= 0: default)."""
+    _check(lib().sol_set_wait_limit_cycles(int(cycles)), "sol_set_wait_limit_cycles")
+
+
+def sol_test_hold_loads(on: bool) -> None:
+    """Test hook: while on, the pair GEMM kernels issue no loads and their waits run into the limit."""
+    _check(lib().sol_test_hold_loads(1 if on else 0), "sol_test_hold_loads")

@@ -3,11 +3,12 @@
 #include "sol_internal.h"
 #include "gemm_common.cuh"
 
+#include <cstddef>
 #include <mutex>
 
 namespace sol {
 
-__device__ uint32_t g_status_word = 0;
+__device__ DeviceStatusBlock g_status_block = {0u, 0u, kDefaultWaitLimitCycles};
 
 namespace {
 
@@ -48,7 +49,7 @@ const DeviceInfo *current_device_info() {
         d.cc_major = prop.major;
         d.cc_minor = prop.minor;
         void *sym = nullptr;
-        if (cudaGetSymbolAddress(&sym, g_status_word) != cudaSuccess) return nullptr;
+        if (cudaGetSymbolAddress(&sym, g_status_block) != cudaSuccess) return nullptr;
         g_status_ptr[dev] = static_cast<uint32_t *>(sym);
         d.ok = true;
     }
@@ -661,6 +662,27 @@ sol_status_t nvfp4_quantize_linear_host(const void *x_host, int64_t ldx, const v
     return SOL_OK;
 }
 
+sol_status_t sol_set_wait_limit_cycles(int64_t cycles) {
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    const long long limit = cycles > 0 ? static_cast<long long>(cycles) : kDefaultWaitLimitCycles;
+    if (cudaMemcpyToSymbol(g_status_block, &limit, sizeof(limit), offsetof(DeviceStatusBlock, wait_limit_cycles)) !=
+        cudaSuccess)
+        return SOL_ERR_CUDA;
+    return SOL_OK;
+}
+
+sol_status_t sol_test_hold_loads(int on) {
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    const uint32_t flag = on ? 1u : 0u;
+    if (cudaMemcpyToSymbol(g_status_block, &flag, sizeof(flag), offsetof(DeviceStatusBlock, hold_loads)) != cudaSuccess)
+        return SOL_ERR_CUDA;
+    return SOL_OK;
+}
+
 sol_status_t sol_last_device_status(void *stream, uint32_t *detail_out) {
     const DeviceInfo *dev = nullptr;
     sol_status_t st = check_arch(&dev);
@@ -668,11 +690,11 @@ sol_status_t sol_last_device_status(void *stream, uint32_t *detail_out) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint32_t word = 0;
     if (cudaStreamSynchronize(s) != cudaSuccess) return SOL_ERR_CUDA;
-    if (cudaMemcpyFromSymbol(&word, g_status_word, sizeof(word)) != cudaSuccess) return SOL_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&word, g_status_block, sizeof(word)) != cudaSuccess) return SOL_ERR_CUDA;
     if (detail_out != nullptr) *detail_out = word;
     if (word != 0) {
         const uint32_t zero = 0;
-        if (cudaMemcpyToSymbol(g_status_word, &zero, sizeof(zero)) != cudaSuccess) return SOL_ERR_CUDA;
+        if (cudaMemcpyToSymbol(g_status_block, &zero, sizeof(zero)) != cudaSuccess) return SOL_ERR_CUDA;
         return SOL_ERR_TIMEOUT;
     }
     return SOL_OK;

@@ -18,7 +18,6 @@ constexpr int kEpiWarps = 4;
 constexpr int kEpiBufBytes = 32 * 128;  // 32 rows x 64 BF16
 constexpr int kTmemCols = 512;
 constexpr int kGroupM = 8;            // tile raster: groups of 8 row tiles sweep all column tiles
-constexpr long long kWaitLimitCycles = 4000000000LL;
 
 // Diagnostic switches, compiled in only with -DSOL_TUNING (never in the product build): they
 // drop one part of the pipeline so its share of the time can be read off a timing run.
@@ -65,13 +64,19 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
     // take issue slots from the few that have work (the epilogue at a tile boundary, above all)
     while (!ptx::mbar_try_wait_suspend(bar, parity, 200000u)) {
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
+        // the limit lives in the device status block (words 2..3); it is read on this slow path only
+        if (clock64() - t0 > *reinterpret_cast<const volatile long long *>(status + 2)) {
             *abort_flag = 1;
             atomicExch(status, code);
             return false;
         }
     }
     return true;
+}
+
+// Test hook (device status block, word 1): the load-issuing warps issue nothing while it is set.
+__device__ __forceinline__ bool loads_held(const uint32_t *status) {
+    return *reinterpret_cast<const volatile uint32_t *>(status + 1) != 0;
 }
 
 __device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int &mt, int &nt) {

@@ -117,7 +117,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             const bool trace = kTuning && (p.dbg & kDbgTrace);
             int stage = 0;
             uint32_t phase = 0;
-            bool ok = true;
+            bool ok = !loads_held(p.status);
             [[maybe_unused]] int pgi = 0;
             for (int t = pair; ok && t < total_tiles; t += num_pairs) {
                 int mt, nt;

@@ -324,7 +324,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         [[maybe_unused]] int gi_trace = 0;
         int stage = 0;
         uint32_t phase = 0;
-        bool ok = true;
+        bool ok = !loads_held(p.status);
         for (int t = pair; ok && t < total_tiles; t += num_pairs) {
             int mt, nt;
             tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
@@ -358,7 +358,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             const uint32_t full0 = ptx::map_to_cta(sf_full_bar(0), kSfViaStore ? rank : 0u);
             int stage = 0;
             uint32_t phase = 0;
-            bool ok = true;
+            bool ok = !loads_held(p.status);
             for (int t = pair; ok && t < total_tiles; t += num_pairs) {
                 int mt, nt;
                 tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);

@@ -34,7 +34,18 @@ inline sol_status_t launch_status() {
     return e == cudaSuccess ? SOL_OK : SOL_ERR_CUDA;
 }
 
-// Device status word written by bounded waits (0 = fine).
+// Device status block, one per device.  `code` is written by a bounded wait that ran out (0 = none)
+// and read and cleared by sol_last_device_status; `wait_limit_cycles` is the limit of every bounded
+// wait in SM cycles (sol_set_wait_limit_cycles); `hold_loads` is the test hook of
+// sol_test_hold_loads: while non-zero the load-issuing warps of the CTA-pair GEMM kernels issue
+// nothing, so every consumer wait of those kernels runs into the limit.
+struct DeviceStatusBlock {
+    uint32_t code;
+    uint32_t hold_loads;
+    long long wait_limit_cycles;
+};
+constexpr long long kDefaultWaitLimitCycles = 4000000000LL;
+// Pointer to the block's first word (kernels receive it as `status`; words 1.. follow the struct).
 uint32_t *device_status_word();
 
 // Internal launchers (arguments already validated).
