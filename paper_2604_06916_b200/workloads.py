@@ -162,6 +162,19 @@ def make_qkv(batch: int, seq: int, heads: int, seed: int, device="cpu", q_gain: 
     return fused, q, k, v
 
 
+def sample_rows(M: int, seed: int = 0):
+    """Row sample of an [M, ...] problem used wherever the CPU oracle cannot afford every row: the first and
+    the last 128-row tile in full plus one pseudo-random row of every other tile (numpy int64, sorted)."""
+    import numpy as np
+
+    rng = np.random.default_rng(seed)
+    tiles = (M + 127) // 128
+    rows = set(range(min(128, M))) | set(range((tiles - 1) * 128, M))
+    for t in range(1, tiles - 1):
+        rows.add(t * 128 + int(rng.integers(0, 128)))
+    return np.array(sorted(rows), dtype=np.int64)
+
+
 def to_bits(t: torch.Tensor):
     """bf16 tensor -> numpy uint16 bit patterns (host)."""
     import numpy as np

@@ -30,12 +30,8 @@ def unswizzle_rows(sf_swizzled: np.ndarray, rows, K: int) -> np.ndarray:
 
 def sample_rows(M: int, seed: int = 0) -> np.ndarray:
     """First and last 128-row tile in full plus one pseudo-random row of every other tile."""
-    rng = np.random.default_rng(seed)
-    tiles = (M + 127) // 128
-    rows = set(range(min(128, M))) | set(range((tiles - 1) * 128, M))
-    for t in range(1, tiles - 1):
-        rows.add(t * 128 + int(rng.integers(0, 128)))
-    return np.array(sorted(rows), dtype=np.int64)
+    from paper_2604_06916_b200 import workloads
+    return workloads.sample_rows(M, seed)
 
 
 def check_linear(y_gpu_bits: np.ndarray, Y: np.ndarray, what: str = ""):
