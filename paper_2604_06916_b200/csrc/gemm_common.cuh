@@ -56,19 +56,43 @@ struct Params {
     int dest_chunks_k;      // scale chunks per 128-row tile of the destination tensor
 };
 
+#ifndef SOL_WAIT_HINT
+#define SOL_WAIT_HINT 200000u
+#endif
 __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
                                              uint32_t *status, uint32_t code) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     // long hardware suspends: a CTA has ~20 warps that mostly wait, and warps that poll in a tight loop
     // take issue slots from the few that have work (the epilogue at a tile boundary, above all)
-    while (!ptx::mbar_try_wait_suspend(bar, parity, 200000u)) {
+    while (!ptx::mbar_try_wait_suspend(bar, parity, SOL_WAIT_HINT)) {
         if (*abort_flag) return false;
         // the limit lives in the device status block (words 2..3); it is read on this slow path only
         if (clock64() - t0 > *reinterpret_cast<const volatile long long *>(status + 2)) {
             *abort_flag = 1;
             atomicExch(status, code);
             return false;
+        }
+    }
+    return true;
+}
+
+// The same for a wait on the critical path of a pipeline: polls without suspending (a suspended thread
+// takes several hundred cycles to resume after the barrier completes), a short sleep between polls.
+__device__ __forceinline__ bool wait_bounded_spin(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                                  uint32_t *status, uint32_t code) {
+    if (ptx::mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t n = 0;
+    while (!ptx::mbar_test_wait(bar, parity)) {
+        __nanosleep(20);
+        if ((++n & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > *reinterpret_cast<const volatile long long *>(status + 2)) {
+                *abort_flag = 1;
+                atomicExch(status, code);
+                return false;
+            }
         }
     }
     return true;

@@ -34,23 +34,34 @@ constexpr int kABytes = kBM * kRowBytes;       // 16 KB: this CTA's 128 rows of 
 constexpr int kBBytes = (kBN / 2) * kRowBytes; // 16 KB: this CTA's half of the B tile
 constexpr int kSfaBytes = 2048;                // 4 k-chunks x 512 bytes
 constexpr int kSfbBytes = 4096;                // 2 row chunks x 4 k-chunks x 512 bytes
-constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 38 912
+constexpr int kStageBytes = kABytes + kBBytes;  // 32 KB: one k-tile of A and B
+constexpr int kSfSlotBytes = kSfaBytes + kSfbBytes;  // 6 KB: one k-tile of scale tiles
+constexpr int kSfSlots = 5;                    // scale-tile ring in shared memory, released as soon as a tile is in registers
 constexpr int kSfBufCols = 48;                 // per k-tile: 4 MMAs x (4 columns of A + 8 of B)
 constexpr int kAccStride = 96;                 // accumulator B starts here; [96,256) is shared
 constexpr int kSfBufs = 3;
 constexpr int kSfCol = kAccStride + kBN;       // 352
 constexpr int kEpiWarpsFp4 = 8;
-constexpr int kSfCopyWarps = 4;                // one per MMA of a k-tile: three tcgen05.cp each
+constexpr int kSfCopyWarps = 4;                // one per TMEM lane quadrant
 constexpr int kWarps = 2 + kEpiWarpsFp4 + kSfCopyWarps + 1;
-#ifdef SOL_SF_COPY
-constexpr bool kSfViaStore = false;
-#else
-constexpr bool kSfViaStore = true;   // scale tiles reach TMEM by tcgen05.st from the copy warps, not tcgen05.cp
+#ifndef SOL_SPIN_MASK
+#define SOL_SPIN_MASK 0
 #endif
-constexpr int kThreadsFp4 = 32 * kWarps;       // 544
+// which waits poll instead of suspending: 1 A/B producer on `empty`, 2 scale-copy warps on the TMEM buffer,
+// 4 MMA thread on `sf_ready` / `full`, 8 epilogue on `acc_full`, 16 MMA thread on `ovl_free` / `acc_empty`
+template <int kBit>
+__device__ __forceinline__ bool wait_site(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
+                                          uint32_t code) {
+    if constexpr ((SOL_SPIN_MASK & kBit) != 0) return wait_bounded_spin(bar, parity, abort_flag, status, code);
+    else return wait_bounded(bar, parity, abort_flag, status, code);
+}
+constexpr int kThreadsFp4 = 32 * (kWarps + (kTuning ? 1 : 0));  // 480 (+ a probe warp in the diagnostic build)
 constexpr int kEpiBytes = kEpiWarpsFp4 * kEpiBufBytes;
 constexpr int kBiasBytes = kEpiWarpsFp4 * 256;  // per epilogue warp: BF16 bias of its two 64-column chunks
-constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kBiasBytes + 256 + 1024;
+constexpr int kNumBars = 2 * kStages + 6 + kSfBufs + 2 * kSfSlots;
+constexpr int kBarBytes = 512;
+constexpr int kSmemBytes = kStages * kStageBytes + kSfSlots * kSfSlotBytes + kEpiBytes + kBiasBytes + kBarBytes + 1024;
+static_assert(8 * kNumBars + 8 <= kBarBytes, "barrier area");
 static_assert(kSfCol + kSfBufs * kSfBufCols <= kTmemCols, "TMEM budget");
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
@@ -254,23 +265,25 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
 
-    const uint32_t epi_base = smem_base + kStages * kStageBytes;
+    const uint32_t sf_base = smem_base + kStages * kStageBytes;
+    const uint32_t epi_base = sf_base + kSfSlots * kSfSlotBytes;
     const uint32_t bias_base = epi_base + kEpiBytes;
     const uint32_t bar_base = bias_base + kBiasBytes;
-    uint8_t *bar_gen = smem_gen + kStages * kStageBytes + kEpiBytes + kBiasBytes;
+    uint8_t *bar_gen = smem_gen + kStages * kStageBytes + kSfSlots * kSfSlotBytes + kEpiBytes + kBiasBytes;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
     auto acc_full_bar = [&](int s) { return bar_base + 8u * (2 * kStages + s); };
     auto acc_empty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 2 + s); };
     auto ovl_free_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 4 + s); };
     auto sf_ready_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 6 + s); };
-    // The scale tiles of a stage complete on a barrier of their own: they are a sixth of the stage's bytes
-    // and land first, so their copy into TMEM (a ~500-cycle chain: copy warp wake-up, tcgen05.cp, commit)
-    // overlaps the arrival of A and B instead of following it.
+    // The scale tiles travel in a ring of their own, a sixth of a k-tile's bytes each.  A slot is handed
+    // back as soon as the copy warps hold its contents in registers, not when the k-tile's MMAs are
+    // done, so the scale loads run several k-tiles ahead of the A and B loads and the copy into tensor
+    // memory (load -> registers -> tcgen05.st -> arrive, ~800 cycles end to end) is off the critical path.
     auto sf_full_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 6 + kSfBufs + s); };
-    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * (3 * kStages + 6 + kSfBufs));
-    volatile uint32_t *abort_flag =
-        reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * (3 * kStages + 6 + kSfBufs) + 4);
+    auto sf_empty_bar = [&](int s) { return bar_base + 8u * (2 * kStages + 6 + kSfBufs + kSfSlots + s); };
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(bar_gen + 8 * kNumBars);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(bar_gen + 8 * kNumBars + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();
@@ -286,15 +299,18 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(full_bar(s), 1);
-            ptx::mbar_init(sf_full_bar(s), 1);
             ptx::mbar_init(empty_bar(s), 1);
+        }
+        for (int s = 0; s < kSfSlots; ++s) {
+            ptx::mbar_init(sf_full_bar(s), 1);
+            ptx::mbar_init(sf_empty_bar(s), kSfCopyWarps);
         }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(acc_full_bar(s), 1);
             ptx::mbar_init(acc_empty_bar(s), 2 * kEpiWarpsFp4);
             ptx::mbar_init(ovl_free_bar(s), 2 * kEpiWarpsFp4);
         }
-        for (int s = 0; s < kSfBufs; ++s) ptx::mbar_init(sf_ready_bar(s), kSfViaStore ? 2 * kSfCopyWarps : kSfCopyWarps);
+        for (int s = 0; s < kSfBufs; ++s) ptx::mbar_init(sf_ready_bar(s), 2 * kSfCopyWarps);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tm_a);
@@ -315,7 +331,23 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     const uint32_t tmem_base = *tmem_ptr_smem;
     ptx::grid_dependency_wait();  // set-up above overlaps the previous kernel; its results are read below
 
-    if (warp == 0) {
+    if (kTuning && warp == kWarps) {
+        // diagnostic build: polls each stage's `full` barrier without suspending and records when it completes
+        if ((p.dbg & kDbgTrace) && leader && lane < 2) {
+            int stage = 0;
+            uint32_t phase = 0;
+            const int n = ((total_tiles - pair + num_pairs - 1) / num_pairs) * k_tiles;
+            for (int gi = 0; gi < n && gi < 512; ++gi) {
+                const long long t0 = clock64();
+                const uint32_t bar = lane == 0 ? full_bar(stage) : empty_bar(stage);
+                while (!ptx::mbar_test_wait(bar, phase) && clock64() - t0 < 4000000) {}
+#ifdef SOL_TUNING
+                if (blockIdx.x < 2) g_trace[lane == 0 ? 11 : 1][gi] = clock64();
+#endif
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 0) {
         // ------------------------------------------------------------ TMA producer: A and B tiles (both CTAs)
         const bool elected = ptx::elect_one();
         const uint32_t full0 = ptx::map_to_cta(full_bar(0), 0);  // the even CTA's barriers
@@ -332,7 +364,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             const int nb0 = nt * kBN + static_cast<int>(rank) * (kBN / 2);
             int kx = 0;
             for (int kt = 0; kt < k_tiles; ++kt, kx += kRowBytes) {
-                if (!wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x100u | stage)) {
+                if (!wait_site<1>(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x100u | stage)) {
                     ok = false;
                     break;
                 }
@@ -352,34 +384,33 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         __syncwarp();
     } else if (warp == kWarps - 1) {
         // ------------------------------------------------------------ TMA producer: scale-factor tiles (both CTAs)
-        if (!(kTuning && (p.dbg & kDbgNoSfLoad))) {
-            const bool elected = ptx::elect_one();
-            // store path: each CTA's tiles complete on its own barrier, where its own copy warps wait
-            const uint32_t full0 = ptx::map_to_cta(sf_full_bar(0), kSfViaStore ? rank : 0u);
-            int stage = 0;
-            uint32_t phase = 0;
-            bool ok = !loads_held(p.status);
-            for (int t = pair; ok && t < total_tiles; t += num_pairs) {
-                int mt, nt;
-                tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
-                const int rca = mt * 2 + static_cast<int>(rank);  // 128-row chunk of A owned by this CTA
-                const int rcb = nt * 2;                            // first of the tile's two 128-row chunks of B
-                for (int kt = 0; kt < k_tiles; ++kt) {
-                    if (!wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x800u | stage)) {
-                        ok = false;
-                        break;
-                    }
-                    const uint32_t ssfa = smem_base + stage * kStageBytes + kABytes + kBBytes;
-                    if (elected) {
-                        if (kSfViaStore) ptx::mbar_arrive_expect_tx(sf_full_bar(stage), kSfLoadBytes);
-                        else if (leader) ptx::mbar_arrive_expect_tx(sf_full_bar(stage), 2u * kSfLoadBytes);
-                        ptx::tma_load_3d_pair(ssfa, &tm_sfa, 0, kt * kSfChunksK, rca, full0 + 8u * stage);
-                        ptx::tma_load_3d_pair(ssfa + kSfaBytes, &tm_sfb, 0, kt * kSfChunksK, rcb, full0 + 8u * stage);
-                    }
-                    if (++stage == kStages) {
-                        stage = 0;
-                        phase ^= 1u;
-                    }
+        // Each CTA's tiles complete on a barrier of its own, where its own copy warps wait.
+        const bool elected = ptx::elect_one();
+        const uint32_t full0 = ptx::map_to_cta(sf_full_bar(0), rank);
+        [[maybe_unused]] int sf_gi_trace = 0;
+        int slot = 0;
+        uint32_t phase = 0;
+        bool ok = !loads_held(p.status);
+        for (int t = pair; ok && t < total_tiles; t += num_pairs) {
+            int mt, nt;
+            tile_coords(t, p.m_tiles, p.n_tiles, mt, nt);
+            const int rca = mt * 2 + static_cast<int>(rank);  // 128-row chunk of A owned by this CTA
+            const int rcb = nt * 2;                            // first of the tile's two 128-row chunks of B
+            for (int kt = 0; kt < k_tiles; ++kt) {
+                if (!wait_bounded(sf_empty_bar(slot), phase ^ 1u, abort_flag, p.status, 0x800u | slot)) {
+                    ok = false;
+                    break;
+                }
+                const uint32_t ssfa = sf_base + slot * kSfSlotBytes;
+                if (kTuning && (p.dbg & kDbgTrace) && leader) { SOL_TRACE(2, sf_gi_trace); ++sf_gi_trace; }
+                if (elected) {
+                    ptx::mbar_arrive_expect_tx(sf_full_bar(slot), kSfLoadBytes);
+                    ptx::tma_load_3d_pair(ssfa, &tm_sfa, 0, kt * kSfChunksK, rca, full0 + 8u * slot);
+                    ptx::tma_load_3d_pair(ssfa + kSfaBytes, &tm_sfb, 0, kt * kSfChunksK, rcb, full0 + 8u * slot);
+                }
+                if (++slot == kSfSlots) {
+                    slot = 0;
+                    phase ^= 1u;
                 }
             }
         }
@@ -399,7 +430,6 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             const uint32_t a_lo0 = (smem_base & 0x3FFFFu) >> 4;
             const uint32_t b_lo0 = ((smem_base + kABytes) & 0x3FFFFu) >> 4;
             constexpr uint32_t kStageLo = kStageBytes >> 4;
-            const bool no_sf_wait = kTuning && (p.dbg & kDbgNoSfCopy);
             const bool no_mma = kTuning && (p.dbg & kDbgNoMma);
             const bool trace = kTuning && (p.dbg & kDbgTrace);
             int stage = 0;
@@ -412,32 +442,24 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 const int x = it & 1;
                 const uint32_t use = static_cast<uint32_t>(it >> 1);
                 // this accumulator's previous tile is fully drained ...
-                if (!wait_bounded(acc_empty_bar(x), (use & 1u) ^ 1u, abort_flag, p.status, 0x200u | x)) break;
+                if (!wait_site<16>(acc_empty_bar(x), (use & 1u) ^ 1u, abort_flag, p.status, 0x200u | x)) break;
                 // ... and the previous tile (other accumulator) has given back the shared columns
-                if (it > 0 && !wait_bounded(ovl_free_bar(x ^ 1), (static_cast<uint32_t>(it - 1) >> 1) & 1u, abort_flag,
+                if (it > 0 && !wait_site<16>(ovl_free_bar(x ^ 1), (static_cast<uint32_t>(it - 1) >> 1) & 1u, abort_flag,
                                             p.status, 0x900u | x))
                     break;
                 ptx::tc_fence_after_sync();
                 if (trace) SOL_TRACE(8, it);
                 const uint32_t d_tmem = tmem_base + x * kAccStride;
                 for (int kt = 0; kt < k_tiles; ++kt) {
-                    // two conditions per k-tile: the scales are in TMEM (`sf_ready`, signalled by the copy warps)
-                    // and A and B are in shared memory (`full`); `sf_seen`: the previous k-tile already saw
-                    // both complete (peek below)
+                    // two conditions per k-tile: the scales are in TMEM (`sf_ready`, signalled by the copy warps,
+                    // normally long before) and A and B are in shared memory (`full`); `sf_seen`: the previous
+                    // k-tile already saw both complete (peek below)
                     if (!sf_seen) {
-                        if (!no_sf_wait &&
-                            !wait_bounded(sf_ready_bar(sf_buf), sf_phase, abort_flag, p.status, 0x500u | sf_buf)) {
+                        if (!wait_site<4>(sf_ready_bar(sf_buf), sf_phase, abort_flag, p.status, 0x500u | sf_buf)) {
                             ok = false;
                             break;
                         }
-                        if (!wait_bounded(full_bar(stage), phase, abort_flag, p.status, 0x300u | stage)) {
-                            ok = false;
-                            break;
-                        }
-                        // diagnostic build without scale copies: nobody else waits for the scale tiles, and the
-                        // stage must not be released (and its barrier re-armed) before they have landed
-                        if (no_sf_wait && !(p.dbg & kDbgNoSfLoad) &&
-                            !wait_bounded(sf_full_bar(stage), phase, abort_flag, p.status, 0x310u | stage)) {
+                        if (!wait_site<4>(full_bar(stage), phase, abort_flag, p.status, 0x300u | stage)) {
                             ok = false;
                             break;
                         }
@@ -477,7 +499,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     bool seen = false;
                     if (elected)
                         seen = ptx::tc_commit_pair_mcast_and_peek2(empty_bar(stage), 3, sf_ready_bar(nb), np, full_bar(ns), nph);
-                    sf_seen = !no_sf_wait && __any_sync(0xFFFFFFFFu, seen) != 0;  // keeps the loop warp-uniform
+                    sf_seen = __any_sync(0xFFFFFFFFu, seen) != 0;  // keeps the loop warp-uniform
                     if (trace) SOL_TRACE(3, gi);
                     ++gi;
                     sf_buf = nb;
@@ -493,14 +515,17 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
         }
         __syncwarp();
     } else if (warp >= 2 + kEpiWarpsFp4) {
-        // ------------------------------------------------------------ scale-factor copy warps (even CTA)
-        // tcgen05.cp blocks its issuing warp for ~100 cycles, so the twelve copies of a k-tile are
-        // spread over four warps and kept off the MMA thread; the third TMEM buffer hides their latency.
-        if ((leader || kSfViaStore) && !(kTuning && (p.dbg & kDbgNoSfCopy))) {
+        // ------------------------------------------------------------ scale-factor copy warps (both CTAs)
+        // One warp per TMEM lane quadrant: lane t takes line t (16 bytes) of each 512-byte chunk into
+        // registers, the slot goes back to the producer at once, and when the k-tile's buffer in tensor
+        // memory is free (the MMAs of three k-tiles ago are done) the lines are written to the warp's own
+        // quadrant with tcgen05.st -- the four warps together give the four-fold replication that the
+        // scaled MMA reads.  Nothing of this passes through the tensor pipe or the MMA thread.
+        {
             const bool elected = ptx::elect_one();
             const int w = warp - (2 + kEpiWarpsFp4);
             const uint32_t ready0 = ptx::map_to_cta(sf_ready_bar(0), 0);  // the even CTA's barriers
-            int stage = 0;
+            int slot = 0;
             uint32_t phase = 0;
             uint32_t gi = 0;
             uint32_t sf_buf = 0;
@@ -509,59 +534,41 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             bool ok = true;
             for (int t = pair; ok && t < total_tiles; t += num_pairs) {
                 for (int kt = 0; kt < k_tiles; ++kt) {
-                    if (!(kTuning && (p.dbg & kDbgNoSfLoad)) &&
-                        !wait_bounded(sf_full_bar(stage), phase, abort_flag, p.status, 0x600u | stage)) {
+                    if (!wait_bounded(sf_full_bar(slot), phase, abort_flag, p.status, 0x600u | slot)) {
                         ok = false;
                         break;
                     }
-                    if (gi >= kSfBufs &&
-                        !wait_bounded(empty_bar(old_stage), old_phase, abort_flag, p.status, 0x700u | old_stage)) {
+                    const uint32_t ssf = sf_base + slot * kSfSlotBytes + lane * 16;
+                    uint4 v[3 * kSfChunksK];
+#pragma unroll
+                    for (int c = 0; c < kSfChunksK; ++c) {
+                        v[c] = ptx::lds128(ssf + c * 512);
+                        v[kSfChunksK + c] = ptx::lds128(ssf + kSfaBytes + c * 512);
+                        v[2 * kSfChunksK + c] = ptx::lds128(ssf + kSfaBytes + kSfRowChunkBytes + c * 512);
+                    }
+                    // the slot's next contents arrive through the async proxy: order these generic-proxy reads
+                    // before it (the release chain to the producer starts at the arrive)
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (elected) ptx::mbar_arrive(sf_empty_bar(slot));
+                    if (gi >= kSfBufs && !(kTuning && (p.dbg & kDbgNoSfCopy)) &&
+                        !wait_site<2>(empty_bar(old_stage), old_phase, abort_flag, p.status, 0x700u | old_stage)) {
                         ok = false;
                         break;
                     }
                     ptx::tc_fence_after_sync();
                     if (kTuning && (p.dbg & kDbgTrace) && w == 0 && leader) SOL_TRACE(4, gi);
-                    const int nmma = (kt + 1 < k_tiles) ? kMmasPerStage : tail_mmas;
-                    if (kSfViaStore) {
-                        // Every warp writes its own TMEM quadrant: lane t takes line t (16 bytes) of each
-                        // 512-byte chunk, the four warps together give the four-fold replication that the
-                        // scaled MMA reads.  Nothing of this passes through the tensor pipe.
-                        const uint32_t ssf = smem_base + stage * kStageBytes + kABytes + kBBytes + lane * 16;
-                        const uint32_t sf_t =
-                            tmem_base + kSfCol + sf_buf * kSfBufCols + (static_cast<uint32_t>(warp & 3) << 21);
-                        uint4 v[3 * kSfChunksK];
+                    const uint32_t sf_t = tmem_base + kSfCol + sf_buf * kSfBufCols + (static_cast<uint32_t>(warp & 3) << 21);
 #pragma unroll
-                        for (int c = 0; c < kSfChunksK; ++c) {
-                            v[c] = ptx::lds128(ssf + c * 512);
-                            v[kSfChunksK + c] = ptx::lds128(ssf + kSfaBytes + c * 512);
-                            v[2 * kSfChunksK + c] = ptx::lds128(ssf + kSfaBytes + kSfRowChunkBytes + c * 512);
-                        }
-#pragma unroll
-                        for (int c = 0; c < kSfChunksK; ++c) {
-                            ptx::tc_store_32x32b_x4(sf_t + 4 * c, v[c]);
-                            ptx::tc_store_32x32b_x4(sf_t + 16 + 8 * c, v[kSfChunksK + c]);
-                            ptx::tc_store_32x32b_x4(sf_t + 20 + 8 * c, v[2 * kSfChunksK + c]);
-                        }
-                        ptx::tc_wait_st();
-                        // the stage's next contents arrive through the async proxy: order these generic-proxy
-                        // reads of the scale tiles before it (the release chain to the producer starts here)
-                        ptx::fence_proxy_async_smem();
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (elected) ptx::mbar_arrive_cluster(ready0 + 8u * sf_buf);
-                    } else if (elected) {
-                        const uint32_t ssf = smem_base + stage * kStageBytes + kABytes + kBBytes;
-                        const uint32_t sf_t = tmem_base + kSfCol + sf_buf * kSfBufCols;
-                        // warp w: scale chunk w of the stage (NVFP4: the scales of MMA w; MXFP4: of MMAs 2w and
-                        // 2w+1) -- the A chunk, then the two B row chunks
-                        if (w < (kMx ? (nmma + 1) / 2 : nmma)) {
-                            ptx::tc_copy_sf_pair(sf_t + 4 * w, ptx::smem_desc_sf(ssf + w * 512));
-                            ptx::tc_copy_sf_pair(sf_t + 16 + 8 * w, ptx::smem_desc_sf(ssf + kSfaBytes + w * 512));
-                            ptx::tc_copy_sf_pair(sf_t + 20 + 8 * w,
-                                                 ptx::smem_desc_sf(ssf + kSfaBytes + kSfRowChunkBytes + w * 512));
-                        }
-                        ptx::tc_commit_pair(sf_ready_bar(sf_buf));
+                    for (int c = 0; c < kSfChunksK; ++c) {
+                        ptx::tc_store_32x32b_x4(sf_t + 4 * c, v[c]);
+                        ptx::tc_store_32x32b_x4(sf_t + 16 + 8 * c, v[kSfChunksK + c]);
+                        ptx::tc_store_32x32b_x4(sf_t + 20 + 8 * c, v[2 * kSfChunksK + c]);
                     }
+                    ptx::tc_wait_st();
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (elected) ptx::mbar_arrive_cluster(ready0 + 8u * sf_buf);
                     if (kTuning && (p.dbg & kDbgTrace) && w == 0 && leader) SOL_TRACE(5, gi);
                     ++gi;
                     if (++sf_buf == kSfBufs) sf_buf = 0;
@@ -569,8 +576,8 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                         old_stage = 0;
                         old_phase ^= 1u;
                     }
-                    if (++stage == kStages) {
-                        stage = 0;
+                    if (++slot == kSfSlots) {
+                        slot = 0;
                         phase ^= 1u;
                     }
                 }
@@ -608,7 +615,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sbias + lane * 8), "r"(bv.x), "r"(bv.y) : "memory");
                 __syncwarp();
             }
-            if (!wait_bounded(acc_full_bar(x), (static_cast<uint32_t>(it) >> 1) & 1u, abort_flag, p.status, 0x400u | x)) break;
+            if (!wait_site<8>(acc_full_bar(x), (static_cast<uint32_t>(it) >> 1) & 1u, abort_flag, p.status, 0x400u | x)) break;
             ptx::tc_fence_after_sync();
             if (kTuning && (p.dbg & kDbgTrace) && warp == 2) SOL_TRACE(9, it);
             const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + x * kAccStride;
