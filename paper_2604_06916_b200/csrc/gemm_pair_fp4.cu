@@ -1,23 +1,20 @@
-// NVFP4 CTA-pair GEMM with 256 x 256 pair tiles (tcgen05.mma.cta_group::2, kind::mxf4nvf4).
+// NVFP4 / MXFP4 CTA-pair GEMM with 256 x 256 pair tiles (tcgen05.mma.cta_group::2, kind::mxf4nvf4 / kind::mxf4).
 //
-// Why this shape: one MMA instruction costs its issuing thread 60-70 cycles and a k-tile needs
-// about 250 more for barrier polling and the commit, so the single MMA-issuing thread spends
-// ~500 cycles per k-tile of four MMAs.  Only at N = 256 does the tensor core need that long
-// (4 x 128 cycles); narrower tiles leave it idle.  N = 256 also has the lowest L2 -> SM traffic
-// per flop (38 KB per CTA per k-tile = 74 B/clk, against the SM's 128 B/clk ingest port).
+// Why this shape: one MMA instruction costs its issuing thread ~50 cycles and a k-tile needs ~250 more
+// for the commit, the look at the next stage's barriers and the loop, so the single MMA-issuing thread
+// spends ~450-520 cycles per k-tile of four MMAs.  Only at N = 256 does the tensor core need that long
+// (4 x 128 cycles); narrower tiles leave it idle.  N = 256 also has the lowest L2 -> SM traffic per flop.
 //
 // TMEM does not hold two 256-column accumulators plus the scale factors, so the two accumulators
 // overlap: A = columns [0,256), B = [96,352), scale-factor buffers 3 x 48 columns at [352,496).
 // Tiles alternate between A and B.  The epilogue drains the shared columns [96,256) first and
 // signals `ovl_free`; the MMAs of the next tile start then, while the rest of the tile is still
 // being converted and stored.  Eight epilogue warps (two per TMEM lane quadrant) shorten that wait.
-// Three scale-factor buffers are needed, not two: tcgen05.cp executes in the tensor pipe in issue
-// order, so a copy for k-tile i that must wait for the MMAs of k-tile i-2 lands behind the MMAs of
-// k-tile i-1 and k-tile i cannot be issued until those have run -- a bubble on every k-tile.
 //
-// Warps per CTA: 0 = TMA producer (A, B); 1 = TMEM owner, MMA issuer in the even CTA;
-// 2..9 = epilogue; 10..13 = scale-factor copy warps (even CTA; tcgen05.cp blocks its warp for
-// ~100 cycles, so the copies stay off the MMA thread); 14 = TMA producer (scales).
+// Warps per CTA: 0 = TMA producer (A, B: five stages of 32 KB); 1 = TMEM owner, MMA issuer in the even
+// CTA; 2..9 = epilogue; 10..13 = scale-factor copy warps, one per TMEM lane quadrant, in both CTAs
+// (shared memory -> registers -> tcgen05.st); 14 = TMA producer of the scale tiles, which travel in a
+// ring of their own (five slots of 6 KB) that runs ahead of the A / B ring.
 // No multicast loads; every mbarrier wait is bounded.
 #include "gemm_common.cuh"
 #include "quant_math.cuh"

@@ -220,3 +220,18 @@ def test_replica_aggregation_without_a_process_group():
     from paper_2604_06916_b200 import replicas
 
     assert replicas.aggregate(3.0, 7.0) == (3.0, 7.0, 1)
+
+
+def test_diagnostic_build_of_the_gemm_kernels_compiles(tmp_path):
+    """The timeline / drop-one-part switches of the GEMM and attention kernels are compiled in only with
+    -DSOL_TUNING; the product never builds them, so this keeps that configuration from rotting."""
+    import shutil
+    import subprocess
+
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    if not os.path.exists(nvcc):
+        pytest.skip("nvcc not available")
+    csrc = os.path.join(ROOT, "paper_2604_06916_b200", "csrc")
+    for src in ("gemm_pair_fp4.cu", "gemm_pair.cu", "gemm.cu", "attention.cu"):
+        subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-DSOL_TUNING", "-c",
+                        "-o", str(tmp_path / (src + ".o")), os.path.join(csrc, src)], check=True)
