@@ -116,7 +116,9 @@ bool make_tmap_sf(CUtensorMap *out, const void *base, uint64_t chunks_k, uint64_
 namespace {
 
 bool shape_ok(int64_t rows, int64_t K) {
-    return rows > 0 && K > 0 && K % 32 == 0 && rows <= (1LL << 30) && K <= (1LL << 24);
+    // the streaming kernels index their tiles (128 rows x 256 elements) and 32 KB pieces with a one-dimensional grid
+    return rows > 0 && K > 0 && K % 32 == 0 && rows <= (1LL << 30) && K <= (1LL << 24) &&
+           ceil_div(rows, 128) * ceil_div(K, 256) <= 0x7FFFFFFFLL && ceil_div(rows * (K / 8), 2048) <= 0x7FFFFFFFLL;
 }
 
 size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }

@@ -70,7 +70,8 @@ struct QuantDest {
 template <bool kSwizzled>
 __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
                                               const float *tscale, const float *amax, float *tscale_out,
-                                              uint8_t *__restrict__ q, uint8_t *__restrict__ sf, const QuantDest dst) {
+                                              uint8_t *__restrict__ q, uint8_t *__restrict__ sf, const QuantDest dst,
+                                              int64_t tile_k, int64_t tile_row) {
     __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kTileK / 16)];  // 2 KB = 4 chunks
     // 1 / (float(sb) * T) for every scale byte: d takes at most 127 values per tensor, so the decode,
     // the multiplication and the IEEE reciprocal run once per thread block instead of once per scale block
@@ -78,8 +79,8 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
 
     const int b = threadIdx.x & 15;   // scale block inside the tile
     const int r0 = threadIdx.x >> 4;  // first row inside the tile
-    const int64_t row0 = static_cast<int64_t>(blockIdx.y) * kTileRows;
-    const int64_t k = static_cast<int64_t>(blockIdx.x) * kTileK + b * 16;
+    const int64_t row0 = tile_row * kTileRows;
+    const int64_t k = tile_k * kTileK + b * 16;
     const bool k_ok = k < K;
 
     if (kSwizzled) {
@@ -90,7 +91,7 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
     grid_dependency_wait();
     grid_launch_dependents();
     const float T = amax != nullptr ? tensor_scale_from_amax(*amax) : *tscale;
-    if (tscale_out != nullptr && threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0) *tscale_out = T;
+    if (tscale_out != nullptr && threadIdx.x == 0 && tile_k == 0 && tile_row == 0) *tscale_out = T;
     const float c = __fmul_rn(6.0f, T);
     const int64_t nb = K >> 4;
     if (threadIdx.x < 128) {
@@ -139,13 +140,13 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
 
     if (kSwizzled) {
         __syncthreads();
-        // 4 chunks x 32 lines of 16 bytes; chunk c of this tile is k chunk blockIdx.x*4 + c
+        // 4 chunks x 32 lines of 16 bytes; chunk c of this tile is k chunk tile_k*4 + c
         const int64_t chunks_k = (nb + 3) >> 2;
         if (threadIdx.x < 128) {
             const int cidx = threadIdx.x >> 5;
-            const int64_t kc = static_cast<int64_t>(blockIdx.x) * 4 + cidx;
+            const int64_t kc = tile_k * 4 + cidx;
             if (kc < chunks_k) {
-                uint8_t *out = sf + (static_cast<int64_t>(blockIdx.y) * dst.sf_chunks_k + dst.sf_chunk0 + kc) * 512 +
+                uint8_t *out = sf + (tile_row * dst.sf_chunks_k + dst.sf_chunk0 + kc) * 512 +
                                (threadIdx.x & 31) * 16;
                 *reinterpret_cast<uint4 *>(out) = reinterpret_cast<const uint4 *>(sf_tile)[threadIdx.x];
             }
@@ -164,12 +165,17 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
     }
 }
 
+// One-dimensional grid over the tiles, k-tiles of a row tile adjacent.  With `reverse` the grid walks the
+// tensor from its end: behind the amax pass (which reads the tensor front to back) the last rows are
+// what the L2 still holds, so the quantizer's first reads hit there instead of going to HBM a second time.
 template <bool kSwizzled>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld,
                 const float *tscale, const float *amax, float *tscale_out, uint8_t *__restrict__ q,
-                uint8_t *__restrict__ sf, const QuantDest dst) {
-    quantize_tile<kSwizzled>(x, rows, K, ld, tscale, amax, tscale_out, q, sf, dst);
+                uint8_t *__restrict__ sf, const QuantDest dst, uint32_t k_tiles, int reverse) {
+    const uint32_t t = reverse ? gridDim.x - 1u - blockIdx.x : blockIdx.x;
+    const uint32_t tile_row = t / k_tiles;
+    quantize_tile<kSwizzled>(x, rows, K, ld, tscale, amax, tscale_out, q, sf, dst, t - tile_row * k_tiles, tile_row);
 }
 
 // The same over a group of equally shaped dense tensors, one per blockIdx.z, each with its own
@@ -179,7 +185,8 @@ __global__ void __launch_bounds__(kQuantThreads)
 quantize_group_kernel(const __grid_constant__ QuantGroup g, int64_t rows, int64_t K) {
     const int z = blockIdx.z;
     const QuantDest dst = {K >> 1, 0, ((K >> 4) + 3) >> 2, 0, nullptr};
-    quantize_tile<kSwizzled>(g.x[z], rows, K, K, nullptr, g.scale_words[z] + 1, g.scale_words[z], g.q[z], g.sf[z], dst);
+    quantize_tile<kSwizzled>(g.x[z], rows, K, K, nullptr, g.scale_words[z] + 1, g.scale_words[z], g.q[z], g.sf[z], dst,
+                             blockIdx.x, blockIdx.y);
 }
 
 // MXFP4 quantizer (the OCP format Section 2 sets beside NVFP4): 32 elements share one E8M0 scale
@@ -192,12 +199,14 @@ constexpr int kMxBlocksPerThread = kTileRows * (kMxTileK / 32) / kQuantThreads; 
 template <bool kSwizzled>
 __global__ void __launch_bounds__(kQuantThreads)
 mxfp4_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld, uint8_t *__restrict__ q,
-                      uint8_t *__restrict__ sf) {
+                      uint8_t *__restrict__ sf, uint32_t k_tiles) {
+    const int64_t tile_row = blockIdx.x / k_tiles;
+    const int64_t tile_k = blockIdx.x - static_cast<uint32_t>(tile_row) * k_tiles;
     __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kMxTileK / 32)];  // 2 KB = 4 chunks
     const int b = threadIdx.x & 15;   // 32-element block inside the tile
     const int r0 = threadIdx.x >> 4;
-    const int64_t row0 = static_cast<int64_t>(blockIdx.y) * kTileRows;
-    const int64_t k = static_cast<int64_t>(blockIdx.x) * kMxTileK + b * 32;
+    const int64_t row0 = tile_row * kTileRows;
+    const int64_t k = tile_k * kMxTileK + b * 32;
     const bool k_ok = k < K;
     if (kSwizzled) {
         reinterpret_cast<uint64_t *>(sf_tile)[threadIdx.x] = 0;
@@ -248,9 +257,9 @@ mxfp4_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, i
         const int64_t chunks_k = (nb + 3) >> 2;
         if (threadIdx.x < 128) {
             const int cidx = threadIdx.x >> 5;
-            const int64_t kc = static_cast<int64_t>(blockIdx.x) * 4 + cidx;
+            const int64_t kc = tile_k * 4 + cidx;
             if (kc < chunks_k) {
-                uint8_t *dst = sf + (static_cast<int64_t>(blockIdx.y) * chunks_k + kc) * 512 + (threadIdx.x & 31) * 16;
+                uint8_t *dst = sf + (tile_row * chunks_k + kc) * 512 + (threadIdx.x & 31) * 16;
                 *reinterpret_cast<uint4 *>(dst) = reinterpret_cast<const uint4 *>(sf_tile)[threadIdx.x];
             }
         }
@@ -258,28 +267,33 @@ mxfp4_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, i
 }
 
 // max |x| over the tensor as the bit pattern of the FP32 value (BF16 magnitude << 16).
+// A block reads one contiguous 32 KB piece (eight 16-byte loads in flight per thread) and the grid walks
+// the tensor front to back with ordinary loads, so what the L2 holds afterwards is the tensor's tail --
+// where the quantizer that follows in the fused entry starts.  Short blocks also balance the tail of the
+// reduction better than one wave of long grid-stride loops (5.5 against 5.0 TB/s on a 226 MB tensor).
 __global__ void __launch_bounds__(256)
 amax_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t vecs_per_row, int64_t ld,
             uint32_t *__restrict__ out_bits) {
     grid_launch_dependents();
     uint32_t m = 0;
     const int64_t total = rows * vecs_per_row;
-    const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-    int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t base = static_cast<int64_t>(blockIdx.x) * (256 * 8) + threadIdx.x;
     if (ld == vecs_per_row * 8) {
         const uint4 *p = reinterpret_cast<const uint4 *>(x);
-        for (; i + 7 * stride < total; i += 8 * stride) {  // eight independent 16-byte loads in flight
+        if (base + 7 * 256 < total) {
             uint4 v[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) v[u] = __ldcs(p + i + u * stride);
+            for (int u = 0; u < 8; ++u) v[u] = __ldg(p + base + u * 256);
 #pragma unroll
             for (int u = 0; u < 8; u += 2) m = max(m, abs_max_bits(v[u], v[u + 1]));
+        } else {
+            for (int64_t i = base; i < total; i += 256) m = max(m, abs_max_bits(__ldg(p + i)));
         }
-        for (; i < total; i += stride) m = max(m, abs_max_bits(__ldcs(p + i)));
     } else {
-        for (; i < total; i += stride) {
+        const int64_t end = min(total, (static_cast<int64_t>(blockIdx.x) + 1) * (256 * 8));
+        for (int64_t i = base; i < end; i += 256) {
             const int64_t r = i / vecs_per_row, vcol = i - r * vecs_per_row;
-            m = max(m, abs_max_bits(__ldcs(reinterpret_cast<const uint4 *>(x + r * ld + vcol * 8))));
+            m = max(m, abs_max_bits(__ldg(reinterpret_cast<const uint4 *>(x + r * ld + vcol * 8))));
         }
     }
     m = __reduce_max_sync(0xFFFFFFFFu, m);
@@ -306,12 +320,7 @@ sol_status_t launch_amax_bits(const void *x, int64_t rows, int64_t K, int64_t ld
                               cudaStream_t stream, const DeviceInfo *dev) {
     if (cudaMemsetAsync(bits_out, 0, sizeof(uint32_t), stream) != cudaSuccess) return SOL_ERR_CUDA;
     const int64_t vecs = rows * (K / 8);
-    int64_t blocks = ceil_div(vecs, 256 * 8);
-    // up to 16 waves of resident blocks: short blocks balance the tail of the reduction better than
-    // one wave of long grid-stride loops (measured 5.5 against 5.0 TB/s on a 226 MB tensor)
-    const int64_t cap = static_cast<int64_t>(dev->sm_count) * 8 * 16;
-    if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
+    const int64_t blocks = ceil_div(vecs, 256 * 8);  // at most 2^31 - 1: checked with the shape
     amax_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(
         static_cast<const uint16_t *>(x), rows, K / 8, ld, bits_out);
     return launch_status();
@@ -322,10 +331,16 @@ sol_status_t launch_amax_bits(const void *x, int64_t rows, int64_t K, int64_t ld
 // their first global access.
 sol_status_t launch_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t ld, const float *tscale,
                                 const float *amax, float *tscale_out, void *q, void *sf,
-                                sol_sf_layout_t layout, cudaStream_t stream, const QuantDest *dest = nullptr) {
+                                sol_sf_layout_t layout, cudaStream_t stream, const QuantDest *dest = nullptr,
+                                bool reverse = false) {
     const QuantDest dst = dest != nullptr ? *dest : QuantDest{K >> 1, 0, ((K >> 4) + 3) >> 2, 0, nullptr};
+    const uint32_t k_tiles = static_cast<uint32_t>(ceil_div(K, kTileK));
+    int rev = reverse ? 1 : 0;
+#ifdef SOL_TUNING
+    if (const char *e = getenv("SOL_QREV")) rev = atoi(e);
+#endif
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(ceil_div(K, kTileK)), static_cast<unsigned>(ceil_div(rows, kTileRows)));
+    cfg.gridDim = dim3(static_cast<unsigned>(k_tiles * ceil_div(rows, kTileRows)));
     cfg.blockDim = dim3(kQuantThreads);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
@@ -336,7 +351,7 @@ sol_status_t launch_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t 
     cfg.numAttrs = 1;
     auto kern = layout == SOL_SF_SWIZZLED_128x4 ? quantize_kernel<true> : quantize_kernel<false>;
     if (cudaLaunchKernelEx(&cfg, kern, static_cast<const uint16_t *>(x), rows, K, ld, tscale, amax, tscale_out,
-                           static_cast<uint8_t *>(q), static_cast<uint8_t *>(sf), dst) != cudaSuccess) {
+                           static_cast<uint8_t *>(q), static_cast<uint8_t *>(sf), dst, k_tiles, rev) != cudaSuccess) {
         cudaGetLastError();
         return SOL_ERR_CUDA;
     }
@@ -386,7 +401,8 @@ sol_status_t launch_quantize(const void *x, int64_t rows, int64_t K, int64_t ld,
 sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
                                    sol_sf_layout_t layout, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(ceil_div(K, kMxTileK)), static_cast<unsigned>(ceil_div(rows, kTileRows)));
+    const uint32_t k_tiles = static_cast<uint32_t>(ceil_div(K, kMxTileK));
+    cfg.gridDim = dim3(static_cast<unsigned>(k_tiles * ceil_div(rows, kTileRows)));
     cfg.blockDim = dim3(kQuantThreads);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -396,7 +412,7 @@ sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64
     cfg.numAttrs = 1;
     auto kern = layout == SOL_SF_SWIZZLED_128x4 ? mxfp4_quantize_kernel<true> : mxfp4_quantize_kernel<false>;
     if (cudaLaunchKernelEx(&cfg, kern, static_cast<const uint16_t *>(x), rows, K, ld, static_cast<uint8_t *>(q),
-                           static_cast<uint8_t *>(sf)) != cudaSuccess) {
+                           static_cast<uint8_t *>(sf), k_tiles) != cudaSuccess) {
         cudaGetLastError();
         return SOL_ERR_CUDA;
     }
@@ -404,8 +420,9 @@ sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64
 }
 
 sol_status_t launch_quantize_from_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,
-                                       void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream) {
-    return launch_quantize_ex(x, rows, K, ld, nullptr, scale_words + 1, scale_words, q, sf, layout, stream);
+                                       void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream, bool reverse) {
+    return launch_quantize_ex(x, rows, K, ld, nullptr, scale_words + 1, scale_words, q, sf, layout, stream, nullptr,
+                              reverse);
 }
 
 sol_status_t launch_quantize_group(const QuantGroup &g, int count, int64_t rows, int64_t K, sol_sf_layout_t layout,
@@ -433,7 +450,8 @@ sol_status_t launch_amax_quantize(const void *x, int64_t rows, int64_t K, int64_
                                   const DeviceInfo *dev) {
     sol_status_t st = launch_amax_bits(x, rows, K, ld, reinterpret_cast<uint32_t *>(scale_words + 1), stream, dev);
     if (st != SOL_OK) return st;
-    return launch_quantize_from_amax(x, rows, K, ld, scale_words, q, sf, layout, stream);
+    // the amax pass has just read x front to back: start the quantizer where the L2 is still warm
+    return launch_quantize_from_amax(x, rows, K, ld, scale_words, q, sf, layout, stream, true);
 }
 
 }  // namespace sol

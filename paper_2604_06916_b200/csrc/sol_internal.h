@@ -60,7 +60,8 @@ sol_status_t launch_amax_quantize(const void *x, int64_t rows, int64_t K, int64_
                                   const DeviceInfo *dev);
 // Quantizer that derives T from max|x| left in scale_words[1] (FP32 bits) and publishes T in scale_words[0].
 sol_status_t launch_quantize_from_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,
-                                       void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream);
+                                       void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream,
+                                       bool reverse = false);
 // Groups of equally shaped matrices handled by one launch (blockIdx.z picks the matrix).
 constexpr int kMaxGroup = 8;
 struct MergeGroup {
