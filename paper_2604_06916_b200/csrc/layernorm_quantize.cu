@@ -50,7 +50,7 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
                           int64_t rows_per_sample, float eps, const float *__restrict__ tscale,
                           uint8_t *__restrict__ q, uint8_t *__restrict__ sf, uint32_t *amax_track,
                           uint32_t *status) {
-    // (1 + scale, shift) of this block's sample for element pairs, laid out [pair within block][block] so
+    // (1 + scale) x 2, shift x 2 of this block's sample for element pairs, laid out [pair within block][block] so
     // that the 32 lanes of a warp (consecutive blocks) read consecutive 16-byte words; behind it the row
     // ring (two slots of K BF16 per warp)
     extern __shared__ __align__(16) float4 mod[];
@@ -69,7 +69,7 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
         const uint32_t sc = __ldg(reinterpret_cast<const uint32_t *>(scale + sample * K) + k2);
         const uint32_t sh = __ldg(reinterpret_cast<const uint32_t *>(shift + sample * K) + k2);
         mod[(k2 & 7) * nblocks + (k2 >> 3)] =
-            make_float4(1.0f + qmath::bf16_lo(sc), qmath::bf16_lo(sh), 1.0f + qmath::bf16_hi(sc), qmath::bf16_hi(sh));
+            make_float4(1.0f + qmath::bf16_lo(sc), 1.0f + qmath::bf16_hi(sc), qmath::bf16_lo(sh), qmath::bf16_hi(sh));
     }
     __syncthreads();
 
@@ -140,19 +140,24 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
         // sum (x - p) and sum (x - p)^2 lose no accuracy to cancellation as long as p lies within the data,
         // and the two warp reductions run side by side instead of one after the other
         const float pivot = __shfl_sync(0xFFFFFFFFu, qmath::bf16_lo(w[0][0]), 0);
-        float s2 = 0.0f;
+        const uint64_t npivot2 = qmath::f32x2(-pivot, -pivot);
+        uint64_t s1_2 = 0, s2_2 = 0;   // two lanes of 0.0f
 #pragma unroll
         for (int i = 0; i < kBlocksPerLane; ++i) {
             if (lane + 32 * i < nblocks) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float d0 = qmath::bf16_lo(w[i][e]) - pivot, d1 = qmath::bf16_hi(w[i][e]) - pivot;
-                    s1 += d0 + d1;
-                    s2 = fmaf(d0, d0, s2);
-                    s2 = fmaf(d1, d1, s2);
+                    const uint64_t d2 = qmath::add2(qmath::f32x2_of_bf16x2(w[i][e]), npivot2);
+                    s1_2 = qmath::add2(s1_2, d2);
+                    s2_2 = qmath::fma2(d2, d2, s2_2);
                 }
             }
         }
+        float s2, s1b, s2b;
+        qmath::f32x2_split(s1_2, s1, s1b);
+        qmath::f32x2_split(s2_2, s2, s2b);
+        s1 += s1b;
+        s2 += s2b;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
@@ -163,6 +168,7 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
         const float var = fmaxf(fmaf(-dm, dm, s2 * inv_k), 0.0f);
         const float rstd = 1.0f / sqrtf(var + eps);
         const float nmr = -mu * rstd;   // xhat = fma(x, rstd, -mu * rstd)
+        const uint64_t rstd2 = qmath::f32x2(rstd, rstd), nmr2 = qmath::f32x2(nmr, nmr);
         const int64_t row_tile = r >> 7;
         const int rr = static_cast<int>(r & 127);
         uint8_t *sf_row = sf + row_tile * chunks_k * 512 + (rr & 31) * 16 + (rr >> 5) * 4;
@@ -177,9 +183,10 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
                 uint32_t bm = 0;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const float4 m = mp[e * nblocks];   // (1 + scale, shift) of two neighbouring elements
-                    const float y0 = fmaf(fmaf(qmath::bf16_lo(w[i][e]), rstd, nmr), m.x, m.y);
-                    const float y1 = fmaf(fmaf(qmath::bf16_hi(w[i][e]), rstd, nmr), m.z, m.w);
+                    const float4 m = mp[e * nblocks];   // (1 + scale) and shift of two neighbouring elements
+                    const uint64_t xh2 = qmath::fma2(qmath::f32x2_of_bf16x2(w[i][e]), rstd2, nmr2);
+                    float y0, y1;
+                    qmath::f32x2_split(qmath::fma2(xh2, qmath::f32x2(m.x, m.y), qmath::f32x2(m.z, m.w)), y0, y1);
                     hw[e] = pack_bf16x2(y0, y1);
                     bm = qmath::absmax2(bm, hw[e]);
                 }
@@ -189,17 +196,14 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
                 const float a = __uint_as_float(abits << 16);
                 sb = qmath::f32_to_e4m3_sat(__fdiv_rn(a, c6T));
                 const float rcp = rcp_tab[sb];
+                const uint64_t rcp2 = qmath::f32x2(rcp, rcp);
                 uint2 packed;
-                packed.x = qmath::quantize8(hw[0], hw[1], hw[2], hw[3], rcp);
-                packed.y = qmath::quantize8(hw[4], hw[5], hw[6], hw[7], rcp);
+                packed.x = qmath::quantize8_x2(hw[0], hw[1], hw[2], hw[3], rcp2);
+                packed.y = qmath::quantize8_x2(hw[4], hw[5], hw[6], hw[7], rcp2);
                 __stcs(reinterpret_cast<uint2 *>(q + r * (K >> 1) + b * 8), packed);
             }
-            // four neighbouring lanes hold the four scale bytes of one (row, chunk) slot: one 4-byte store
-            uint32_t word = sb;
-            word |= __shfl_down_sync(0xFFFFFFFFu, sb, 1) << 8;
-            word |= __shfl_down_sync(0xFFFFFFFFu, sb, 2) << 16;
-            word |= __shfl_down_sync(0xFFFFFFFFu, sb, 3) << 24;
-            if ((lane & 3) == 0 && b < nblocks) *reinterpret_cast<uint32_t *>(sf_row + (b >> 2) * 512) = word;
+            // the lane's scale byte of its (row, chunk) slot (four neighbouring lanes fill one 4-byte slot)
+            if (b < nblocks) sf_row[(b >> 2) * 512 + (b & 3)] = static_cast<uint8_t>(sb);
         }
     }
     // rows past M inside the last 128-row scale chunk are padding and read as 0 (first block only)

@@ -51,6 +51,43 @@ __device__ __forceinline__ uint32_t quantize8(uint32_t w0, uint32_t w1, uint32_t
                        __fmul_rn(bf16_lo(w3), rcp), __fmul_rn(bf16_hi(w3), rcp));
 }
 
+// Two-lane FP32 arithmetic (one instruction for two IEEE operations, each rounded on its own: results
+// are bit for bit those of the scalar forms).  A pair lives in a 64-bit register, low lane first.
+__device__ __forceinline__ uint64_t f32x2(float lo, float hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ void f32x2_split(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f32x2_of_bf16x2(uint32_t w) { return f32x2(bf16_lo(w), bf16_hi(w)); }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// Eight packed BF16 values (four words) times rcp -> eight nibbles, the products taken two at a time.
+__device__ __forceinline__ uint32_t quantize8_x2(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, uint64_t rcp2) {
+    float y[8];
+    f32x2_split(mul2(f32x2_of_bf16x2(w0), rcp2), y[0], y[1]);
+    f32x2_split(mul2(f32x2_of_bf16x2(w1), rcp2), y[2], y[3]);
+    f32x2_split(mul2(f32x2_of_bf16x2(w2), rcp2), y[4], y[5]);
+    f32x2_split(mul2(f32x2_of_bf16x2(w3), rcp2), y[6], y[7]);
+    return pack_e2m1x8(y[0], y[1], y[2], y[3], y[4], y[5], y[6], y[7]);
+}
+
 // Block scale byte and reciprocal from the block's max magnitude a, c = 6 T and T.
 __device__ __forceinline__ uint32_t block_scale(float a, float c, float T, float &rcp) {
     const float sv = __fdiv_rn(a, c);
