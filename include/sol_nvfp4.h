@@ -374,6 +374,23 @@ sol_status_t mxfp4_linear_quantized_out(const void *xq, const void *xsf, const v
                                         float *amax_out, int64_t M, int64_t N, int64_t K, void *stream);
 
 /*
+ * The MXFP4 forms of nvfp4_linear_split_out and nvfp4_quantize_into (Section 2 names MXFP4 beside NVFP4;
+ * the concatenated input of a single-stream block's second linear, as there): columns [0, n_split) of the
+ * linear leave as BF16, columns [n_split, N) pass through the activation and leave as MXFP4 into columns
+ * [dest_col0, dest_col0 + N - n_split) of a wider MXFP4 tensor [M, dest_K]; mxfp4_quantize_into quantizes a
+ * BF16 tensor [M, K] into columns [dest_col0, dest_col0 + K) of such a tensor and touches no other column.
+ *   hq_dest / q_dest  packed nibbles [M, dest_K/2];  hsf_dest / sf_dest  chunked MXFP4 scales of an [M, dest_K] tensor
+ *   n_split % 256 == 0;  N - n_split, K, dest_K and dest_col0 multiples of 128 (a scale chunk spans 128 columns).
+ * No tensor scale: the format has none.  Errors as the NVFP4 forms.
+ */
+sol_status_t mxfp4_linear_split_out(const void *xq, const void *xsf, const void *wq, const void *wsf,
+                                    const void *bias_bf16, void *y_bf16, int64_t ldy, int64_t n_split,
+                                    sol_activation_t activation, void *hq_dest, void *hsf_dest, int64_t dest_K,
+                                    int64_t dest_col0, float *amax_out, int64_t M, int64_t N, int64_t K, void *stream);
+sol_status_t mxfp4_quantize_into(const void *x_bf16, int64_t M, int64_t K, int64_t ldx, void *q_dest, void *sf_dest,
+                                 int64_t dest_K, int64_t dest_col0, void *stream);
+
+/*
  * Stage-1 selection (Section 3.4; Section 4.1 "Rollout Generation": N = 96 candidates per prompt,
  * the 12 best and 12 worst kept, their initial noises preserved) and the group-standardised
  * advantages of the GRPO equation in Section 2, A_i = (R_i - mean) / population std.

@@ -27,6 +27,7 @@ EXPORTS = [
     "mxfp4_linear", "nvfp4_linear_split_out", "nvfp4_quantize_into",
     "nvfp4_quantize_linear_delayed", "sol_roll_tensor_scale", "nvfp4_layernorm_quantize", "sol_attention_bf16", "sol_attention_bf16_joint",
     "sol_attention_nvfp4_out", "mxfp4_linear_quantized_out", "sol_set_wait_limit_cycles", "sol_test_hold_loads",
+    "mxfp4_linear_split_out", "mxfp4_quantize_into",
 ]
 
 _lib = None
@@ -102,6 +103,10 @@ def lib() -> ctypes.CDLL:
     L.sol_attention_bf16.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, i64, i64, i64, i64, i64, vp]
     L.nvfp4_layernorm_quantize.restype = i32
     L.nvfp4_layernorm_quantize.argtypes = [vp, i64, i64, i64, vp, vp, i64, ctypes.c_float, vp, vp, vp, vp, vp]
+    L.mxfp4_linear_split_out.restype = i32
+    L.mxfp4_linear_split_out.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i32, vp, vp, i64, i64, vp, i64, i64, i64, vp]
+    L.mxfp4_quantize_into.restype = i32
+    L.mxfp4_quantize_into.argtypes = [vp, i64, i64, i64, vp, vp, i64, i64, vp]
     L.sol_set_wait_limit_cycles.restype, L.sol_set_wait_limit_cycles.argtypes = i32, [i64]
     L.sol_test_hold_loads.restype, L.sol_test_hold_loads.argtypes = i32, [i32]
     L.sol_last_device_status.restype = i32
@@ -446,6 +451,29 @@ def mxfp4_linear(xq, xsf, wq, wsf, bias=None, out: torch.Tensor | None = None):
     _check(lib().mxfp4_linear(_ptr(xq), _ptr(xsf), _ptr(wq), _ptr(wsf), _ptr(bias), _ptr(out), M, N, K, out.stride(0),
                               _stream()), "mxfp4_linear")
     return out
+
+
+def mxfp4_linear_split_out(xq, xsf, wq, wsf, bias, n_split: int, activation: int, dest, dest_col0: int,
+                           y_out: torch.Tensor | None = None, amax_out: torch.Tensor | None = None):
+    """Columns below n_split -> BF16 `y_out`; the rest -> activation -> MXFP4 into dest = (q [M, dest_K/2], sf)."""
+    M, K = xq.shape[0], xq.shape[1] * 2
+    N = wq.shape[0]
+    hq, hsf = dest
+    if y_out is None:
+        y_out = torch.empty((M, n_split), dtype=torch.bfloat16, device=xq.device)
+    _check(lib().mxfp4_linear_split_out(_ptr(xq), _ptr(xsf), _ptr(wq), _ptr(wsf), _ptr(bias), _ptr(y_out), y_out.stride(0),
+                                        n_split, activation, _ptr(hq), _ptr(hsf), hq.shape[1] * 2, dest_col0,
+                                        _ptr(amax_out), M, N, K, _stream()), "mxfp4_linear_split_out")
+    return y_out
+
+
+def mxfp4_quantize_into(x: torch.Tensor, dest, dest_col0: int):
+    """Quantize BF16 x [M, K] into columns [dest_col0, dest_col0 + K) of the MXFP4 tensor dest = (q, sf)."""
+    _need_2d_bf16(x, "x")
+    M, K = x.shape
+    hq, hsf = dest
+    _check(lib().mxfp4_quantize_into(_ptr(x), M, K, x.stride(0), _ptr(hq), _ptr(hsf), hq.shape[1] * 2, dest_col0,
+                                     _stream()), "mxfp4_quantize_into")
 
 
 def solrl_select_contrastive(rewards: torch.Tensor, K: int, seeds: torch.Tensor | None = None,

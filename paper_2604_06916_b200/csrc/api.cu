@@ -404,6 +404,45 @@ sol_status_t mxfp4_linear_quantized_out(const void *xq, const void *xsf, const v
                                                 static_cast<cudaStream_t>(stream), dev);
 }
 
+sol_status_t mxfp4_linear_split_out(const void *xq, const void *xsf, const void *wq, const void *wsf,
+                                    const void *bias_bf16, void *y_bf16, int64_t ldy, int64_t n_split,
+                                    sol_activation_t activation, void *hq_dest, void *hsf_dest, int64_t dest_K,
+                                    int64_t dest_col0, float *amax_out, int64_t M, int64_t N, int64_t K, void *stream) {
+    if (xq == nullptr || xsf == nullptr || wq == nullptr || wsf == nullptr || y_bf16 == nullptr || hq_dest == nullptr ||
+        hsf_dest == nullptr)
+        return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(M, K) || N <= 0 || N > (1LL << 24) || n_split <= 0 || n_split >= N || n_split % 256 != 0 ||
+        (N - n_split) % 128 != 0 || ldy < n_split || dest_K <= 0 || dest_K % 128 != 0 || dest_col0 < 0 ||
+        dest_col0 % 128 != 0 || dest_col0 + (N - n_split) > dest_K)
+        return SOL_ERR_BAD_SHAPE;
+    if (activation != SOL_ACT_NONE && activation != SOL_ACT_GELU_TANH) return SOL_ERR_BAD_LAYOUT;
+    if (!aligned16(xq) || !aligned16(xsf) || !aligned16(wq) || !aligned16(wsf) || !aligned16(y_bf16) ||
+        !aligned16(hq_dest) || !aligned16(hsf_dest) || ldy % 8 != 0 || (bias_bf16 != nullptr && !aligned16(bias_bf16)) ||
+        (reinterpret_cast<uintptr_t>(amax_out) & 3u))
+        return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return gemm::launch_pair256_mxfp4_split_out(xq, xsf, wq, wsf, bias_bf16, y_bf16, ldy, n_split,
+                                                activation == SOL_ACT_GELU_TANH ? 1 : 0, hq_dest, hsf_dest, dest_K,
+                                                dest_col0, reinterpret_cast<uint32_t *>(amax_out), M, N, K,
+                                                static_cast<cudaStream_t>(stream), dev);
+}
+
+sol_status_t mxfp4_quantize_into(const void *x_bf16, int64_t M, int64_t K, int64_t ldx, void *q_dest, void *sf_dest,
+                                 int64_t dest_K, int64_t dest_col0, void *stream) {
+    if (x_bf16 == nullptr || q_dest == nullptr || sf_dest == nullptr) return SOL_ERR_NULL_POINTER;
+    if (!shape_ok(M, K) || ldx < K || K % 128 != 0 || dest_K <= 0 || dest_K % 128 != 0 || dest_col0 < 0 ||
+        dest_col0 % 128 != 0 || dest_col0 + K > dest_K)
+        return SOL_ERR_BAD_SHAPE;
+    if (!aligned16(x_bf16) || !aligned16(q_dest) || !aligned16(sf_dest) || ldx % 8 != 0) return SOL_ERR_ALIGNMENT;
+    const DeviceInfo *dev = nullptr;
+    sol_status_t st = check_arch(&dev);
+    if (st != SOL_OK) return st;
+    return launch_mxfp4_quantize_into(x_bf16, M, K, ldx, q_dest, sf_dest, dest_K, dest_col0,
+                                      static_cast<cudaStream_t>(stream));
+}
+
 sol_status_t solrl_select_contrastive(const float *rewards, const uint64_t *seeds, int64_t P, int64_t N, int64_t K,
                                       int32_t *idx_out, uint64_t *seeds_out, float *advantages_out, void *stream) {
     if (rewards == nullptr || idx_out == nullptr || (seeds_out != nullptr && seeds == nullptr)) return SOL_ERR_NULL_POINTER;

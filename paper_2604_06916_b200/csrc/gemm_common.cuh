@@ -202,6 +202,10 @@ sol_status_t launch_pair256_mxfp4(const void *xq, const void *xsf, const void *w
 sol_status_t launch_pair256_mxfp4_quant_out(const void *xq, const void *xsf, const void *wq, const void *wsf,
                                             const void *bias, int act, void *hq, void *hsf, uint32_t *amax_out, int64_t M,
                                             int64_t N, int64_t K, cudaStream_t stream, const DeviceInfo *dev);
+sol_status_t launch_pair256_mxfp4_split_out(const void *xq, const void *xsf, const void *wq, const void *wsf,
+                                            const void *bias, void *y_bf16, int64_t ldy, int64_t n_split, int act,
+                                            void *hq, void *hsf, int64_t dest_K, int64_t dest_col0, uint32_t *amax_out,
+                                            int64_t M, int64_t N, int64_t K, cudaStream_t stream, const DeviceInfo *dev);
 sol_status_t launch_pair256_nvfp4(const void *xq, const void *xsf, const float *xts, const void *wq,
                                   const void *wsf, const float *wts, const void *bias, void *y, int64_t M,
                                   int64_t N, int64_t K, int64_t ldy, cudaStream_t stream, const DeviceInfo *dev);

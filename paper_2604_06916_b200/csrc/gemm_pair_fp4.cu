@@ -187,8 +187,8 @@ __device__ __forceinline__ void epilogue_quant_store(const CUtensorMap *tm_q, co
 // chunk's two scale bytes are one 2-byte store into the lower or upper half of a (row, chunk) slot.
 __device__ __forceinline__ void epilogue_quant_store_mx(const CUtensorMap *tm_q, const Params &p, const uint32_t (&lo)[32],
                                                         const uint32_t (&hi)[32], int m0, int quad_in_tile, int row_tile,
-                                                        int nc, float alpha, uint32_t sbuf, uint32_t sbias, int lane,
-                                                        uint32_t &amax2) {
+                                                        int nc, int nc_dst, float alpha, uint32_t sbuf, uint32_t sbias,
+                                                        int lane, uint32_t &amax2) {
     const bool gelu = p.act != 0;
     if (lane == 0) ptx::tma_store_wait_read<0>();
     __syncwarp();
@@ -237,14 +237,14 @@ __device__ __forceinline__ void epilogue_quant_store_mx(const CUtensorMap *tm_q,
     const bool unit_ok = nc < p.N && !(kTuning && (p.dbg & kDbgNoStore));
     if (unit_ok && row_tile * 128 < p.M) {
         if (m0 + lane >= p.M) sfw = 0;  // rows past M inside the last 128-row chunk are padding and read as 0
-        const int64_t chunk = static_cast<int64_t>(row_tile) * p.dest_chunks_k + (nc >> 7);
-        *reinterpret_cast<uint16_t *>(p.sf_out + chunk * 512 + lane * 16 + quad_in_tile * 4 + ((nc >> 6) & 1) * 2) =
+        const int64_t chunk = static_cast<int64_t>(row_tile) * p.dest_chunks_k + (nc_dst >> 7);
+        *reinterpret_cast<uint16_t *>(p.sf_out + chunk * 512 + lane * 16 + quad_in_tile * 4 + ((nc_dst >> 6) & 1) * 2) =
             static_cast<uint16_t>(sfw);
     }
     ptx::fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) {
-        if (unit_ok && m0 < p.M) ptx::tma_store_2d(tm_q, nc >> 1, m0, sbuf);
+        if (unit_ok && m0 < p.M) ptx::tma_store_2d(tm_q, nc_dst >> 1, m0, sbuf);
         ptx::tma_store_commit();
     }
 }
@@ -648,8 +648,8 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             if (as_bf16)
                 epilogue_store(&tm_y, p, a_lo, a_hi, m0, n0 + first * 64, alpha, sbuf, sbias, lane);
             else if constexpr (kMx)
-                epilogue_quant_store_mx(&tm_q, p, a_lo, a_hi, m0, quad, row_tile, n0 + first * 64, alpha, sbuf, sbias, lane,
-                                        amax2);
+                epilogue_quant_store_mx(&tm_q, p, a_lo, a_hi, m0, quad, row_tile, n0 + first * 64,
+                                        n0 + first * 64 + dst_shift, alpha, sbuf, sbias, lane, amax2);
             else
                 epilogue_quant_store(&tm_q, p, a_lo, a_hi, m0, quad, row_tile, n0 + first * 64,
                                      n0 + first * 64 + dst_shift, alpha, Tq, c6T, sbuf, sbias, lane, amax2);
@@ -666,11 +666,11 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     epilogue_store(&tm_y, p, b_sh, b_ot, m0, n0 + second * 64, alpha, sbuf, sbias + 128, lane);
             } else if constexpr (kMx) {
                 if (x == 0)
-                    epilogue_quant_store_mx(&tm_q, p, b_ot, b_sh, m0, quad, row_tile, n0 + second * 64, alpha, sbuf,
-                                            sbias + 128, lane, amax2);
+                    epilogue_quant_store_mx(&tm_q, p, b_ot, b_sh, m0, quad, row_tile, n0 + second * 64,
+                                            n0 + second * 64 + dst_shift, alpha, sbuf, sbias + 128, lane, amax2);
                 else
-                    epilogue_quant_store_mx(&tm_q, p, b_sh, b_ot, m0, quad, row_tile, n0 + second * 64, alpha, sbuf,
-                                            sbias + 128, lane, amax2);
+                    epilogue_quant_store_mx(&tm_q, p, b_sh, b_ot, m0, quad, row_tile, n0 + second * 64,
+                                            n0 + second * 64 + dst_shift, alpha, sbuf, sbias + 128, lane, amax2);
             } else {
                 if (x == 0)
                     epilogue_quant_store(&tm_q, p, b_ot, b_sh, m0, quad, row_tile, n0 + second * 64,
@@ -757,12 +757,14 @@ sol_status_t launch_pair256(int out_mode, bool mx, const void *xq, const void *x
 #ifdef SOL_TUNING
     if (const char *e = getenv("SOL_DBG")) p.dbg = static_cast<uint32_t>(atoi(e));
 #endif
-    auto kern = mx ? (out_mode == kOutQuant ? gemm_pair_fp4_kernel<kOutQuant, true> : gemm_pair_fp4_kernel<kOutBf16, true>)
+    auto kern = mx ? (out_mode == kOutBf16    ? gemm_pair_fp4_kernel<kOutBf16, true>
+                      : out_mode == kOutQuant ? gemm_pair_fp4_kernel<kOutQuant, true>
+                                              : gemm_pair_fp4_kernel<kOutSplit, true>)
                 : out_mode == kOutBf16 ? gemm_pair_fp4_kernel<kOutBf16, false>
                 : out_mode == kOutQuant ? gemm_pair_fp4_kernel<kOutQuant, false>
                                         : gemm_pair_fp4_kernel<kOutSplit, false>;
-    static bool configured[5][64] = {};
-    const int slot = mx ? (out_mode == kOutQuant ? 4 : 3) : out_mode;
+    static bool configured[6][64] = {};
+    const int slot = (mx ? 3 : 0) + out_mode;
     if (dev->device < 64 && !configured[slot][dev->device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return SOL_ERR_CUDA;
@@ -822,6 +824,21 @@ sol_status_t launch_pair256_mxfp4_quant_out(const void *xq, const void *xsf, con
     qo.amax_out = amax_out;
     qo.dest_K = N;
     return launch_pair256(kOutQuant, true, xq, xsf, nullptr, wq, wsf, nullptr, bias, nullptr, 0, qo, M, N, K, stream, dev);
+}
+
+sol_status_t launch_pair256_mxfp4_split_out(const void *xq, const void *xsf, const void *wq, const void *wsf,
+                                            const void *bias, void *y_bf16, int64_t ldy, int64_t n_split, int act,
+                                            void *hq, void *hsf, int64_t dest_K, int64_t dest_col0, uint32_t *amax_out,
+                                            int64_t M, int64_t N, int64_t K, cudaStream_t stream, const DeviceInfo *dev) {
+    QuantOut qo;
+    qo.act = act;
+    qo.hq = hq;
+    qo.hsf = hsf;
+    qo.amax_out = amax_out;
+    qo.n_split = n_split;
+    qo.dest_K = dest_K;
+    qo.dest_col0 = dest_col0;
+    return launch_pair256(kOutSplit, true, xq, xsf, nullptr, wq, wsf, nullptr, bias, y_bf16, ldy, qo, M, N, K, stream, dev);
 }
 
 sol_status_t launch_pair256_nvfp4_quant_out(const void *xq, const void *xsf, const float *xts, const void *wq,

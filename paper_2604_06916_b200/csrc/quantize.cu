@@ -199,7 +199,7 @@ constexpr int kMxBlocksPerThread = kTileRows * (kMxTileK / 32) / kQuantThreads; 
 template <bool kSwizzled>
 __global__ void __launch_bounds__(kQuantThreads)
 mxfp4_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, int64_t ld, uint8_t *__restrict__ q,
-                      uint8_t *__restrict__ sf, uint32_t k_tiles) {
+                      uint8_t *__restrict__ sf, uint32_t k_tiles, const QuantDest dst) {
     const int64_t tile_row = blockIdx.x / k_tiles;
     const int64_t tile_k = blockIdx.x - static_cast<uint32_t>(tile_row) * k_tiles;
     __shared__ __align__(16) uint8_t sf_tile[kTileRows * (kMxTileK / 32)];  // 2 KB = 4 chunks
@@ -243,7 +243,7 @@ mxfp4_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, i
             packed.z = quantize8(v[i][2], inv);
             packed.w = quantize8(v[i][3], inv);
             if (k_ok && r < rows) {
-                __stcs(reinterpret_cast<uint4 *>(q + r * (K >> 1) + (k >> 1)), packed);
+                __stcs(reinterpret_cast<uint4 *>(q + r * dst.q_pitch + dst.q_col0 + (k >> 1)), packed);
                 if (kSwizzled) {
                     sf_tile[(b >> 2) * 512 + (rl & 31) * 16 + (rl >> 5) * 4 + (b & 3)] = static_cast<uint8_t>(sb);
                 } else {
@@ -259,8 +259,8 @@ mxfp4_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int64_t K, i
             const int cidx = threadIdx.x >> 5;
             const int64_t kc = tile_k * 4 + cidx;
             if (kc < chunks_k) {
-                uint8_t *dst = sf + (tile_row * chunks_k + kc) * 512 + (threadIdx.x & 31) * 16;
-                *reinterpret_cast<uint4 *>(dst) = reinterpret_cast<const uint4 *>(sf_tile)[threadIdx.x];
+                uint8_t *out = sf + (tile_row * dst.sf_chunks_k + dst.sf_chunk0 + kc) * 512 + (threadIdx.x & 31) * 16;
+                *reinterpret_cast<uint4 *>(out) = reinterpret_cast<const uint4 *>(sf_tile)[threadIdx.x];
             }
         }
     }
@@ -398,8 +398,26 @@ sol_status_t launch_quantize(const void *x, int64_t rows, int64_t K, int64_t ld,
     return launch_quantize_ex(x, rows, K, ld, tscale, nullptr, nullptr, q, sf, layout, stream);
 }
 
+namespace {
+sol_status_t launch_mxfp4_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
+                                      sol_sf_layout_t layout, cudaStream_t stream, const QuantDest &dst);
+}
+
 sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
                                    sol_sf_layout_t layout, cudaStream_t stream) {
+    return launch_mxfp4_quantize_ex(x, rows, K, ld, q, sf, layout, stream,
+                                    QuantDest{K >> 1, 0, ((K >> 5) + 3) >> 2, 0, nullptr});
+}
+
+sol_status_t launch_mxfp4_quantize_into(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
+                                        int64_t dest_K, int64_t dest_col0, cudaStream_t stream) {
+    return launch_mxfp4_quantize_ex(x, rows, K, ld, q, sf, SOL_SF_SWIZZLED_128x4, stream,
+                                    QuantDest{dest_K >> 1, dest_col0 >> 1, dest_K >> 7, dest_col0 >> 7, nullptr});
+}
+
+namespace {
+sol_status_t launch_mxfp4_quantize_ex(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
+                                      sol_sf_layout_t layout, cudaStream_t stream, const QuantDest &dst) {
     cudaLaunchConfig_t cfg = {};
     const uint32_t k_tiles = static_cast<uint32_t>(ceil_div(K, kMxTileK));
     cfg.gridDim = dim3(static_cast<unsigned>(k_tiles * ceil_div(rows, kTileRows)));
@@ -412,12 +430,13 @@ sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64
     cfg.numAttrs = 1;
     auto kern = layout == SOL_SF_SWIZZLED_128x4 ? mxfp4_quantize_kernel<true> : mxfp4_quantize_kernel<false>;
     if (cudaLaunchKernelEx(&cfg, kern, static_cast<const uint16_t *>(x), rows, K, ld, static_cast<uint8_t *>(q),
-                           static_cast<uint8_t *>(sf), k_tiles) != cudaSuccess) {
+                           static_cast<uint8_t *>(sf), k_tiles, dst) != cudaSuccess) {
         cudaGetLastError();
         return SOL_ERR_CUDA;
     }
     return launch_status();
 }
+}  // namespace
 
 sol_status_t launch_quantize_from_amax(const void *x, int64_t rows, int64_t K, int64_t ld, float *scale_words,
                                        void *q, void *sf, sol_sf_layout_t layout, cudaStream_t stream, bool reverse) {

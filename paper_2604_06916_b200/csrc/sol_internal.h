@@ -100,6 +100,10 @@ sol_status_t launch_layernorm_quantize(const void *x, int64_t rows, int64_t K, i
 int layernorm_max_k();
 sol_status_t launch_mxfp4_quantize(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
                                    sol_sf_layout_t layout, cudaStream_t stream);
+// The same into columns [dest_col0, dest_col0 + K) of a wider MXFP4 tensor [rows, dest_K] (chunked scales;
+// K, dest_K and dest_col0 multiples of 128).
+sol_status_t launch_mxfp4_quantize_into(const void *x, int64_t rows, int64_t K, int64_t ld, void *q, void *sf,
+                                        int64_t dest_K, int64_t dest_col0, cudaStream_t stream);
 // Stage-1 selection and rank-consistency metrics (one block per prompt).
 sol_status_t launch_select_contrastive(const float *rewards, const uint64_t *seeds, int64_t P, int64_t N, int64_t K,
                                        int32_t *idx_out, uint64_t *seeds_out, float *adv_out, cudaStream_t stream);

@@ -195,3 +195,106 @@ def test_quantized_output_with_gelu_against_oracle(B):
     assert np.all(np.abs(deq - H) <= reach * (1 + 2.0 ** -6) + tol)
     # and it is the oracle's own output almost everywhere
     assert (hq.cpu().numpy() == q_star).mean() >= 0.98
+
+
+def pow2_mx(rng, rows, K):
+    """Random nibbles with power-of-two MXFP4 scales in a narrow range: sums stay exact in FP32."""
+    q = rng.integers(0, 256, size=(rows, K // 2), dtype=np.uint8)
+    return q, (rng.integers(-2, 3, size=(rows, K // 32)) + 127).astype(np.uint8)
+
+
+def concat_reference(B, parts):
+    """MXFP4 of the column-wise concatenation of BF16 tensors, from the library's own quantizer (itself bit for
+    bit the oracle's, see above)."""
+    return B.mxfp4_quantize(torch.cat(parts, dim=1).contiguous())
+
+
+@pytest.mark.parametrize("M,K1,K2", [(256, 128, 256), (300, 384, 128), (130, 1024, 3072)])
+def test_quantize_into_two_slices_equals_quantizer_on_the_concatenation(B, M, K1, K2):
+    g = torch.Generator(device="cuda").manual_seed(M + K1)
+    a = workloads.make_activation("student_t", M, K1, g, "cuda")
+    b = workloads.make_activation("student_t", M, K2, g, "cuda")
+    want_q, want_sf = concat_reference(B, [a, b])
+    xb = bits_of(torch.cat([a, b], dim=1))
+    q_or, sf_or = oracle.mxfp4_quantize(xb)
+    assert np.array_equal(want_q.cpu().numpy(), q_or)            # the reference itself against the oracle
+    assert np.array_equal(want_sf.cpu().numpy(), oracle.mx_sf_swizzle(sf_or, K1 + K2))
+    dest = (torch.full((M, (K1 + K2) // 2), 0xEE, dtype=torch.uint8, device="cuda"),
+            torch.full((B.mxfp4_scale_bytes(M, K1 + K2),), 0xEE, dtype=torch.uint8, device="cuda"))
+    B.mxfp4_quantize_into(b, dest, K1)
+    assert torch.all(dest[0][:, :K1 // 2] == 0xEE)               # the other column range is untouched
+    B.mxfp4_quantize_into(a, dest, 0)
+    B.sol_last_device_status()
+    assert torch.equal(dest[0], want_q)
+    got_sf = dest[1].cpu().numpy()[mx_offsets(np.arange(M), K1 + K2)]
+    assert np.array_equal(got_sf, sf_or)
+
+
+@pytest.mark.parametrize("M,N,n_split,K,col0,dest_K", [(256, 512, 256, 64, 0, 256), (300, 896, 256, 256, 128, 1024),
+                                                      (520, 768, 512, 512, 384, 640)])
+def test_split_output_integer_exact_bit_for_bit(B, M, N, n_split, K, col0, dest_K):
+    rng = np.random.default_rng(M + N + K)
+    qx, sfx = pow2_mx(rng, M, K)
+    qw, sfw = pow2_mx(rng, N, K)
+    Y = oracle.mxfp4_linear(qx, sfx, qw, sfw)
+    if np.abs(Y).max() * 4 >= 2 ** 24:
+        pytest.skip("sum too large for an exact FP32 accumulator")
+    part = N - n_split
+    h_bits = oracle.round_bf16(Y[:, n_split:])
+    q_ref, sf_ref = oracle.mxfp4_quantize(h_bits)
+    dest = (torch.full((M, dest_K // 2), 0xEE, dtype=torch.uint8, device="cuda"),
+            torch.full((B.mxfp4_scale_bytes(M, dest_K),), 0xEE, dtype=torch.uint8, device="cuda"))
+    amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    y = B.mxfp4_linear_split_out(dev(qx), dev(oracle.mx_sf_swizzle(sfx, K)), dev(qw), dev(oracle.mx_sf_swizzle(sfw, K)),
+                                 None, n_split, B.ACT_NONE, dest, col0, amax_out=amax)
+    B.sol_last_device_status()
+    assert np.array_equal(bits_of(y), oracle.round_bf16(Y[:, :n_split]))
+    got_q = dest[0].cpu().numpy()
+    assert np.array_equal(got_q[:, col0 // 2:(col0 + part) // 2], q_ref)
+    untouched = np.ones(dest_K // 2, bool)
+    untouched[col0 // 2:(col0 + part) // 2] = False
+    assert np.all(got_q[:, untouched] == 0xEE)
+    offs = mx_offsets(np.arange(M), dest_K)
+    got_sf = dest[1].cpu().numpy()[offs]
+    assert np.array_equal(got_sf[:, col0 // 32:(col0 + part) // 32], sf_ref)
+    keep = np.ones(dest_K // 32, bool)
+    keep[col0 // 32:(col0 + part) // 32] = False
+    assert np.all(got_sf[:, keep] == 0xEE)
+    assert amax.item() == np.abs(oracle.bits_to_f64(h_bits)).max()
+
+
+def test_single_stream_chain_in_mxfp4(B):
+    # split linear (q/k/v BF16 | GELU(MLP) as MXFP4 into the concat) + slice quantizer for the attention part,
+    # then the second linear on the concatenated MXFP4 tensor: equal to the unfused chain built from the
+    # entries checked above (mxfp4_linear, torch's tanh-GELU rounded to BF16 is NOT used: the quantized part is
+    # compared through its dequantized values against the oracle's FP64 GELU within the format's step)
+    M, K, n_split, n_mlp, attn_w, N2 = 384, 512, 768, 1024, 256, 256
+    N = n_split + n_mlp
+    g = torch.Generator(device="cuda").manual_seed(5)
+    X = workloads.make_activation("student_t", M, K, g, "cuda")
+    W1 = (torch.randn(N, K, generator=g, device="cuda") * K ** -0.5).to(torch.bfloat16)
+    b1 = (torch.randn(N, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    attn = workloads.make_activation("student_t", M, attn_w, g, "cuda")
+    xq, w1q = B.mxfp4_quantize(X), B.mxfp4_quantize(W1)
+    dest_K = attn_w + n_mlp
+    dest = (torch.zeros((M, dest_K // 2), dtype=torch.uint8, device="cuda"),
+            torch.zeros(B.mxfp4_scale_bytes(M, dest_K), dtype=torch.uint8, device="cuda"))
+    y_qkv = B.mxfp4_linear_split_out(*xq, *w1q, b1, n_split, B.ACT_GELU_TANH, dest, attn_w)
+    B.mxfp4_quantize_into(attn, dest, 0)
+    B.sol_last_device_status()
+    y_full = B.mxfp4_linear(*xq, *w1q, b1)
+    assert torch.equal(y_qkv, y_full[:, :n_split].contiguous())
+    # the attention slice is bit for bit the quantizer's output on that slice
+    aq, asf = B.mxfp4_quantize(attn)
+    assert torch.equal(dest[0][:, :attn_w // 2], aq)
+    # the MLP slice against the oracle's FP64 GELU of the FP64 linear
+    qx, sfx = oracle.mxfp4_quantize(bits_of(X))
+    qw, sfw = oracle.mxfp4_quantize(bits_of(W1))
+    Y = oracle.mxfp4_linear(qx, sfx, qw, sfw, bits_of(b1))[:, n_split:]
+    H = oracle.gelu_tanh(Y)
+    sf_rm = dest[1].cpu().numpy()[mx_offsets(np.arange(M), dest_K)][:, attn_w // 32:]
+    deq = oracle.mxfp4_dequantize(dest[0][:, attn_w // 2:].contiguous().cpu().numpy(), sf_rm)
+    scale = np.repeat(np.ldexp(1.0, sf_rm.astype(np.int32) - 127), 32, axis=1)
+    tol = 1.2 * oracle.linear_tolerance(Y) + 2.0 ** -8 * np.abs(H)
+    reach = np.maximum(1.0 * scale, np.abs(H) - 6.0 * scale)
+    assert np.all(np.abs(deq - H) <= reach * (1 + 2.0 ** -6) + tol)
