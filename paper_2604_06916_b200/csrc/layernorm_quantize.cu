@@ -8,9 +8,11 @@
 //
 // One warp owns one row at a time: its K values stay in registers between the mean, the centred
 // variance and the normalise / modulate / quantize sweep, and there is no block-level
-// synchronisation in the row loop.  Rows reach the warp through a two-slot ring in shared memory
-// filled by bulk asynchronous copies (cp.async.bulk + mbarrier) that the warp issues two rows ahead,
-// so the HBM latency is not paid by a warp that holds 160 registers per thread.  A lane owns whole 16-element
+// synchronisation in the row loop.  Rows reach the warp through one row-sized slot in shared memory
+// filled by a bulk asynchronous copy (cp.async.bulk + mbarrier): as soon as the row is in registers the
+// warp requests the next one, which lands while this one is computed (a row takes several times the
+// HBM latency), so the latency is not paid by a warp that holds 120 registers per thread, and a warp
+// costs 6 KB of shared memory at K = 3072: sixteen warps fit an SM beside the modulation tables.  A lane owns whole 16-element
 // scale blocks (blocks lane, lane + 32, ...), so K <= 4096.  A thread block works on rows of ONE
 // sample and keeps that sample's modulation in shared memory as FP32 pairs (1 + scale, shift).  The
 // block scale and the sixteen codes follow the quantizer's FP32 sequence on h = bf16(y); max|h| is
@@ -32,7 +34,6 @@ __device__ __forceinline__ void bulk_load_row(uint32_t dst, const void *src, uin
                  : "memory");
 }
 
-constexpr long long kLnWaitLimitCycles = 2000000000LL;
 
 // two FP32 -> packed BF16 (first argument in the low half), round to nearest even
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -51,10 +52,10 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
                           uint8_t *__restrict__ q, uint8_t *__restrict__ sf, uint32_t *amax_track,
                           uint32_t *status) {
     // (1 + scale) x 2, shift x 2 of this block's sample for element pairs, laid out [pair within block][block] so
-    // that the 32 lanes of a warp (consecutive blocks) read consecutive 16-byte words; behind it the row
-    // ring (two slots of K BF16 per warp)
+    // that the 32 lanes of a warp (consecutive blocks) read consecutive 16-byte words; behind it one row
+    // slot of K BF16 per warp
     extern __shared__ __align__(16) float4 mod[];
-    __shared__ __align__(8) uint64_t ring_bar[kLnMaxWarps][2];
+    __shared__ __align__(8) uint64_t ring_bar[kLnMaxWarps];
     __shared__ float rcp_tab[128];
     __shared__ uint32_t warp_seen[kLnMaxWarps];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -79,37 +80,35 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
     const float inv_k = 1.0f / static_cast<float>(K);
     uint32_t seen = 0;
     const uint32_t row_bytes = static_cast<uint32_t>(K) * 2u;
-    const uint32_t ring = ptx::smem_u32(mod) + static_cast<uint32_t>(K) * 8u + warp * 2u * row_bytes;
-    const uint32_t bar0 = ptx::smem_u32(&ring_bar[warp][0]);
+    const uint32_t ring = ptx::smem_u32(mod) + static_cast<uint32_t>(K) * 8u + warp * row_bytes;
+    const uint32_t bar0 = ptx::smem_u32(&ring_bar[warp]);
     const int64_t stride = static_cast<int64_t>(gridDim.x) * kLnWarps;
     const int64_t r_first = first + static_cast<int64_t>(blockIdx.x) * kLnWarps + warp;
     if (lane == 0) {
         ptx::mbar_init(bar0, 1);
-        ptx::mbar_init(bar0 + 8, 1);
         ptx::fence_mbar_init();
     }
     __syncwarp();
-    if (lane == 0) {   // rows 0 and 1 of this warp
-        for (int j = 0; j < 2; ++j)
-            if (r_first + j * stride < last) {
-                ptx::mbar_arrive_expect_tx(bar0 + 8u * j, row_bytes);
-                bulk_load_row(ring + j * row_bytes, x + (r_first + j * stride) * ld, row_bytes, bar0 + 8u * j);
-            }
+    if (lane == 0 && r_first < last) {   // the warp's first row
+        ptx::mbar_arrive_expect_tx(bar0, row_bytes);
+        bulk_load_row(ring, x + r_first * ld, row_bytes, bar0);
     }
-    int64_t j = 0;
-    for (int64_t r = r_first; r < last; r += stride, ++j) {
-        const uint32_t slot = static_cast<uint32_t>(j) & 1u, parity = static_cast<uint32_t>(j >> 1) & 1u;
-        if (!ptx::mbar_try_wait(bar0 + 8u * slot, parity)) {   // bounded: a copy that never lands ends the loop
+    uint32_t parity = 0;
+    for (int64_t r = r_first; r < last; r += stride, parity ^= 1u) {
+        // bounded, and every decision taken by a warp-wide vote: a copy that never lands ends the loop for the
+        // whole warp (no other copy of this warp is in flight then)
+        if (!__all_sync(0xFFFFFFFFu, ptx::mbar_try_wait(bar0, parity))) {
             const long long t0 = clock64();
+            const long long limit = *reinterpret_cast<const volatile long long *>(status + 2);
             bool ok = true;
-            while (!ptx::mbar_try_wait(bar0 + 8u * slot, parity)) {
-                if (clock64() - t0 > kLnWaitLimitCycles) {
+            while (!__all_sync(0xFFFFFFFFu, ptx::mbar_try_wait(bar0, parity))) {
+                if (__any_sync(0xFFFFFFFFu, clock64() - t0 > limit)) {
                     ok = false;
                     break;
                 }
             }
-            if (!__all_sync(0xFFFFFFFFu, ok)) {   // warp-uniform exit
-                if (lane == 0 && status != nullptr) atomicExch(status, 0xA00u);
+            if (!ok) {
+                if (lane == 0) atomicExch(status, 0xA00u);
                 break;
             }
         }
@@ -121,7 +120,7 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
             const int b = lane + 32 * i;
             uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0;
             if (b < nblocks) {
-                const uint32_t src = ring + slot * row_bytes + b * 32;
+                const uint32_t src = ring + b * 32;
                 asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v0.x), "=r"(v0.y), "=r"(v0.z), "=r"(v0.w) : "r"(src));
                 asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v1.x), "=r"(v1.y), "=r"(v1.z), "=r"(v1.w) : "r"(src + 16));
             }
@@ -132,30 +131,31 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
         // through the async proxy, which an mbarrier or a warp barrier alone does not order behind generic reads)
         ptx::fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0 && r + 2 * stride < last) {   // the slot is free again: fetch the row after next
-            ptx::mbar_arrive_expect_tx(bar0 + 8u * slot, row_bytes);
-            bulk_load_row(ring + slot * row_bytes, x + (r + 2 * stride) * ld, row_bytes, bar0 + 8u * slot);
+        if (lane == 0 && r + stride < last) {   // the slot is free again: fetch the next row
+            ptx::mbar_arrive_expect_tx(bar0, row_bytes);
+            bulk_load_row(ring, x + (r + stride) * ld, row_bytes, bar0);
         }
         // mean and variance in one sweep over data shifted by a pivot taken from the row (its first element):
         // sum (x - p) and sum (x - p)^2 lose no accuracy to cancellation as long as p lies within the data,
         // and the two warp reductions run side by side instead of one after the other
         const float pivot = __shfl_sync(0xFFFFFFFFu, qmath::bf16_lo(w[0][0]), 0);
         const uint64_t npivot2 = qmath::f32x2(-pivot, -pivot);
-        uint64_t s1_2 = 0, s2_2 = 0;   // two lanes of 0.0f
+        // four independent accumulator pairs per sum: a single one is a chain of 48 dependent additions per lane
+        uint64_t s1_2[4] = {0, 0, 0, 0}, s2_2[4] = {0, 0, 0, 0};   // lanes of 0.0f
 #pragma unroll
         for (int i = 0; i < kBlocksPerLane; ++i) {
             if (lane + 32 * i < nblocks) {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const uint64_t d2 = qmath::add2(qmath::f32x2_of_bf16x2(w[i][e]), npivot2);
-                    s1_2 = qmath::add2(s1_2, d2);
-                    s2_2 = qmath::fma2(d2, d2, s2_2);
+                    s1_2[e & 3] = qmath::add2(s1_2[e & 3], d2);
+                    s2_2[e & 3] = qmath::fma2(d2, d2, s2_2[e & 3]);
                 }
             }
         }
         float s2, s1b, s2b;
-        qmath::f32x2_split(s1_2, s1, s1b);
-        qmath::f32x2_split(s2_2, s2, s2b);
+        qmath::f32x2_split(qmath::add2(qmath::add2(s1_2[0], s1_2[1]), qmath::add2(s1_2[2], s1_2[3])), s1, s1b);
+        qmath::f32x2_split(qmath::add2(qmath::add2(s2_2[0], s2_2[1]), qmath::add2(s2_2[2], s2_2[3])), s2, s2b);
         s1 += s1b;
         s2 += s2b;
 #pragma unroll
@@ -172,38 +172,49 @@ layernorm_quantize_kernel(const uint16_t *__restrict__ x, int64_t rows, int K, i
         const int64_t row_tile = r >> 7;
         const int rr = static_cast<int>(r & 127);
         uint8_t *sf_row = sf + row_tile * chunks_k * 512 + (rr & 31) * 16 + (rr >> 5) * 4;
-        // ---- normalise, modulate, round to BF16, quantize
+        // ---- normalise, modulate, round to BF16 (h takes the row's registers), then the block scales of all
+        // the lane's blocks side by side (a division and a table look-up each), then the codes
+        uint32_t bmax[kBlocksPerLane];
 #pragma unroll
         for (int i = 0; i < kBlocksPerLane; ++i) {
             const int b = lane + 32 * i;
-            uint32_t sb = 0;
+            uint32_t bm0 = 0, bm1 = 0;
             if (b < nblocks) {
                 const float4 *mp = mod + b;
-                uint32_t hw[8];
-                uint32_t bm = 0;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const float4 m = mp[e * nblocks];   // (1 + scale) and shift of two neighbouring elements
                     const uint64_t xh2 = qmath::fma2(qmath::f32x2_of_bf16x2(w[i][e]), rstd2, nmr2);
                     float y0, y1;
                     qmath::f32x2_split(qmath::fma2(xh2, qmath::f32x2(m.x, m.y), qmath::f32x2(m.z, m.w)), y0, y1);
-                    hw[e] = pack_bf16x2(y0, y1);
-                    bm = qmath::absmax2(bm, hw[e]);
+                    w[i][e] = pack_bf16x2(y0, y1);
+                    if (e & 1) bm1 = qmath::absmax2(bm1, w[i][e]);
+                    else bm0 = qmath::absmax2(bm0, w[i][e]);
                 }
-                bm &= 0x7FFF7FFFu;
-                const uint32_t abits = max(bm & 0xFFFFu, bm >> 16);
-                seen = max(seen, abits);
-                const float a = __uint_as_float(abits << 16);
-                sb = qmath::f32_to_e4m3_sat(__fdiv_rn(a, c6T));
-                const float rcp = rcp_tab[sb];
-                const uint64_t rcp2 = qmath::f32x2(rcp, rcp);
-                uint2 packed;
-                packed.x = qmath::quantize8_x2(hw[0], hw[1], hw[2], hw[3], rcp2);
-                packed.y = qmath::quantize8_x2(hw[4], hw[5], hw[6], hw[7], rcp2);
-                __stcs(reinterpret_cast<uint2 *>(q + r * (K >> 1) + b * 8), packed);
             }
-            // the lane's scale byte of its (row, chunk) slot (four neighbouring lanes fill one 4-byte slot)
-            if (b < nblocks) sf_row[(b >> 2) * 512 + (b & 3)] = static_cast<uint8_t>(sb);
+            const uint32_t bm = qmath::absmax2(bm0, bm1) & 0x7FFF7FFFu;
+            bmax[i] = max(bm & 0xFFFFu, bm >> 16);
+        }
+        uint32_t sbv[kBlocksPerLane];
+        float rcpv[kBlocksPerLane];
+#pragma unroll
+        for (int i = 0; i < kBlocksPerLane; ++i) {
+            seen = max(seen, bmax[i]);
+            sbv[i] = qmath::f32_to_e4m3_sat(__fdiv_rn(__uint_as_float(bmax[i] << 16), c6T));
+            rcpv[i] = rcp_tab[sbv[i]];
+        }
+#pragma unroll
+        for (int i = 0; i < kBlocksPerLane; ++i) {
+            const int b = lane + 32 * i;
+            if (b < nblocks) {
+                const uint64_t rcp2 = qmath::f32x2(rcpv[i], rcpv[i]);
+                uint2 packed;
+                packed.x = qmath::quantize8_x2(w[i][0], w[i][1], w[i][2], w[i][3], rcp2);
+                packed.y = qmath::quantize8_x2(w[i][4], w[i][5], w[i][6], w[i][7], rcp2);
+                __stcs(reinterpret_cast<uint2 *>(q + r * (K >> 1) + b * 8), packed);
+                // the lane's scale byte of its (row, chunk) slot (four neighbouring lanes fill one 4-byte slot)
+                sf_row[(b >> 2) * 512 + (b & 3)] = static_cast<uint8_t>(sbv[i]);
+            }
         }
     }
     // rows past M inside the last 128-row scale chunk are padding and read as 0 (first block only)
@@ -238,17 +249,17 @@ sol_status_t launch_layernorm_quantize(const void *x, int64_t rows, int64_t K, i
     if (samples > 65535) return SOL_ERR_BAD_SHAPE;
     const DeviceInfo *dev = current_device_info();
     const int sms = dev != nullptr && dev->ok ? dev->sm_count : 148;
-    // modulation table (8 bytes per element) + per warp two row slots of 2 bytes per element.  Four warps
-    // per block, three blocks per SM at K = 3072; one block of 14-16 warps per SM measured no faster
-    // (the kernel is bound by instruction issue, not by rows in flight).
+    // modulation table (8 bytes per element) + per warp one row slot of 2 bytes per element: four warps per
+    // block, four blocks per SM at K = 3072 (registers allow no more)
     const int kLnWarps = 4;
     const int kLnThreads = kLnWarps * 32;
-    const size_t smem = static_cast<size_t>(K) * 8 + static_cast<size_t>(kLnWarps) * 2 * K * 2;
+    const size_t smem = static_cast<size_t>(K) * 8 + static_cast<size_t>(kLnWarps) * K * 2;
     const int per_lane = static_cast<int>(ceil_div(K / 16, 32));
     auto launch = [&](auto kern) {
         // one wave of resident blocks, split evenly over the samples, never more blocks per sample
         // than it has groups of rows
-        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024);
+        // (the static tables count against the 48 KB default too)
+        if (smem + 1024 > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024);
         int per_sm = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kLnThreads, smem) != cudaSuccess || per_sm < 1)
             per_sm = 1;
