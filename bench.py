@@ -973,6 +973,39 @@ def run_only(args):
     from paper_2604_06916_b200 import binding as B
     from paper_2604_06916_b200 import workloads
 
+    if args.only == "step":
+        # the six-layer step alone (launch lists and profiler captures): warm-up, then `steps` NVFP4 steps and
+        # `steps` BF16 steps, each timed as one region
+        cfg = workloads.CONFIGS[args.workload]
+        M = args.rows if args.rows > 0 else None
+        data = []
+        for i, l in enumerate(cfg.layers):
+            X, W, bias = workloads.make_layer(cfg, i, "cuda", M=M)
+            wq, wsf, wts = B.nvfp4_quantize_weight(W)
+            Y = torch.empty((X.shape[0], l.N), dtype=torch.bfloat16, device="cuda")
+            ws = torch.empty(B.linear_workspace_bytes(X.shape[0], l.N, l.K), dtype=torch.uint8, device="cuda")
+            data.append((X, W, bias, wq, wsf, wts, Y, ws))
+        res = {}
+        for name in ("nvfp4", "bf16"):
+            def step():
+                for X, W, bias, wq, wsf, wts, Y, ws in data:
+                    if name == "nvfp4":
+                        B.nvfp4_quantize_linear(X, wq, wsf, wts, bias, workspace=ws, out=Y)
+                    else:
+                        B.bf16_linear(X, W, bias, out=Y)
+            for _ in range(args.warmup):
+                step()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                step()
+            e1.record()
+            torch.cuda.synchronize()
+            res[name + "_ms_per_step"] = e0.elapsed_time(e1) / args.steps
+        B.sol_last_device_status()
+        print(json.dumps({"only": "step", "workload": cfg.name, "rows": data[0][0].shape[0], **res}))
+        return
     if args.only == "weight_refresh":
         # eight FLUX attention projections (3072 x 3072, rank-32 adapters) through the batched entry
         n = 3072
@@ -1242,7 +1275,7 @@ def run_only(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'weight_refresh' / 'mlp_pair' / 'mxfp4:<layer>' / 'layernorm_quantize' / 'single_block' / 'attention'")
+    ap.add_argument("--only", default="", help="profile mode: run just this layer of the workload, or 'step' / 'weight_refresh' / 'mlp_pair' / 'mxfp4:<layer>' / 'layernorm_quantize' / 'single_block' / 'attention'")
     ap.add_argument("--rows", type=int, default=0, help="profile mode: override M")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
