@@ -124,9 +124,10 @@ __device__ __forceinline__ void quantize_tile(const uint16_t *__restrict__ x, in
             const float sv = __fdiv_rn(a, c);
             const uint32_t sb = f32_to_e4m3_sat(sv);
             const float rcp = rcp_tab[sb];
+            const uint64_t rcp2 = qmath::f32x2(rcp, rcp);   // the sixteen products two at a time (same roundings)
             uint2 packed;
-            packed.x = quantize8(lo[i], rcp);
-            packed.y = quantize8(hi[i], rcp);
+            packed.x = qmath::quantize8_x2(lo[i].x, lo[i].y, lo[i].z, lo[i].w, rcp2);
+            packed.y = qmath::quantize8_x2(hi[i].x, hi[i].y, hi[i].z, hi[i].w, rcp2);
             if (k_ok && r < rows) {
                 __stcs(reinterpret_cast<uint2 *>(q + r * dst.q_pitch + dst.q_col0 + (k >> 1)), packed);
                 if (kSwizzled) {
