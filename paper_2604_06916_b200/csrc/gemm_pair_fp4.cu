@@ -35,6 +35,12 @@ constexpr int kStageBytes = kABytes + kBBytes;  // 32 KB: one k-tile of A and B
 constexpr int kSfSlotBytes = kSfaBytes + kSfbBytes;  // 6 KB: one k-tile of scale tiles
 constexpr int kSfSlots = 5;                    // scale-tile ring in shared memory, released as soon as a tile is in registers
 constexpr int kSfBufCols = 48;                 // per k-tile: 4 MMAs x (4 columns of A + 8 of B)
+#ifdef SOL_SPAN
+// Diagnostic build only (-DSOL_SPAN, otherwise identical to the product kernel): SM cycles and nanoseconds
+// CTA 0 spent between the dependency wait and the final cluster barrier of the last launch.  Their ratio
+// is the SM clock the kernel really ran at, which under the board's power cap is far from the maximum.
+__device__ long long g_span[2];
+#endif
 constexpr int kAccStride = 96;                 // accumulator B starts here; [96,256) is shared
 constexpr int kSfBufs = 3;
 constexpr int kSfCol = kAccStride + kBN;       // 352
@@ -327,6 +333,13 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_smem;
     ptx::grid_dependency_wait();  // set-up above overlaps the previous kernel; its results are read below
+#ifdef SOL_SPAN
+    long long span_c0 = 0, span_g0 = 0;
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        span_c0 = clock64();
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(span_g0));
+    }
+#endif
 
     if (kTuning && warp == kWarps) {
         // diagnostic build: polls each stage's `full` barrier without suspending and records when it completes
@@ -694,6 +707,14 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::cluster_sync();  // neither CTA frees TMEM or exits while its partner may still touch it
+#ifdef SOL_SPAN
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        long long g1;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(g1));
+        g_span[0] = clock64() - span_c0;
+        g_span[1] = g1 - span_g0;
+    }
+#endif
     if (warp == 1) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
@@ -880,5 +901,11 @@ sol_status_t launch_pair256_nvfp4_split_out(const void *xq, const void *xsf, con
 #ifdef SOL_TUNING
 extern "C" int sol_debug_trace256(long long *host_out) {
     return cudaMemcpyFromSymbol(host_out, sol::gemm::g_trace, sizeof(sol::gemm::g_trace)) == cudaSuccess ? 0 : 1;
+}
+#endif
+
+#ifdef SOL_SPAN
+extern "C" int sol_debug_span(long long *host_out) {
+    return cudaMemcpyFromSymbol(host_out, sol::gemm::g_span, 16) == cudaSuccess ? 0 : 1;
 }
 #endif

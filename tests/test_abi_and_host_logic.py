@@ -233,5 +233,6 @@ def test_diagnostic_build_of_the_gemm_kernels_compiles(tmp_path):
         pytest.skip("nvcc not available")
     csrc = os.path.join(ROOT, "paper_2604_06916_b200", "csrc")
     for src in ("gemm_pair_fp4.cu", "gemm_pair.cu", "gemm.cu", "attention.cu"):
-        subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", "-DSOL_TUNING", "-c",
+        flags = ["-DSOL_TUNING"] + (["-DSOL_SPAN"] if src == "gemm_pair_fp4.cu" else [])  # + cycle / time span of CTA 0
+        subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", *flags, "-c",
                         "-o", str(tmp_path / (src + ".o")), os.path.join(csrc, src)], check=True)
