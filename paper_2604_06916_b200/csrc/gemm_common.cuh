@@ -77,27 +77,6 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
     return true;
 }
 
-// The same for a wait on the critical path of a pipeline: polls without suspending (a suspended thread
-// takes several hundred cycles to resume after the barrier completes), a short sleep between polls.
-__device__ __forceinline__ bool wait_bounded_spin(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                                  uint32_t *status, uint32_t code) {
-    if (ptx::mbar_test_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    uint32_t n = 0;
-    while (!ptx::mbar_test_wait(bar, parity)) {
-        __nanosleep(20);
-        if ((++n & 255u) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > *reinterpret_cast<const volatile long long *>(status + 2)) {
-                *abort_flag = 1;
-                atomicExch(status, code);
-                return false;
-            }
-        }
-    }
-    return true;
-}
-
 // Test hook (device status block, word 1): the load-issuing warps issue nothing while it is set.
 __device__ __forceinline__ bool loads_held(const uint32_t *status) {
     return *reinterpret_cast<const volatile uint32_t *>(status + 1) != 0;

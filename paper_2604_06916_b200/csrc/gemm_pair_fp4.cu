@@ -47,17 +47,6 @@ constexpr int kSfCol = kAccStride + kBN;       // 352
 constexpr int kEpiWarpsFp4 = 8;
 constexpr int kSfCopyWarps = 4;                // one per TMEM lane quadrant
 constexpr int kWarps = 2 + kEpiWarpsFp4 + kSfCopyWarps + 1;
-#ifndef SOL_SPIN_MASK
-#define SOL_SPIN_MASK 0
-#endif
-// which waits poll instead of suspending: 1 A/B producer on `empty`, 2 scale-copy warps on the TMEM buffer,
-// 4 MMA thread on `sf_ready` / `full`, 8 epilogue on `acc_full`, 16 MMA thread on `ovl_free` / `acc_empty`
-template <int kBit>
-__device__ __forceinline__ bool wait_site(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag, uint32_t *status,
-                                          uint32_t code) {
-    if constexpr ((SOL_SPIN_MASK & kBit) != 0) return wait_bounded_spin(bar, parity, abort_flag, status, code);
-    else return wait_bounded(bar, parity, abort_flag, status, code);
-}
 constexpr int kThreadsFp4 = 32 * (kWarps + (kTuning ? 1 : 0));  // 480 (+ a probe warp in the diagnostic build)
 constexpr int kEpiBytes = kEpiWarpsFp4 * kEpiBufBytes;
 constexpr int kBiasBytes = kEpiWarpsFp4 * 256;  // per epilogue warp: BF16 bias of its two 64-column chunks
@@ -374,7 +363,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
             const int nb0 = nt * kBN + static_cast<int>(rank) * (kBN / 2);
             int kx = 0;
             for (int kt = 0; kt < k_tiles; ++kt, kx += kRowBytes) {
-                if (!wait_site<1>(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x100u | stage)) {
+                if (!wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 0x100u | stage)) {
                     ok = false;
                     break;
                 }
@@ -452,9 +441,9 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 const int x = it & 1;
                 const uint32_t use = static_cast<uint32_t>(it >> 1);
                 // this accumulator's previous tile is fully drained ...
-                if (!wait_site<16>(acc_empty_bar(x), (use & 1u) ^ 1u, abort_flag, p.status, 0x200u | x)) break;
+                if (!wait_bounded(acc_empty_bar(x), (use & 1u) ^ 1u, abort_flag, p.status, 0x200u | x)) break;
                 // ... and the previous tile (other accumulator) has given back the shared columns
-                if (it > 0 && !wait_site<16>(ovl_free_bar(x ^ 1), (static_cast<uint32_t>(it - 1) >> 1) & 1u, abort_flag,
+                if (it > 0 && !wait_bounded(ovl_free_bar(x ^ 1), (static_cast<uint32_t>(it - 1) >> 1) & 1u, abort_flag,
                                             p.status, 0x900u | x))
                     break;
                 ptx::tc_fence_after_sync();
@@ -465,11 +454,11 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     // normally long before) and A and B are in shared memory (`full`); `sf_seen`: the previous
                     // k-tile already saw both complete (peek below)
                     if (!sf_seen) {
-                        if (!wait_site<4>(sf_ready_bar(sf_buf), sf_phase, abort_flag, p.status, 0x500u | sf_buf)) {
+                        if (!wait_bounded(sf_ready_bar(sf_buf), sf_phase, abort_flag, p.status, 0x500u | sf_buf)) {
                             ok = false;
                             break;
                         }
-                        if (!wait_site<4>(full_bar(stage), phase, abort_flag, p.status, 0x300u | stage)) {
+                        if (!wait_bounded(full_bar(stage), phase, abort_flag, p.status, 0x300u | stage)) {
                             ok = false;
                             break;
                         }
@@ -562,7 +551,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                     __syncwarp();
                     if (elected) ptx::mbar_arrive(sf_empty_bar(slot));
                     if (gi >= kSfBufs && !(kTuning && (p.dbg & kDbgNoSfCopy)) &&
-                        !wait_site<2>(empty_bar(old_stage), old_phase, abort_flag, p.status, 0x700u | old_stage)) {
+                        !wait_bounded(empty_bar(old_stage), old_phase, abort_flag, p.status, 0x700u | old_stage)) {
                         ok = false;
                         break;
                     }
@@ -625,7 +614,7 @@ gemm_pair_fp4_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
                 asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(sbias + lane * 8), "r"(bv.x), "r"(bv.y) : "memory");
                 __syncwarp();
             }
-            if (!wait_site<8>(acc_full_bar(x), (static_cast<uint32_t>(it) >> 1) & 1u, abort_flag, p.status, 0x400u | x)) break;
+            if (!wait_bounded(acc_full_bar(x), (static_cast<uint32_t>(it) >> 1) & 1u, abort_flag, p.status, 0x400u | x)) break;
             ptx::tc_fence_after_sync();
             if (kTuning && (p.dbg & kDbgTrace) && warp == 2) SOL_TRACE(9, it);
             const uint32_t t_acc = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + x * kAccStride;
