@@ -7,7 +7,9 @@ missing or a call fails, an exception is raised.
 from __future__ import annotations
 
 import ctypes
+import functools
 import os
+import types
 
 import torch
 
@@ -128,6 +130,65 @@ def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
+# Guard bands (debugging aid, off unless SOL_NVFP4_GUARD=1): every output this module allocates sits between
+# two 4 KB bands of a fixed byte, and after each call the device is synchronised and the bands are checked, so
+# a kernel that writes outside its output is caught by the call that did it.  Callers' own `out=` buffers
+# are theirs to guard.
+GUARD_BYTES = 4096
+GUARD_BYTE = 0xA5
+_guard_pending: list = []
+
+
+def guard_mode() -> bool:
+    return os.environ.get("SOL_NVFP4_GUARD", "0") not in ("", "0")
+
+
+def _empty(shape, dtype, device) -> torch.Tensor:
+    """torch.empty, or (guard mode) a view between two guard bands of one larger allocation."""
+    if not guard_mode():
+        return torch.empty(shape, dtype=dtype, device=device)
+    shape = (shape,) if isinstance(shape, int) else tuple(shape)
+    n = 1
+    for d in shape:
+        n *= int(d)
+    nbytes = n * torch.empty((), dtype=dtype).element_size()
+    padded = (nbytes + 255) // 256 * 256          # the back band starts on a 256-byte boundary
+    raw = torch.empty(2 * GUARD_BYTES + padded, dtype=torch.uint8, device=device)
+    raw[:GUARD_BYTES].fill_(GUARD_BYTE)
+    raw[GUARD_BYTES + nbytes:].fill_(GUARD_BYTE)
+    _guard_pending.append((raw, nbytes))
+    return raw[GUARD_BYTES:GUARD_BYTES + nbytes].view(dtype).view(shape)
+
+
+def check_guards(where: str = "") -> None:
+    """Verify and forget the guard bands of the outputs allocated since the last check."""
+    pending, bad = list(_guard_pending), []
+    _guard_pending.clear()
+    if not pending:
+        return
+    if pending[0][0].is_cuda:
+        torch.cuda.synchronize()
+    for raw, nbytes in pending:
+        front = bool((raw[:GUARD_BYTES] == GUARD_BYTE).all())
+        back = bool((raw[GUARD_BYTES + nbytes:] == GUARD_BYTE).all())
+        if not (front and back):
+            bad.append(f"{nbytes}-byte output: {'front' if not front else 'back'} band overwritten")
+    if bad:
+        raise AssertionError(f"{where}: write outside an output buffer ({'; '.join(bad)})")
+
+
+def _guarded(fn):
+    @functools.wraps(fn)
+    def call(*args, **kwargs):
+        if not guard_mode():
+            return fn(*args, **kwargs)
+        try:
+            return fn(*args, **kwargs)
+        finally:
+            check_guards(fn.__name__)
+    return call
+
+
 def _ptr(t) -> int | None:
     return None if t is None else t.data_ptr()
 
@@ -153,7 +214,7 @@ def sol_amax_bf16(x: torch.Tensor, out: torch.Tensor | None = None) -> torch.Ten
     """Per-tensor scale T = max|x| / 2688 (1 for zeros) as a 1-element float32 device tensor."""
     _need_2d_bf16(x, "x")
     if out is None:
-        out = torch.empty(1, dtype=torch.float32, device=x.device)
+        out = _empty(1, torch.float32, x.device)
     _check(lib().sol_amax_bf16(_ptr(x), x.shape[0], x.shape[1], x.stride(0), _ptr(out), _stream()), "sol_amax_bf16")
     return out
 
@@ -162,8 +223,8 @@ def _alloc_q(rows: int, K: int, layout: int, device):
     nq, ns = data_bytes(rows, K), scale_bytes(rows, K, layout)
     if nq == 0 or ns == 0:
         raise SolError(2, "shape check")
-    q = torch.empty((rows, K // 2), dtype=torch.uint8, device=device)
-    sf = torch.empty(ns, dtype=torch.uint8, device=device)
+    q = _empty((rows, K // 2), torch.uint8, device)
+    sf = _empty(ns, torch.uint8, device)
     return q, sf
 
 
@@ -183,7 +244,7 @@ def nvfp4_quantize_weight(w: torch.Tensor, layout: int = SF_SWIZZLED_128x4):
     _need_2d_bf16(w, "w")
     N, K = w.shape
     q, sf = _alloc_q(N, K, layout, w.device)
-    ts = torch.empty(1, dtype=torch.float32, device=w.device)
+    ts = _empty(1, torch.float32, w.device)
     _check(lib().nvfp4_quantize_weight(_ptr(w), N, K, w.stride(0), _ptr(q), _ptr(sf), _ptr(ts), layout, _stream()),
            "nvfp4_quantize_weight")
     return q, sf, ts
@@ -204,10 +265,10 @@ def nvfp4_requantize_lora(w: torch.Tensor, lora_a: torch.Tensor, lora_b: torch.T
     if lora_a.shape[1] != K or tuple(lora_b.shape) != (N, r):
         raise ValueError("shapes: w [N, K], lora_a [r, K], lora_b [N, r]")
     if merged is None:
-        merged = torch.empty((N, K), dtype=torch.bfloat16, device=w.device)
+        merged = _empty((N, K), torch.bfloat16, w.device)
     if out is None:
         q, sf = _alloc_q(N, K, layout, w.device)
-        ts2 = torch.empty(2, dtype=torch.float32, device=w.device)
+        ts2 = _empty(2, torch.float32, w.device)
     else:
         q, sf, ts2 = out
         if ts2.numel() < 2:
@@ -242,11 +303,11 @@ class LoraRefreshPlan:
         self.items = list(items)
         self.N, self.K, self.r, self.scaling, self.layout = N, K, r, float(scaling), layout
         self.group = max(1, min(group, len(items)))
-        self.merged = torch.empty((self.group, N, K), dtype=torch.bfloat16, device=dev)
+        self.merged = _empty((self.group, N, K), torch.bfloat16, dev)
         self.outputs = []
         for _ in items:
             q, sf = _alloc_q(N, K, layout, dev)
-            self.outputs.append((q, sf, torch.empty(2, dtype=torch.float32, device=dev)))
+            self.outputs.append((q, sf, _empty(2, torch.float32, dev)))
         n = len(items)
         arr = ctypes.c_void_p * n
         self._lists = [arr(*[t[i].data_ptr() for t in items]) for i in range(3)] + \
@@ -264,7 +325,7 @@ def nvfp4_linear(xq, xsf, x_tscale, wq, wsf, w_tscale, bias=None, out: torch.Ten
     M, K = xq.shape[0], xq.shape[1] * 2
     N = wq.shape[0]
     if out is None:
-        out = torch.empty((M, N), dtype=torch.bfloat16, device=xq.device)
+        out = _empty((M, N), torch.bfloat16, xq.device)
     _check(lib().nvfp4_linear(_ptr(xq), _ptr(xsf), _ptr(x_tscale), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
                               _ptr(out), M, N, K, out.stride(0), _stream()), "nvfp4_linear")
     return out
@@ -282,7 +343,7 @@ def nvfp4_linear_split_out(xq, xsf, x_tscale, wq, wsf, w_tscale, bias, n_split: 
     hq, hsf = dest
     dest_K = hq.shape[1] * 2
     if y_out is None:
-        y_out = torch.empty((M, n_split), dtype=torch.bfloat16, device=xq.device)
+        y_out = _empty((M, n_split), torch.bfloat16, xq.device)
     _check(lib().nvfp4_linear_split_out(_ptr(xq), _ptr(xsf), _ptr(x_tscale), _ptr(wq), _ptr(wsf), _ptr(w_tscale),
                                         _ptr(bias), _ptr(y_out), y_out.stride(0), n_split, activation, _ptr(out_tscale),
                                         _ptr(hq), _ptr(hsf), dest_K, dest_col0, _ptr(amax_out), M, N, K, _stream()),
@@ -306,9 +367,9 @@ def nvfp4_quantize_linear_delayed(x, wq, wsf, w_tscale, bias, scale_state: torch
     M, K = x.shape
     N = wq.shape[0]
     if workspace is None:
-        workspace = torch.empty(linear_workspace_bytes(M, N, K), dtype=torch.uint8, device=x.device)
+        workspace = _empty(linear_workspace_bytes(M, N, K), torch.uint8, x.device)
     if out is None:
-        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+        out = _empty((M, N), torch.bfloat16, x.device)
     _check(lib().nvfp4_quantize_linear_delayed(_ptr(x), x.stride(0), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
                                                _ptr(out), M, N, K, out.stride(0), _ptr(scale_state), _ptr(workspace),
                                                workspace.numel(), _stream()), "nvfp4_quantize_linear_delayed")
@@ -371,7 +432,7 @@ def sol_attention_bf16_joint(first, second, out=None):
         if q.shape != k.shape or q.shape != v.shape:
             raise ValueError("q, k and v of a stream must have one shape")
         if outs[i] is None:
-            outs[i] = torch.empty(tuple(q.shape), dtype=torch.bfloat16, device=q.device)
+            outs[i] = _empty(tuple(q.shape), torch.bfloat16, q.device)
         _check_attention_view("out", outs[i])
         streams.append(AttentionStream(_ptr(q), _ptr(k), _ptr(v), _ptr(outs[i]), q.shape[1], _token_pitch(q),
                                        _token_pitch(k), _token_pitch(v), _token_pitch(outs[i])))
@@ -396,7 +457,7 @@ def sol_attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, out: t
     if k.shape != v.shape or k.shape[0] != B or k.shape[2] != H or k.shape[3] != D:
         raise ValueError("k and v must share [B, Skv, H, D] with q's batch, heads and head dimension")
     if out is None:
-        out = torch.empty((B, Sq, H, D), dtype=torch.bfloat16, device=q.device)
+        out = _empty((B, Sq, H, D), torch.bfloat16, q.device)
     _check_attention_view("out", out)
     _check(lib().sol_attention_bf16(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, Sq, k.shape[1], H, D, _token_pitch(q),
                                     _token_pitch(k), _token_pitch(v), _token_pitch(out), _stream()), "sol_attention_bf16")
@@ -435,8 +496,8 @@ def mxfp4_quantize(x: torch.Tensor, layout: int = SF_SWIZZLED_128x4, out=None):
         nbytes = mxfp4_scale_bytes(rows, K, layout)
         if nbytes == 0:
             raise ValueError("bad shape for mxfp4_quantize")
-        out = (torch.empty((rows, K // 2), dtype=torch.uint8, device=x.device),
-               torch.empty(nbytes, dtype=torch.uint8, device=x.device))
+        out = (_empty((rows, K // 2), torch.uint8, x.device),
+               _empty(nbytes, torch.uint8, x.device))
     q, sf = out
     _check(lib().mxfp4_quantize(_ptr(x), rows, K, x.stride(0), _ptr(q), _ptr(sf), layout, _stream()), "mxfp4_quantize")
     return q, sf
@@ -447,7 +508,7 @@ def mxfp4_linear(xq, xsf, wq, wsf, bias=None, out: torch.Tensor | None = None):
     M, K = xq.shape[0], xq.shape[1] * 2
     N = wq.shape[0]
     if out is None:
-        out = torch.empty((M, N), dtype=torch.bfloat16, device=xq.device)
+        out = _empty((M, N), torch.bfloat16, xq.device)
     _check(lib().mxfp4_linear(_ptr(xq), _ptr(xsf), _ptr(wq), _ptr(wsf), _ptr(bias), _ptr(out), M, N, K, out.stride(0),
                               _stream()), "mxfp4_linear")
     return out
@@ -460,7 +521,7 @@ def mxfp4_linear_split_out(xq, xsf, wq, wsf, bias, n_split: int, activation: int
     N = wq.shape[0]
     hq, hsf = dest
     if y_out is None:
-        y_out = torch.empty((M, n_split), dtype=torch.bfloat16, device=xq.device)
+        y_out = _empty((M, n_split), torch.bfloat16, xq.device)
     _check(lib().mxfp4_linear_split_out(_ptr(xq), _ptr(xsf), _ptr(wq), _ptr(wsf), _ptr(bias), _ptr(y_out), y_out.stride(0),
                                         n_split, activation, _ptr(hq), _ptr(hsf), hq.shape[1] * 2, dest_col0,
                                         _ptr(amax_out), M, N, K, _stream()), "mxfp4_linear_split_out")
@@ -482,12 +543,12 @@ def solrl_select_contrastive(rewards: torch.Tensor, K: int, seeds: torch.Tensor 
     if rewards.dtype != torch.float32 or rewards.dim() != 2 or not rewards.is_contiguous():
         raise ValueError("rewards must be a dense 2-D float32 tensor")
     P, N = rewards.shape
-    idx = torch.empty((P, K), dtype=torch.int32, device=rewards.device)
+    idx = _empty((P, K), torch.int32, rewards.device)
     sel = None
     if seeds is not None:
         if seeds.dtype != torch.int64 or tuple(seeds.shape) != (P, N) or not seeds.is_contiguous():
             raise ValueError("seeds must be a dense [P, N] int64 tensor")
-        sel = torch.empty((P, K), dtype=torch.int64, device=rewards.device)
+        sel = _empty((P, K), torch.int64, rewards.device)
     adv = torch.empty_like(rewards) if with_advantages else None
     _check(lib().solrl_select_contrastive(_ptr(rewards), _ptr(seeds), P, N, K, _ptr(idx), _ptr(sel), _ptr(adv),
                                           _stream()), "solrl_select_contrastive")
@@ -502,8 +563,8 @@ def solrl_rank_consistency(ref: torch.Tensor, proxy: torch.Tensor, k: int):
     if ref.shape != proxy.shape:
         raise ValueError("shapes differ")
     P, N = ref.shape
-    counts = torch.empty((P, 4), dtype=torch.int64, device=ref.device)
-    metrics = torch.empty((P, 4), dtype=torch.float32, device=ref.device)
+    counts = _empty((P, 4), torch.int64, ref.device)
+    metrics = _empty((P, 4), torch.float32, ref.device)
     _check(lib().solrl_rank_consistency(_ptr(ref), _ptr(proxy), P, N, k, _ptr(counts), _ptr(metrics), _stream()),
            "solrl_rank_consistency")
     return counts, metrics
@@ -528,8 +589,8 @@ def mxfp4_linear_quantized_out(xq, xsf, wq, wsf, bias, activation: int, amax_out
     M, K = xq.shape[0], xq.shape[1] * 2
     N = wq.shape[0]
     if out is None:
-        out = (torch.empty((M, N // 2), dtype=torch.uint8, device=xq.device),
-               torch.empty(mxfp4_scale_bytes(M, N), dtype=torch.uint8, device=xq.device))
+        out = (_empty((M, N // 2), torch.uint8, xq.device),
+               _empty(mxfp4_scale_bytes(M, N), torch.uint8, xq.device))
     hq, hsf = out
     _check(lib().mxfp4_linear_quantized_out(_ptr(xq), _ptr(xsf), _ptr(wq), _ptr(wsf), _ptr(bias), activation, _ptr(hq),
                                             _ptr(hsf), _ptr(amax_out), M, N, K, _stream()), "mxfp4_linear_quantized_out")
@@ -543,7 +604,7 @@ def bf16_linear(x, w, bias=None, out: torch.Tensor | None = None):
     M, K = x.shape
     N = w.shape[0]
     if out is None:
-        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+        out = _empty((M, N), torch.bfloat16, x.device)
     _check(lib().bf16_linear(_ptr(x), _ptr(w), _ptr(bias), _ptr(out), M, N, K, x.stride(0), w.stride(0),
                              out.stride(0), _stream()), "bf16_linear")
     return out
@@ -556,9 +617,9 @@ def nvfp4_quantize_linear(x, wq, wsf, w_tscale, bias=None, workspace: torch.Tens
     M, K = x.shape
     N = wq.shape[0]
     if workspace is None:
-        workspace = torch.empty(linear_workspace_bytes(M, N, K), dtype=torch.uint8, device=x.device)
+        workspace = _empty(linear_workspace_bytes(M, N, K), torch.uint8, x.device)
     if out is None:
-        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+        out = _empty((M, N), torch.bfloat16, x.device)
     _check(lib().nvfp4_quantize_linear(_ptr(x), x.stride(0), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
                                        _ptr(out), M, N, K, out.stride(0), _ptr(workspace), workspace.numel(),
                                        _stream()), "nvfp4_quantize_linear")
@@ -588,7 +649,7 @@ def nvfp4_quantize_linear_static(x, wq, wsf, w_tscale, bias=None, out: torch.Ten
     M, K = x.shape
     N = wq.shape[0]
     if out is None:
-        out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+        out = _empty((M, N), torch.bfloat16, x.device)
     _check(lib().nvfp4_quantize_linear_static(_ptr(x), x.stride(0), _ptr(wq), _ptr(wsf), _ptr(w_tscale), _ptr(bias),
                                               _ptr(out), M, N, K, out.stride(0), _stream()),
            "nvfp4_quantize_linear_static")
@@ -614,3 +675,11 @@ def sol_set_wait_limit_cycles(cycles: int) -> None:
 def sol_test_hold_loads(on: bool) -> None:
     """Test hook: while on, the pair GEMM kernels issue no loads and their waits run into the limit."""
     _check(lib().sol_test_hold_loads(1 if on else 0), "sol_test_hold_loads")
+
+
+# every public entry checks the guard bands of what it allocated (a no-op outside guard mode)
+for _name, _fn in list(globals().items()):
+    if (isinstance(_fn, types.FunctionType) and _fn.__module__ == __name__ and not _name.startswith("_")
+            and _name not in ("lib", "guard_mode", "check_guards", "status_string")):
+        globals()[_name] = _guarded(_fn)
+del _name, _fn

@@ -236,3 +236,27 @@ def test_diagnostic_build_of_the_gemm_kernels_compiles(tmp_path):
         flags = ["-DSOL_TUNING"] + (["-DSOL_SPAN"] if src == "gemm_pair_fp4.cu" else [])  # + cycle / time span of CTA 0
         subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-std=c++17", *flags, "-c",
                         "-o", str(tmp_path / (src + ".o")), os.path.join(csrc, src)], check=True)
+
+
+def test_guard_mode_of_the_binding_catches_a_write_past_an_output(monkeypatch):
+    """SOL_NVFP4_GUARD=1 puts 4 KB bands round every output the binding allocates and checks them after each
+    call; here on host tensors: intact bands pass, one byte behind the buffer is reported."""
+    import torch
+    from paper_2604_06916_b200 import binding as B
+
+    monkeypatch.setenv("SOL_NVFP4_GUARD", "1")
+    t = B._empty((3, 5), torch.bfloat16, "cpu")
+    assert t.shape == (3, 5) and t.dtype == torch.bfloat16
+    assert t.data_ptr() - B._guard_pending[-1][0].data_ptr() == B.GUARD_BYTES   # keeps the allocation's alignment
+    t.fill_(1.0)                                   # writing the whole buffer leaves the bands alone
+    B.check_guards("intact")
+    u = B._empty(7, torch.uint8, "cpu")
+    raw, nbytes = B._guard_pending[-1]
+    assert nbytes == 7 and u.numel() == 7
+    raw[B.GUARD_BYTES + nbytes] = 0
+    with pytest.raises(AssertionError, match="back band"):
+        B.check_guards("past the end")
+    assert not B._guard_pending                    # forgotten after the check
+    monkeypatch.setenv("SOL_NVFP4_GUARD", "0")
+    B._empty((2, 2), torch.float32, "cpu")
+    assert not B._guard_pending                    # off: plain allocations, nothing to check
