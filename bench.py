@@ -305,6 +305,7 @@ class LegTimer:
     def __init__(self, torch, replicas, dev, dist, sampler, steps, min_s, rounds):
         self.torch, self.replicas, self.dev, self.dist = torch, replicas, dev, dist
         self.sampler, self.steps, self.min_s, self.rounds = sampler, steps, min_s, rounds
+        self.nvtx = os.environ.get("SOL_BENCH_NVTX", "0") not in ("", "0")
 
     def barrier(self):
         if self.dist is not None:
@@ -341,7 +342,11 @@ class LegTimer:
         for rnd in range(self.rounds):
             k = rnd % len(names)
             for n in names[k:] + names[:k]:
+                if self.nvtx:                 # a named range per region, for `ncu --nvtx --nvtx-include <leg>/`
+                    self.torch.cuda.nvtx.range_push(n)
                 ms, secs, win = self.region(legs[n], blocks[n])
+                if self.nvtx:
+                    self.torch.cuda.nvtx.range_pop()
                 out[n]["per_round"].append(ms)
                 out[n]["region_s"].append(secs)
                 out[n]["windows"].append(win)
