@@ -291,12 +291,15 @@ attention_kernel(const __grid_constant__ CUtensorMap tm_qa, const __grid_constan
             const float alpha = move ? ex2(m - m_new) : 1.0f;   // 0 on the first tile (m = -inf)
             if (tracer) ATTN_TRACE(6, j);
             float sum = 0.0f;
+            const uint64_t c2 = qmath::f32x2(p.scale_log2, p.scale_log2), nm2 = qmath::f32x2(-m_new, -m_new);
 #pragma unroll
             for (int c = 0; c < 4; ++c)
 #pragma unroll
                 for (int e = 0; e < 32; e += 2) {
-                    const float p0 = ex2(fmaf(__uint_as_float(s[c][e]), p.scale_log2, -m_new));
-                    const float p1 = ex2(fmaf(__uint_as_float(s[c][e + 1]), p.scale_log2, -m_new));
+                    // s c - m for two scores in one two-lane FMA (each lane rounded as the scalar form would be)
+                    float x0, x1;
+                    qmath::f32x2_split(qmath::fma2(qmath::f32x2(__uint_as_float(s[c][e]), __uint_as_float(s[c][e + 1])), c2, nm2), x0, x1);
+                    const float p0 = ex2(x0), p1 = ex2(x1);
                     sum += p0 + p1;
                     s[c][e >> 1] = pack_bf16(p0, p1);  // 16 words per 32 keys, packed in place
                 }
